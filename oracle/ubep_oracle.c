@@ -1,0 +1,459 @@
+/*
+ * CPU oracle for MoE token dispatch / combine with virtual expert-parallel ranks.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain definition of what the
+ * dispatch/combine hot path computes.  Only the tests, the smoke check and the
+ * benchmark's cpu_baseline / reference legs may build or call it.  It shares no
+ * code, header, table or constant with the CUDA library and never calls it.
+ *
+ * What is defined here, and the passages of the paper it follows:
+ *   - dispatch routes every token to the locations of its selected experts and
+ *     combine gathers the expert outputs back into token order (Sec. 2.3,
+ *     "Deploying MoE on CM384");
+ *   - every destination rank owns a receive region partitioned by source rank
+ *     and expert whose ranges follow from the per-expert token counts of each
+ *     source rank alone (Sec. 2.3) -- `cnt`, `src_offset`;
+ *   - the counts are prefix-summed into offsets (Sec. 2.3 phase 5; Sec. 3.2
+ *     TokenCnt / CalCumSum) and the rows end up contiguous per expert
+ *     (Sec. 2.3 phase 5, Token-Reordering);
+ *   - senders store rows straight into the pre-partitioned destination memory
+ *     (Sec. 4, "Global Load/Store for Point-to-Point Synchronization").
+ * The paper gives no numerics for combine, no FP8 format and no per-rank token
+ * de-duplication; those follow the build's stated readings (one fp32 fused
+ * multiply-add per slot in slot order and one final round-to-nearest-even to
+ * bf16; e4m3 payload with one fp32 scale per 128 channels; one row per
+ * (token, rank) in dedup mode).
+ *
+ * Pins (tests, no GPU): literal brute force of the definitions on tiny inputs,
+ * numpy bincount / cumsum / stable argsort, an exhaustive nearest-code search
+ * over all 256 e4m3 codes, torch's CPU float8 cast for in-range values, closed
+ * forms (y == 1, identity experts round trip), a float64 error bound, and the
+ * post-condition of the prefix-sum search (Algorithm 1) against searchsorted.
+ * Parity unpinned: none of the functions below.
+ *
+ * Notation: T tokens, H hidden size, E physical experts, R ranks, L = E / R
+ * experts per rank, k = top-k, S source ranks.  All arrays are row-major.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORC_OK 0
+#define ORC_ERR_ARG (-1)
+#define ORC_ERR_DUPLICATE (-2)
+#define ORC_ERR_CAPACITY (-3)
+
+/* ------------------------------------------------------------------ scalars */
+
+static float bf16_to_f32(uint16_t b)
+{
+    uint32_t u = (uint32_t)b << 16;
+    float f;
+    memcpy(&f, &u, 4);
+    return f;
+}
+
+/* fp32 -> bf16, round to nearest, ties to even; NaN stays a (quiet) NaN. */
+static uint16_t f32_to_bf16_rne(float f)
+{
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x0040u);
+    uint32_t lsb = (u >> 16) & 1u;
+    u += 0x7fffu + lsb;
+    return (uint16_t)(u >> 16);
+}
+
+uint16_t orc_f32_to_bf16(float f) { return f32_to_bf16_rne(f); }
+float orc_bf16_to_f32(uint16_t b) { return bf16_to_f32(b); }
+
+/*
+ * fp32 -> FP8 e4m3 ("fn" flavour: bias 7, no infinities, largest finite 448,
+ * subnormal step 2^-9).  Round to nearest even onto that grid; magnitudes above
+ * 448 (and infinities) saturate to +-448; NaN -> 0x7F; the sign of zero is kept.
+ */
+uint8_t orc_f32_to_e4m3(float v)
+{
+    if (v != v) return 0x7f;
+    uint8_t sign = signbit(v) ? 0x80 : 0x00;
+    float a = fabsf(v);
+    if (a > 448.0f) return sign | 0x7e;
+    if (a < 0.015625f) {                      /* below 2^-6: subnormal codes 0..7, or 8 */
+        float q = nearbyintf(ldexpf(a, 9));   /* exact scaling, then RNE to an integer  */
+        return sign | (uint8_t)q;             /* q == 8 is the smallest normal, code 8  */
+    }
+    int e;
+    (void)frexpf(a, &e);                      /* a = m * 2^e, m in [0.5, 1)             */
+    e -= 1;                                   /* a = m' * 2^e, m' in [1, 2)             */
+    float q = nearbyintf(ldexpf(a, 3 - e));   /* in [8, 16]; 16 carries into exponent   */
+    int qi = (int)q;
+    if (qi == 16) { qi = 8; e += 1; }
+    return sign | (uint8_t)(((e + 7) << 3) | (qi - 8));
+}
+
+float orc_e4m3_to_f32(uint8_t c)
+{
+    int s = c >> 7, e = (c >> 3) & 15, m = c & 7;
+    float v;
+    if (e == 15 && m == 7) return NAN;
+    if (e == 0) v = ldexpf((float)m, -9);
+    else v = ldexpf((float)(8 + m), e - 10);
+    return s ? -v : v;
+}
+
+/* ------------------------------------------------- step 1: expert-id resolve */
+/*
+ * Logical expert id -> physical expert slot.  A logical expert with several
+ * physical copies sends token t to copy (t mod ncopies).  -1 (empty slot) stays
+ * -1.  phys is [E_log][C]; ncopies is [E_log].
+ */
+int orc_resolve_ids(const int32_t *topk_idx, int T, int k, const int32_t *phys,
+                    const int32_t *ncopies, int E_log, int C, int32_t *out)
+{
+    for (int t = 0; t < T; ++t)
+        for (int j = 0; j < k; ++j) {
+            int32_t l = topk_idx[(size_t)t * k + j];
+            if (l < 0) { out[(size_t)t * k + j] = -1; continue; }
+            if (l >= E_log) return ORC_ERR_ARG;
+            int nc = ncopies[l];
+            if (nc < 1 || nc > C) return ORC_ERR_ARG;
+            out[(size_t)t * k + j] = phys[(size_t)l * C + (t % nc)];
+        }
+    return ORC_OK;
+}
+
+/* --------------------------------------------------- step 2: rank of a token */
+/* Source rank of token t: the s with floor(s*T/S) <= t < floor((s+1)*T/S). */
+int orc_source_rank(int t, int T, int S)
+{
+    for (int s = 0; s < S; ++s) {
+        int64_t lo = (int64_t)s * T / S, hi = (int64_t)(s + 1) * T / S;
+        if (t >= lo && t < hi) return s;
+    }
+    return -1;
+}
+
+/* ------------------------------------------- steps 3-5: counts, offsets, rows */
+/*
+ * ids          [T][k]  physical expert id or -1; ids of one token are distinct
+ * cnt          [S][E]  tokens of source rank s that select expert p
+ * num_tokens_per_expert [E]
+ * is_token_in_rank [T][R] (bytes)   num_tokens_per_rank [R] (distinct tokens)
+ * expert_offset [E]   exclusive sum of num_tokens_per_expert inside the rank
+ * src_offset   [S][E] expert_offset[p] + sum_{s' < s} cnt[s'][p]
+ * num_rows_per_rank [R]
+ * slot_row     [T][k] region-local destination row of slot (t, j); -1 if empty
+ * expert_rows  [R][er_cap]  dedup mode only (may be NULL otherwise): for every
+ *              local expert, at expert_offset[p], the ascending region rows of
+ *              the tokens that select it
+ *
+ * dedup == 0: region r holds, expert after expert, one row per (token, slot),
+ *             ascending token id inside an expert.
+ * dedup == 1: region r holds one row per distinct token routed to r, ascending
+ *             token id; slots of one token on the same rank share that row.
+ */
+int orc_layout(const int32_t *ids, int T, int k, int E, int R, int S, int dedup,
+               int32_t *cnt, int32_t *num_tokens_per_expert, uint8_t *is_token_in_rank,
+               int32_t *num_tokens_per_rank, int32_t *expert_offset, int32_t *src_offset,
+               int32_t *num_rows_per_rank, int32_t *slot_row, int32_t *expert_rows, int er_cap)
+{
+    if (T < 0 || k < 1 || E < 1 || R < 1 || S < 1 || E % R != 0) return ORC_ERR_ARG;
+    const int L = E / R;
+
+    /* preconditions: ids in range, distinct within a token */
+    for (int t = 0; t < T; ++t)
+        for (int j = 0; j < k; ++j) {
+            int32_t p = ids[(size_t)t * k + j];
+            if (p < -1 || p >= E) return ORC_ERR_ARG;
+            if (p < 0) continue;
+            for (int i = 0; i < j; ++i)
+                if (ids[(size_t)t * k + i] == p) return ORC_ERR_DUPLICATE;
+        }
+
+    /* step 3: counts */
+    memset(cnt, 0, sizeof(int32_t) * (size_t)S * E);
+    memset(num_tokens_per_expert, 0, sizeof(int32_t) * (size_t)E);
+    memset(is_token_in_rank, 0, (size_t)T * R);
+    memset(num_tokens_per_rank, 0, sizeof(int32_t) * (size_t)R);
+    for (int t = 0; t < T; ++t) {
+        int s = orc_source_rank(t, T, S);
+        for (int j = 0; j < k; ++j) {
+            int32_t p = ids[(size_t)t * k + j];
+            if (p < 0) continue;
+            cnt[(size_t)s * E + p] += 1;
+            num_tokens_per_expert[p] += 1;
+            is_token_in_rank[(size_t)t * R + p / L] = 1;
+        }
+    }
+    for (int t = 0; t < T; ++t)
+        for (int r = 0; r < R; ++r)
+            num_tokens_per_rank[r] += is_token_in_rank[(size_t)t * R + r];
+
+    /* offsets: prefix sums inside each rank's region, then over source ranks */
+    for (int r = 0; r < R; ++r) {
+        int32_t run = 0;
+        for (int l = 0; l < L; ++l) {
+            expert_offset[r * L + l] = run;
+            run += num_tokens_per_expert[r * L + l];
+        }
+        num_rows_per_rank[r] = dedup ? num_tokens_per_rank[r] : run;
+    }
+    for (int p = 0; p < E; ++p) {
+        int32_t run = expert_offset[p];
+        for (int s = 0; s < S; ++s) {
+            src_offset[(size_t)s * E + p] = run;
+            run += cnt[(size_t)s * E + p];
+        }
+    }
+
+    /* rows: walk tokens in ascending order; `seen` counts earlier arrivals */
+    if (!dedup) {
+        int32_t *seen = (int32_t *)calloc((size_t)S * E, sizeof(int32_t));
+        if (!seen) return ORC_ERR_ARG;
+        for (int t = 0; t < T; ++t) {
+            int s = orc_source_rank(t, T, S);
+            for (int j = 0; j < k; ++j) {
+                int32_t p = ids[(size_t)t * k + j];
+                if (p < 0) { slot_row[(size_t)t * k + j] = -1; continue; }
+                slot_row[(size_t)t * k + j] =
+                    src_offset[(size_t)s * E + p] + seen[(size_t)s * E + p];
+                seen[(size_t)s * E + p] += 1;
+            }
+        }
+        free(seen);
+    } else {
+        int32_t *rows_in_rank = (int32_t *)calloc((size_t)R, sizeof(int32_t));
+        int32_t *seen = (int32_t *)calloc((size_t)E, sizeof(int32_t));
+        if (!rows_in_rank || !seen) { free(rows_in_rank); free(seen); return ORC_ERR_ARG; }
+        for (int t = 0; t < T; ++t) {
+            for (int r = 0; r < R; ++r) {
+                if (!is_token_in_rank[(size_t)t * R + r]) continue;
+                int32_t row = rows_in_rank[r]++;
+                for (int j = 0; j < k; ++j) {
+                    int32_t p = ids[(size_t)t * k + j];
+                    if (p >= 0 && p / L == r) {
+                        slot_row[(size_t)t * k + j] = row;
+                        if (expert_rows) {
+                            int32_t at = expert_offset[p] + seen[p];
+                            if (at >= er_cap) { free(rows_in_rank); free(seen); return ORC_ERR_CAPACITY; }
+                            expert_rows[(size_t)r * er_cap + at] = row;
+                        }
+                        seen[p] += 1;
+                    }
+                }
+            }
+            for (int j = 0; j < k; ++j)
+                if (ids[(size_t)t * k + j] < 0) slot_row[(size_t)t * k + j] = -1;
+        }
+        free(rows_in_rank);
+        free(seen);
+    }
+    return ORC_OK;
+}
+
+/* ------------------------------------------------------ step 6: FP8 payload */
+/*
+ * One row of H bf16 channels -> H e4m3 bytes + H/128 fp32 scales.  Per group of
+ * 128 consecutive channels, all in IEEE fp32 without contraction:
+ *   a = max |x| ; a' = max(a, 1e-4) ; scale = a' / 448 ; inv = 448 / a' ;
+ *   q = e4m3( x * inv ).
+ */
+int orc_fp8_quantize_row(const uint16_t *x, int H, uint8_t *q, float *scale)
+{
+    if (H % 128 != 0) return ORC_ERR_ARG;
+    for (int g = 0; g < H / 128; ++g) {
+        float a = 0.0f;
+        for (int c = 0; c < 128; ++c) {
+            float v = fabsf(bf16_to_f32(x[g * 128 + c]));
+            if (v > a) a = v;
+        }
+        float a1 = a > 1e-4f ? a : 1e-4f;
+        volatile float sc = a1 / 448.0f;
+        volatile float inv = 448.0f / a1;
+        scale[g] = sc;
+        for (int c = 0; c < 128; ++c) {
+            volatile float prod = bf16_to_f32(x[g * 128 + c]) * inv;
+            q[g * 128 + c] = orc_f32_to_e4m3(prod);
+        }
+    }
+    return ORC_OK;
+}
+
+/* --------------------------------------------------- steps 4-5: row contents */
+/*
+ * Fill the receive regions.  payload: 0 = bf16 rows (2H bytes), 1 = e4m3 rows
+ * (H bytes) + scales [R][cap][H/128].  Rows at or beyond num_rows_per_rank are
+ * left untouched.
+ *   dedup == 0: recv_src_idx [R][cap], recv_weight [R][cap]
+ *   dedup == 1: recv_src_idx [R][cap], recv_topk_idx [R][cap][k] (local expert
+ *               id or -1), recv_topk_w [R][cap][k] (weight or 0)
+ * Returns ORC_ERR_CAPACITY if a region needs more than cap rows.
+ */
+int orc_dispatch(const uint16_t *x, const int32_t *ids, const float *topk_w, const int32_t *slot_row,
+                 int T, int H, int k, int E, int R, int cap, int payload, int dedup,
+                 uint8_t *recv_x, float *recv_scale, int32_t *recv_src_idx, float *recv_weight,
+                 int32_t *recv_topk_idx, float *recv_topk_w, int num_threads)
+{
+    if (E % R != 0 || (payload && H % 128 != 0)) return ORC_ERR_ARG;
+    const int L = E / R;
+    const size_t rowB = payload ? (size_t)H : (size_t)H * 2;
+    const int G = H / 128;
+    int err = ORC_OK;
+    (void)num_threads;
+#pragma omp parallel for num_threads(num_threads) schedule(static)
+    for (int t = 0; t < T; ++t) {
+        uint8_t *qrow = NULL;
+        float *srow = NULL;
+        if (payload) {              /* quantised once per token; every copy is identical */
+            qrow = (uint8_t *)malloc((size_t)H);
+            srow = (float *)malloc(sizeof(float) * (size_t)G);
+            orc_fp8_quantize_row(x + (size_t)t * H, H, qrow, srow);
+        }
+        for (int j = 0; j < k; ++j) {
+            int32_t p = ids[(size_t)t * k + j];
+            if (p < 0) continue;
+            int r = p / L;
+            int32_t row = slot_row[(size_t)t * k + j];
+            if (row >= cap) {
+#pragma omp atomic write
+                err = ORC_ERR_CAPACITY;
+                continue;
+            }
+            size_t at = (size_t)r * cap + row;
+            if (payload) {
+                memcpy(recv_x + at * rowB, qrow, rowB);
+                memcpy(recv_scale + at * G, srow, sizeof(float) * (size_t)G);
+            } else {
+                memcpy(recv_x + at * rowB, x + (size_t)t * H, rowB);
+            }
+            recv_src_idx[at] = t;
+            if (!dedup) {
+                recv_weight[at] = topk_w[(size_t)t * k + j];
+            } else {
+                for (int i = 0; i < k; ++i) {
+                    int32_t pi = ids[(size_t)t * k + i];
+                    int here = pi >= 0 && pi / L == r;
+                    recv_topk_idx[at * k + i] = here ? pi % L : -1;
+                    recv_topk_w[at * k + i] = here ? topk_w[(size_t)t * k + i] : 0.0f;
+                }
+            }
+        }
+        free(qrow);
+        free(srow);
+    }
+    return err;
+}
+
+/* ---------------------------------------------------------- step 7: combine */
+/*
+ * out[t][c] = bf16_rne( sum_j w[t][j] * f32(y[rank(p_tj)][slot_row[t][j]][c]) )
+ * accumulated in fp32, one fused multiply-add per slot, slots in order j = 0..k-1.
+ * y is [R][cap][H] bf16.  out64 (optional) receives the same sum in float64.
+ */
+int orc_combine(const uint16_t *y, const int32_t *ids, const float *topk_w, const int32_t *slot_row,
+                int T, int H, int k, int E, int R, int cap, uint16_t *out, double *out64,
+                int num_threads)
+{
+    if (E % R != 0) return ORC_ERR_ARG;
+    const int L = E / R;
+    (void)num_threads;
+#pragma omp parallel for num_threads(num_threads) schedule(static)
+    for (int t = 0; t < T; ++t) {
+        for (int c = 0; c < H; ++c) {
+            float acc = 0.0f;
+            double acc64 = 0.0;
+            for (int j = 0; j < k; ++j) {
+                int32_t p = ids[(size_t)t * k + j];
+                int32_t row = slot_row[(size_t)t * k + j];
+                if (p < 0 || row < 0) continue;
+                size_t at = ((size_t)(p / L) * cap + row) * H + c;
+                float v = bf16_to_f32(y[at]);
+                acc = fmaf(topk_w[(size_t)t * k + j], v, acc);
+                acc64 += (double)topk_w[(size_t)t * k + j] * (double)v;
+            }
+            if (out) out[(size_t)t * H + c] = f32_to_bf16_rne(acc);
+            if (out64) out64[(size_t)t * H + c] = acc64;
+        }
+    }
+    return ORC_OK;
+}
+
+/* ------------------------------------------ Algorithm 1: prefix-sum search */
+/*
+ * Quaternary search over the expert space (Sec. 3.3, Algorithm 1).  `order` is
+ * the (re-mapped) expert sequence of length n and counts[e] the tokens sent to
+ * expert e; the global send sequence is the concatenation of the experts'
+ * tokens in that order.  Finds the position i whose cumulative range covers
+ * target, i.e. C(i) <= target < C(i+1) with C(i) = sum_{i' < i} counts[order[i']],
+ * and the offset target - C(i).  C(.) stands for the paper's VectorCount of
+ * sequence entries below a pivot.
+ *
+ * Reading of the printed algorithm: as printed the gap ceil((R-L)/4) never drops
+ * below 1 once R - L = 1 and pivots L + i*gap can pass R; here the loop runs
+ * while R - L > 1, pivots are clamped to R, and the invariant
+ * C(L) <= target < C(R) is kept.  Returns 0 and fills *pos / *offset / *iters,
+ * or 1 if target is at or past the end of the sequence (no work for the caller).
+ */
+static int64_t cum_before(const int32_t *order, const int32_t *counts, int upto)
+{
+    int64_t c = 0;
+    for (int i = 0; i < upto; ++i) c += counts[order[i]];
+    return c;
+}
+
+int orc_quaternary_search(const int32_t *order, const int32_t *counts, int n, int64_t target,
+                          int32_t *pos, int64_t *offset, int32_t *iters)
+{
+    int lo = 0, hi = n, it = 0;
+    int64_t c_lo = 0;
+    if (target < 0 || target >= cum_before(order, counts, n)) return 1;
+    while (hi - lo > 1) {
+        int gap = (hi - lo + 3) / 4;
+        int piv[5];
+        int64_t c[5];
+        piv[0] = lo; c[0] = c_lo;
+        for (int i = 1; i <= 3; ++i) {
+            piv[i] = lo + i * gap;
+            if (piv[i] > hi) piv[i] = hi;
+            c[i] = cum_before(order, counts, piv[i]);
+        }
+        piv[4] = hi;
+        int q = 4;
+        for (int i = 1; i <= 3; ++i)
+            if (target < c[i]) { q = i; break; }
+        lo = piv[q - 1];
+        hi = piv[q];
+        c_lo = c[q - 1];
+        ++it;
+    }
+    *pos = lo;
+    *offset = target - cum_before(order, counts, lo);
+    if (iters) *iters = it;
+    return 0;
+}
+
+/*
+ * Expert re-mapping by logical matrix transposition (Sec. 3.3): ids 0..n-1 fill
+ * a matrix with `rows` rows row-major (ceil(n/rows) columns); reading it column
+ * by column, skipping the padding, gives the visiting order.
+ */
+void orc_stride_remap(int n, int rows, int32_t *order)
+{
+    int cols = (n + rows - 1) / rows, w = 0;
+    for (int c = 0; c < cols; ++c)
+        for (int r = 0; r < rows; ++r) {
+            int id = r * cols + c;
+            if (id < n) order[w++] = id;
+        }
+}
+
+/*
+ * Token-level load partition (Sec. 3.3): the send sequence of `total` tokens is
+ * cut into `workers` contiguous slices whose sizes differ by at most one.
+ * Slice w covers [floor(w*total/workers), floor((w+1)*total/workers)).
+ */
+void orc_equal_slices(int64_t total, int workers, int64_t *begin)
+{
+    for (int w = 0; w <= workers; ++w) begin[w] = (int64_t)w * total / workers;
+}
