@@ -1,0 +1,414 @@
+#!/usr/bin/env python
+"""Benchmark of the MoE dispatch + combine hot path on B200.
+
+One "step" = one ubep_dispatch followed by one ubep_combine over one batch of synthetic
+input of the decode-shaped configuration (T=512, H=7168 bf16, E=256 over R=32 virtual
+ranks, top-8, per-rank token de-duplication).  `value` is the algorithmic bytes the two
+calls must move divided by the measured time (GB/s, whole job), next to microseconds per
+layer.  Rotating buffer sets larger than L2 keep every step cold.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload decode|prefill|...]
+
+For N > 1 launch with torchrun: every rank runs an independent replica on its own GPU
+(the path has no exchange step between GPUs), timing is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+for p in (ROOT, os.path.join(ROOT, "tests")):
+    if p not in sys.path:
+        sys.path.insert(0, p)
+
+import numpy as np
+
+METRIC = "dispatch+combine achieved HBM GB/s (algorithmic bytes / time); us/layer beside it"
+L2_BYTES = 126e6
+
+
+def algorithmic_bytes(cfg, n_rows: int):
+    """Bytes the method must move (counts and flags are < 0.2 % and left out).
+    dispatch: read every token once + ids and weights + write N rows (payload, source id, weight);
+    combine: read N expert-output rows + weights and rows handle + write T rows."""
+    T, H, k = cfg.T, cfg.H, cfg.k
+    rowB = H + 4 * (H // 128) if cfg.payload else 2 * H
+    disp = T * H * 2 + T * k * 8 + n_rows * (rowB + 8)
+    comb = n_rows * 2 * H + T * k * 8 + T * 2 * H
+    return disp, comb
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.stop_flag = [], set(), False
+        self.max_mhz = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if self.nv is None:
+            return
+        nv = self.nv
+        names = {"hw_slowdown": nv.nvmlClocksThrottleReasonHwSlowdown,
+                 "hw_thermal_slowdown": nv.nvmlClocksThrottleReasonHwThermalSlowdown,
+                 "sw_thermal_slowdown": nv.nvmlClocksThrottleReasonSwThermalSlowdown,
+                 "sw_power_cap": nv.nvmlClocksThrottleReasonSwPowerCap}
+        while not self.stop_flag:
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for n, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(n)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def result(self):
+        self.stop_flag = True
+        if self.is_alive():
+            self.join(timeout=1.0)
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_index: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_index])
+        except Exception:
+            return local_index
+    return local_index
+
+
+# ------------------------------------------------------------------ reference (oracle) arm
+
+def run_reference(args, cfg, rank: int):
+    """Times the CPU oracle, as it stands, on the host cores; rank 0 only."""
+    if rank != 0:
+        return
+    import oracle
+    import harness as Hn
+    from paper_2607_06202_b200 import workload as W
+    wl = W.make_workload(cfg)
+    cores = oracle.host_cores()
+    ids, lay, cap, _ = Hn.oracle_reference(wl)
+    y = W.make_expert_outputs(cfg, cap)
+    n_rows = int(lay.num_rows_per_rank.sum())
+    disp_b, comb_b = algorithmic_bytes(cfg, n_rows)
+
+    def step():
+        ids_ = wl.topk_idx if wl.phys is None else oracle.resolve_ids(wl.topk_idx, wl.phys, wl.ncopies)
+        lay_ = oracle.layout(ids_, cfg.E, cfg.R, cfg.S, cfg.dedup, er_cap=cap * min(cfg.k, cfg.L))
+        oracle.dispatch(wl.x, ids_, wl.topk_w, lay_.slot_row, cfg.E, cfg.R, cap, cfg.payload, cfg.dedup,
+                        num_threads=cores)
+        oracle.combine(y, ids_, wl.topk_w, lay_.slot_row, cfg.E, cfg.R, num_threads=cores)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / args.steps
+    gbs = (disp_b + comb_b) / dt / 1e9
+    sample = f"the whole {cfg.name} workload (layout + dispatch + combine), {args.steps} passes"
+    line = {"impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "us_per_layer": dt * 1e6,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": workload_config(cfg, n_rows, cap, "host memory"),
+            "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(cfg, n_rows, cap, l2_policy):
+    return {"workload": f"{cfg.name}: T={cfg.T} H={cfg.H} E={cfg.E} R={cfg.R} k={cfg.k} "
+                        f"payload={'fp8_e4m3+f32/128' if cfg.payload else 'bf16'} dedup={cfg.dedup} seed={cfg.seed}",
+            "rows_dispatched": n_rows, "rows_per_rank_cap": cap, "virtual_ranks": cfg.R,
+            "l2": l2_policy, "paper_context": "UBEP on CM384: 73-112 us dispatch at 16-256 ranks (Table 4, other hardware)"}
+
+
+# ------------------------------------------------------------------------------ our arm
+
+def run_ours(args, cfg, rank: int, world: int, local_rank: int):
+    import torch
+    import torch.distributed as dist
+    from paper_2607_06202_b200 import binding as B
+    from paper_2607_06202_b200 import workload as W
+
+    assert torch.cuda.is_available(), "bench.py needs a GPU (there is no CPU fallback)"
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    B.load()
+
+    wl = W.make_workload(cfg)
+    # region capacity from the library's own count pass (TokenCnt only), rounded up to 128 rows
+    probe = B.Buffer(num_ranks=cfg.R, num_experts=cfg.E, hidden=cfg.H, topk=cfg.k, max_tokens=cfg.T,
+                     rows_per_rank_cap=1, num_src_ranks=cfg.S, payload=cfg.payload, dedup=cfg.dedup,
+                     device=local_rank)
+    idx0 = torch.from_numpy(wl.topk_idx.astype(np.int32)).to(dev)
+    if wl.phys is not None:
+        probe.set_replicas(torch.from_numpy(wl.phys).to(dev), torch.from_numpy(wl.ncopies).to(dev))
+    npr, npe, _ = probe.get_dispatch_layout(idx0)
+    rows_per_rank = npr if cfg.dedup else npe.view(cfg.R, cfg.L).sum(1)
+    cap = W.round_up(max(1, int(rows_per_rank.max().item())), 128)
+    n_rows = int(rows_per_rank.sum().item())
+    probe.close()
+    disp_b, comb_b = algorithmic_bytes(cfg, n_rows)
+    y_bits = W.make_expert_outputs(cfg, cap)
+
+    # rotating sets: by the time a set comes round again, several L2s' worth of other data went by
+    def make_set():
+        buf = B.Buffer(num_ranks=cfg.R, num_experts=cfg.E, hidden=cfg.H, topk=cfg.k, max_tokens=cfg.T,
+                       rows_per_rank_cap=cap, num_src_ranks=cfg.S, payload=cfg.payload, dedup=cfg.dedup,
+                       device=local_rank, pipeline=args.pipeline)
+        x = torch.from_numpy(wl.x).view(torch.bfloat16).to(dev)
+        idx = torch.from_numpy(wl.topk_idx.astype(np.int32)).to(dev)
+        w = torch.from_numpy(wl.topk_w).to(dev)
+        if wl.phys is not None:
+            buf.set_replicas(torch.from_numpy(wl.phys).to(dev), torch.from_numpy(wl.ncopies).to(dev))
+        y = torch.from_numpy(y_bits).view(torch.bfloat16).to(dev)
+        out = torch.empty((cfg.T, cfg.H), dtype=torch.bfloat16, device=dev)
+        return dict(buf=buf, x=x, idx=idx, w=w, y=y, out=out)
+
+    touched = disp_b + comb_b
+    nsets = int(min(16, max(4, np.ceil(4 * L2_BYTES / touched) + 1)))
+    sets = [make_set() for _ in range(nsets)]
+    stream = torch.cuda.Stream(device=dev)
+
+    def step(s):
+        B.ubep_dispatch(s["buf"].handle, s["x"], s["idx"], s["w"], cfg.T, stream)
+        B.ubep_combine(s["buf"].handle, s["y"], s["w"], cfg.T, s["out"], stream)
+
+    with torch.cuda.stream(stream):
+        step(sets[0])
+    stream.synchronize()
+    assert sets[0]["buf"].status() == 0
+    first_out = sets[0]["out"].clone()
+
+    # one CUDA graph holds one pass over all sets; the epoch lives on the device, so replays are valid
+    graph = None
+    if not args.no_graph:
+        with torch.cuda.stream(stream):
+            for s in sets:
+                step(s)
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for s in sets:
+                step(s)
+
+    def run_steps(n):
+        done = 0
+        with torch.cuda.stream(stream):
+            if graph is not None:
+                while n - done >= nsets:
+                    graph.replay()
+                    done += nsets
+            while done < n:
+                step(sets[done % nsets])
+                done += 1
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    run_steps(max(args.warmup, 3))
+    barrier()
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    sampler.start()
+    n0 = B.ubep_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+    run_steps(args.steps)
+    with torch.cuda.stream(stream):
+        e1.record(stream)
+    barrier()
+    clocks = sampler.result()
+    total_ms = e0.elapsed_time(e1)
+    launches = 2 * args.steps        # one dispatch kernel + one combine kernel per step
+    if args.pipeline == B.UBEP_PIPELINE_PHASED:
+        launches = 4 * args.steps
+    _ = n0
+    if world > 1:
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * (disp_b + comb_b) / (ms_per_step * 1e-3) / 1e9
+
+    # per-kernel durations, CUDA events on the launching stream, same rotating sets
+    n_k = min(args.steps, 400)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(n_k)]
+    with torch.cuda.stream(stream):
+        for i in range(n_k):
+            s = sets[i % nsets]
+            evs[i][0].record(stream)
+            B.ubep_dispatch(s["buf"].handle, s["x"], s["idx"], s["w"], cfg.T, stream)
+            evs[i][1].record(stream)
+            B.ubep_combine(s["buf"].handle, s["y"], s["w"], cfg.T, s["out"], stream)
+            evs[i][2].record(stream)
+    stream.synchronize()
+    d_us = np.array([e[0].elapsed_time(e[1]) for e in evs]) * 1e3
+    c_us = np.array([e[1].elapsed_time(e[2]) for e in evs]) * 1e3
+    disp_us, comb_us = float(np.mean(d_us)), float(np.mean(c_us))
+
+    # end to end through the C ABI with host buffers: pinned inputs -> device -> dispatch ->
+    # combine over identity experts (bf16 payload) or the synthetic y (FP8) -> host
+    hx = torch.from_numpy(wl.x).view(torch.bfloat16).pin_memory()
+    hidx = torch.from_numpy(wl.topk_idx.astype(np.int32)).pin_memory()
+    hw = torch.from_numpy(wl.topk_w).pin_memory()
+    hout = torch.empty((cfg.T, cfg.H), dtype=torch.bfloat16).pin_memory()
+    n_e = min(args.steps, 200)
+    ee0, ee1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def e2e_step(s):
+        s["x"].copy_(hx, non_blocking=True)
+        s["idx"].copy_(hidx, non_blocking=True)
+        s["w"].copy_(hw, non_blocking=True)
+        B.ubep_dispatch(s["buf"].handle, s["x"], s["idx"], s["w"], cfg.T, stream)
+        yy = s["y"] if cfg.payload else s["buf"].recv_x.view(torch.bfloat16).view(cfg.R, cap, cfg.H)
+        B.ubep_combine(s["buf"].handle, yy, s["w"], cfg.T, s["out"], stream)
+        hout.copy_(s["out"], non_blocking=True)
+
+    with torch.cuda.stream(stream):
+        for i in range(3):
+            e2e_step(sets[i % nsets])
+    barrier()
+    with torch.cuda.stream(stream):
+        ee0.record(stream)
+        for i in range(n_e):
+            e2e_step(sets[i % nsets])
+        ee1.record(stream)
+    barrier()
+    e2e_ms = ee0.elapsed_time(ee1) / n_e
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    h2d = hx.numel() * 2 + hidx.numel() * 4 + hw.numel() * 4
+    d2h = hout.numel() * 2
+    e2e = {"value": world * (disp_b + comb_b) / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s",
+           "us_per_layer": e2e_ms * 1e3, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+           "experts": "synthetic y" if cfg.payload else "identity (y = receive regions)"}
+
+    if rank != 0:
+        return
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except Exception:
+        pass
+    peak = float(peaks.get("hbm_gbs", 6650.0))
+    peak_kind = "measured copy bandwidth (MEASURED_PEAKS.json)" if peaks else "fallback 6650 GB/s"
+    dom = "dispatch" if disp_us >= comb_us else "combine"
+    dom_bytes, dom_us = (disp_b, disp_us) if dom == "dispatch" else (comb_b, comb_us)
+    achieved = dom_bytes / (dom_us * 1e-6) / 1e9
+    traffic = None
+    try:
+        prof = json.load(open(os.path.join(ROOT, "profiles", "traffic.json")))
+        traffic = prof.get(cfg.name, {}).get(dom)
+    except Exception:
+        pass
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_kind": peak_kind, "traffic": traffic,
+                "frac_of_nominal_8TBs": achieved / 8000.0,
+                "dispatch_us": disp_us, "combine_us": comb_us,
+                "dispatch_gbs": disp_b / (disp_us * 1e-6) / 1e9, "combine_gbs": comb_b / (comb_us * 1e-6) / 1e9,
+                "layer_frac_of_peak": ((disp_b + comb_b) / ((disp_us + comb_us) * 1e-6) / 1e9) / peak,
+                "layer_frac_of_nominal_8TBs": ((disp_b + comb_b) / ((disp_us + comb_us) * 1e-6) / 1e9) / 8000.0}
+
+    # the oracle, as it stands, on a bounded sample of the same workload (its result also
+    # cross-checks what the GPU produced for the first buffer set)
+    import oracle
+    import harness as Hn
+    cores = oracle.host_cores()
+    reps, t_cpu = 0, 0.0
+    cap_e = cap * min(cfg.k, cfg.L)
+    want = None
+    while t_cpu < 10.0 and reps < 50:
+        t0 = time.perf_counter()
+        ids_ = wl.topk_idx if wl.phys is None else oracle.resolve_ids(wl.topk_idx, wl.phys, wl.ncopies)
+        lay_ = oracle.layout(ids_, cfg.E, cfg.R, cfg.S, cfg.dedup, er_cap=cap_e)
+        oracle.dispatch(wl.x, ids_, wl.topk_w, lay_.slot_row, cfg.E, cfg.R, cap, cfg.payload, cfg.dedup,
+                        num_threads=cores)
+        want, _ = oracle.combine(y_bits, ids_, wl.topk_w, lay_.slot_row, cfg.E, cfg.R, num_threads=cores)
+        t_cpu += time.perf_counter() - t0
+        reps += 1
+    Hn.check_combine(first_out, want)
+    cpu = {"value": (disp_b + comb_b) * reps / t_cpu / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
+           "us_per_layer": t_cpu / reps * 1e6,
+           "sample": f"the whole {cfg.name} workload (layout + dispatch + combine), {reps} passes, "
+                     f"row copies and combine on {cores} threads"}
+
+    line = {"metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "us_per_layer": ms_per_step * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": workload_config(cfg, n_rows, cap, f"{nsets} rotating buffer sets, "
+                                      f"{nsets * touched / 1e6:.0f} MB touched per cycle (> L2), no flush kernels"),
+            "algorithmic_bytes": {"dispatch": disp_b, "combine": comb_b},
+            "frac_of_peak": value / world / peak, "frac_of_nominal_8TBs": value / world / 8000.0,
+            "cuda_graph": graph is not None, "pipeline": args.pipeline,
+            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="decode")
+    ap.add_argument("--pipeline", type=int, default=0)
+    ap.add_argument("--no-graph", action="store_true")
+    args = ap.parse_args()
+
+    from paper_2607_06202_b200 import workload as W
+    cfg = W.CONFIGS[args.workload]
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        args.steps = args.steps if args.steps is not None else 20
+        args.warmup = args.warmup if args.warmup is not None else 3
+        run_reference(args, cfg, rank)
+        return
+    args.steps = args.steps if args.steps is not None else 20000
+    args.warmup = args.warmup if args.warmup is not None else 200
+    if world > 1:
+        import torch
+        import torch.distributed as dist
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    try:
+        run_ours(args, cfg, rank, world, local_rank)
+    finally:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,202 @@
+/*
+ * ubep.h -- C ABI of the B200 (sm_100a) MoE token dispatch / combine library.
+ *
+ * The expert-parallel ranks are virtual: R disjoint receive regions inside one device
+ * arena that the caller allocates.  The library allocates no device memory, creates no
+ * stream and never synchronises the host except in ubep_status().  Every pointer below
+ * is marked [host] or [dev]; all device pointers must be 16-byte aligned; `cuda_stream`
+ * is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *
+ * Notation: T tokens, H hidden size, E physical experts, R ranks, L = E / R experts per
+ * rank (expert p lives on rank p / L), k = top-k, S source ranks (token t belongs to the
+ * source rank s with floor(s*T/S) <= t < floor((s+1)*T/S)), cap = rows_per_rank_cap.
+ *
+ * All functions return UBEP_OK (0) or a negative error code.  Argument errors are
+ * reported synchronously and nothing is launched.  Conditions found on the device
+ * (a region overflowing its capacity, a bounded flag wait running out, an expert id out
+ * of range) never trap: the kernel records the first such code in a device status word,
+ * skips the offending access and returns; ubep_status() reads and clears that word.
+ */
+#ifndef UBEP_H
+#define UBEP_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ubep_buffer ubep_buffer_t; /* opaque host-side bookkeeping, library-owned */
+
+enum {
+    UBEP_OK = 0,
+    UBEP_ERR_ARG = -1,       /* null / misaligned pointer, size out of range, bad config      */
+    UBEP_ERR_CUDA = -2,      /* a CUDA runtime call failed (see ubep_last_cuda_error)         */
+    UBEP_ERR_CAPACITY = -3,  /* device: a region needs more than cap rows; extra rows dropped */
+    UBEP_ERR_TIMEOUT = -4,   /* device: a bounded wait on a readiness flag ran out            */
+    UBEP_ERR_BAD_INDEX = -5, /* device: an expert id outside [-1, E) was skipped              */
+    UBEP_ERR_ARENA = -6      /* arena too small or not 256-byte aligned                       */
+};
+
+enum { UBEP_PAYLOAD_BF16 = 0, UBEP_PAYLOAD_FP8_E4M3 = 1 };
+
+/* How ubep_dispatch schedules its steps. */
+enum {
+    UBEP_PIPELINE_AUTO = 0,   /* FUSED                                                        */
+    UBEP_PIPELINE_PHASED = 1, /* count -> prefix sums -> scatter as three launches; the        */
+                              /* kernel boundaries play the role of the global barriers of    */
+                              /* the bulk-synchronous dispatch (Sec. 2.3, phases 2-5)         */
+    UBEP_PIPELINE_FUSED = 2,  /* one persistent kernel: count / prefix-sum warps publish      */
+                              /* offsets through release/acquire flags while mover warps      */
+                              /* already stream rows (kernel decomposition, Sec. 3.2)         */
+    UBEP_PIPELINE_LOCAL = 3   /* one persistent kernel in which every CTA derives its offsets */
+                              /* from the whole routing table itself (no flags; small T*k)    */
+};
+
+typedef struct {
+    int32_t num_ranks;         /* R >= 1                                                       */
+    int32_t num_experts;       /* E physical experts, E % R == 0                               */
+    int32_t hidden;            /* H, multiple of 8 (bf16 payload) or of 128 (FP8 payload)      */
+    int32_t topk;              /* k in [1, 32]                                                 */
+    int32_t max_tokens;        /* largest T any call will pass                                 */
+    int32_t rows_per_rank_cap; /* cap: rows each receive region can hold                       */
+    int32_t num_src_ranks;     /* S >= 1 (0 = R)                                               */
+    int32_t payload;           /* UBEP_PAYLOAD_*                                               */
+    int32_t dedup;             /* 0: one row per (token, slot), expert-major;                  */
+                               /* 1: one row per (token, rank), ascending token                */
+    int32_t device;            /* CUDA device ordinal                                          */
+    int32_t pipeline;          /* UBEP_PIPELINE_*                                              */
+    int32_t num_ctas;          /* persistent CTAs / token chunks; 0 = number of SMs            */
+} ubep_config_t;
+
+/* Arrays that live in the arena; ubep_view() returns their device address and shape. */
+enum {
+    UBEP_VIEW_RECV_X = 0,        /* u8  [R, cap, rowB]  rowB = 2H (bf16) or H (FP8)            */
+    UBEP_VIEW_RECV_SCALE = 1,    /* f32 [R, cap, H/128] FP8 payload only                       */
+    UBEP_VIEW_RECV_SRC_IDX = 2,  /* i32 [R, cap]        token id of each row                   */
+    UBEP_VIEW_RECV_WEIGHT = 3,   /* f32 [R, cap]        gate weight of the row (dedup = 0)     */
+    UBEP_VIEW_RECV_TOPK_IDX = 4, /* i32 [R, cap, k]     local expert id or -1  (dedup = 1)     */
+    UBEP_VIEW_RECV_TOPK_W = 5,   /* f32 [R, cap, k]     weight or 0            (dedup = 1)     */
+    UBEP_VIEW_EXPERT_ROWS = 6,   /* i32 [R, er_cap]     per local expert, at expert_offset,    */
+                                 /*                     ascending rows selecting it (dedup = 1)*/
+    UBEP_VIEW_CNT = 7,           /* i32 [S, E]          tokens of source s choosing expert p   */
+    UBEP_VIEW_SRC_OFFSET = 8,    /* i32 [S, E]          expert_offset + sum_{s'<s} cnt         */
+    UBEP_VIEW_EXPERT_OFFSET = 9, /* i32 [E]             exclusive sum of counts inside a rank  */
+    UBEP_VIEW_NUM_TOKENS_PER_EXPERT = 10, /* i32 [E]                                           */
+    UBEP_VIEW_NUM_ROWS_PER_RANK = 11,     /* i32 [R]    rows written to each region            */
+    UBEP_VIEW_NUM_TOKENS_PER_RANK = 12,   /* i32 [R]    distinct tokens routed to each rank    */
+    UBEP_VIEW_SLOT_ROW = 13,     /* i32 [max_tokens, k] region-local row of each slot, or -1;  */
+                                 /*                     the handle ubep_combine uses           */
+    UBEP_VIEW_ARRIVAL = 14,      /* u32 [2, R]          rows landed per region; the half the   */
+                                 /*                     n-th dispatch uses is (n & 1)          */
+    UBEP_VIEW_EPOCH = 15,        /* u32 [1]             dispatches completed on this buffer;   */
+                                 /*                     readiness flags hold this count + 1    */
+                                 /*                     while a dispatch runs, so replaying a  */
+                                 /*                     captured CUDA graph needs no reset     */
+    UBEP_VIEW_COUNT_ = 16
+};
+
+/*
+ * Bytes of device memory the arena needs for this configuration (0 if the configuration
+ * is invalid).  Operation: the receive address space is partitioned once, at
+ * initialisation, so that senders can store rows straight into the destination's memory
+ * (Sec. 4, "Global Load/Store for Point-to-Point Synchronization"; Sec. 2.3).
+ */
+size_t ubep_buffer_bytes(const ubep_config_t *cfg /*[host]*/);
+
+/*
+ * Lay the arrays out inside `dev_arena` ([dev], 256-byte aligned, >= ubep_buffer_bytes)
+ * and zero the flag words (one synchronous memset).  The caller keeps ownership of the
+ * arena and must keep it alive until ubep_buffer_destroy.  *out receives the handle.
+ */
+int ubep_buffer_create(const ubep_config_t *cfg /*[host]*/, void *dev_arena /*[dev]*/,
+                       size_t bytes, ubep_buffer_t **out /*[host]*/);
+
+/* Free the host bookkeeping.  The arena is the caller's and is not touched. */
+int ubep_buffer_destroy(ubep_buffer_t *buf);
+
+/*
+ * Logical -> physical expert table for replicated experts (the paper only names expert
+ * replication as an upper-layer strategy the library accepts, Sec. 6).  Slot (t, j) with
+ * logical id l goes to phys[l][t mod ncopies[l]].  phys [dev] is [E_log, C] int32,
+ * ncopies [dev] is [E_log] int32; both stay owned by the caller and must outlive the calls
+ * that use them.  Passing NULLs removes the table.
+ */
+int ubep_set_replicas(ubep_buffer_t *buf, const int32_t *phys /*[dev]*/,
+                      const int32_t *ncopies /*[dev]*/, int32_t E_log, int32_t C);
+
+/*
+ * Destination-ordering table (Sec. 3.3: the re-mapped expert sequence each worker sends
+ * in).  `order` [host] is a permutation of 0..R-1; worker w issues the copies of one row
+ * in the table's order rotated by w.  Results never depend on it.  NULL = identity.
+ */
+int ubep_set_dest_order(ubep_buffer_t *buf, const int32_t *order /*[host] [R]*/);
+
+/*
+ * TokenCnt only (Sec. 3.2; Sec. 2.3: ranges follow from per-expert counts): counts how
+ * many distinct tokens go to each rank and how many tokens select each expert, and marks
+ * which ranks each token visits.  topk_idx [dev] int32 [T, k] (expert id, or -1 = empty
+ * slot; ids of one token distinct).  Outputs [dev], caller-owned:
+ * num_tokens_per_rank [R], num_tokens_per_expert [E], is_token_in_rank u8 [T, R]
+ * (any of them may be NULL).  One launch on `cuda_stream`.
+ */
+int ubep_get_dispatch_layout(ubep_buffer_t *buf, const int32_t *topk_idx /*[dev]*/, int32_t T,
+                             int32_t *num_tokens_per_rank /*[dev]*/,
+                             int32_t *num_tokens_per_expert /*[dev]*/,
+                             uint8_t *is_token_in_rank /*[dev]*/, void *cuda_stream);
+
+/*
+ * Dispatch (Sec. 2.3 phases 1-5 fused as in Sec. 3.2): counts, prefix-sum offsets, row
+ * assignment, optional FP8 quantisation, and the copy of every token row into the receive
+ * regions of the ranks that host its experts.  x [dev] bf16 [T, H]; topk_idx [dev] int32
+ * [T, k]; topk_w [dev] fp32 [T, k].  Results land in the arena (ubep_view).  Rows at or
+ * beyond a region's row count are not written.  Asynchronous on `cuda_stream`; calls on
+ * one buffer must be stream-ordered.
+ */
+int ubep_dispatch(ubep_buffer_t *buf, const void *x /*[dev]*/, const int32_t *topk_idx /*[dev]*/,
+                  const float *topk_w /*[dev]*/, int32_t T, void *cuda_stream);
+
+/*
+ * Combine (Sec. 2.3: gathers expert outputs and restores the original token order):
+ * out[t] = bf16( sum_j topk_w[t][j] * y[rank of slot j][slot_row[t][j]] ), fp32
+ * accumulation in slot order with one fused multiply-add per slot.  y [dev] bf16
+ * [R, cap, H] is caller-owned and indexed like the receive regions; out [dev] bf16
+ * [T, H].  Uses the slot_row handle left by the last ubep_dispatch on this buffer.
+ */
+int ubep_combine(ubep_buffer_t *buf, const void *y /*[dev]*/, const float *topk_w /*[dev]*/,
+                 int32_t T, void *out /*[dev]*/, void *cuda_stream);
+
+/* Device address and shape (unused dims = 1) of one arena array; valid until destroy. */
+int ubep_view(ubep_buffer_t *buf, int which, void **dev_ptr /*[host]*/, int64_t shape[4] /*[host]*/);
+
+/*
+ * Synchronises the stream of the last call, copies the device status word to
+ * *last_async_status ([host]; UBEP_OK or a UBEP_ERR_* code found on the device) and
+ * clears it.
+ */
+int ubep_status(ubep_buffer_t *buf, int32_t *last_async_status /*[host]*/);
+
+/* Number of non-empty dispatches issued through ubep_dispatch on this buffer so far
+ * (graph replays are not counted; the device-side count is UBEP_VIEW_EPOCH). */
+uint32_t ubep_epoch(const ubep_buffer_t *buf);
+
+/* Kernels launched by this library since it was loaded (all buffers). */
+uint64_t ubep_launch_count(void);
+
+/*
+ * Test hook for the bounded-wait path: the next ubep_dispatch skips the release store of
+ * the readiness flag of token chunk `chunk` (-1 = none), so that the waits on it run out
+ * after about a second, the kernel returns and ubep_status reports UBEP_ERR_TIMEOUT.
+ */
+int ubep_debug_withhold_flag(ubep_buffer_t *buf, int32_t chunk);
+
+/* Text of the last CUDA runtime error seen by this buffer's calls ("" if none). */
+const char *ubep_last_cuda_error(const ubep_buffer_t *buf);
+
+const char *ubep_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* UBEP_H */

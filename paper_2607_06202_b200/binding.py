@@ -1,0 +1,267 @@
+"""ctypes binding of the C-ABI library ``libubep.so`` (see ``include/ubep.h``).
+
+The module-level ``ubep_*`` functions have the names and argument order of the C entry
+points and only marshal arguments (torch tensors -> device pointers, the current torch
+stream -> ``void*``).  ``Buffer`` is a small convenience holder for an arena tensor and its
+views.  PyTorch supplies device memory and streams; every step of dispatch / combine runs
+in the library's kernels.  There is no fallback: if the library is missing, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libubep.so")
+
+UBEP_OK = 0
+UBEP_ERR_ARG, UBEP_ERR_CUDA, UBEP_ERR_CAPACITY, UBEP_ERR_TIMEOUT, UBEP_ERR_BAD_INDEX, UBEP_ERR_ARENA = \
+    -1, -2, -3, -4, -5, -6
+UBEP_PAYLOAD_BF16, UBEP_PAYLOAD_FP8_E4M3 = 0, 1
+UBEP_PIPELINE_AUTO, UBEP_PIPELINE_PHASED, UBEP_PIPELINE_FUSED, UBEP_PIPELINE_LOCAL = 0, 1, 2, 3
+
+VIEW_NAMES = ["recv_x", "recv_scale", "recv_src_idx", "recv_weight", "recv_topk_idx", "recv_topk_w",
+              "expert_rows", "cnt", "src_offset", "expert_offset", "num_tokens_per_expert",
+              "num_rows_per_rank", "num_tokens_per_rank", "slot_row", "arrival", "epoch"]
+_VIEW_DTYPES = [torch.uint8, torch.float32, torch.int32, torch.float32, torch.int32, torch.float32,
+                torch.int32, torch.int32, torch.int32, torch.int32, torch.int32, torch.int32, torch.int32,
+                torch.int32, torch.int32, torch.int32]
+
+# every symbol include/ubep.h declares
+EXPORTS = ["ubep_buffer_bytes", "ubep_buffer_create", "ubep_buffer_destroy", "ubep_set_replicas",
+           "ubep_set_dest_order", "ubep_get_dispatch_layout", "ubep_dispatch", "ubep_combine", "ubep_view",
+           "ubep_status", "ubep_epoch", "ubep_launch_count", "ubep_debug_withhold_flag",
+           "ubep_last_cuda_error", "ubep_strerror"]
+
+
+class ubep_config_t(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("num_ranks", "num_experts", "hidden", "topk", "max_tokens", "rows_per_rank_cap",
+                 "num_src_ranks", "payload", "dedup", "device", "pipeline", "num_ctas")]
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Load libubep.so; raises if it has not been built (no CPU or eager fallback exists)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2607_06202_b200.build`")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, u32, u64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_uint32, ctypes.c_uint64
+    cfgp = ctypes.POINTER(ubep_config_t)
+    lib.ubep_buffer_bytes.restype, lib.ubep_buffer_bytes.argtypes = ctypes.c_size_t, [cfgp]
+    lib.ubep_buffer_create.restype = ctypes.c_int
+    lib.ubep_buffer_create.argtypes = [cfgp, vp, ctypes.c_size_t, ctypes.POINTER(vp)]
+    lib.ubep_buffer_destroy.restype, lib.ubep_buffer_destroy.argtypes = ctypes.c_int, [vp]
+    lib.ubep_set_replicas.restype, lib.ubep_set_replicas.argtypes = ctypes.c_int, [vp, vp, vp, i32, i32]
+    lib.ubep_set_dest_order.restype, lib.ubep_set_dest_order.argtypes = ctypes.c_int, [vp, vp]
+    lib.ubep_get_dispatch_layout.restype = ctypes.c_int
+    lib.ubep_get_dispatch_layout.argtypes = [vp, vp, i32, vp, vp, vp, vp]
+    lib.ubep_dispatch.restype, lib.ubep_dispatch.argtypes = ctypes.c_int, [vp, vp, vp, vp, i32, vp]
+    lib.ubep_combine.restype, lib.ubep_combine.argtypes = ctypes.c_int, [vp, vp, vp, i32, vp, vp]
+    lib.ubep_view.restype = ctypes.c_int
+    lib.ubep_view.argtypes = [vp, ctypes.c_int, ctypes.POINTER(vp), ctypes.POINTER(ctypes.c_int64)]
+    lib.ubep_status.restype, lib.ubep_status.argtypes = ctypes.c_int, [vp, ctypes.POINTER(i32)]
+    lib.ubep_epoch.restype, lib.ubep_epoch.argtypes = u32, [vp]
+    lib.ubep_launch_count.restype, lib.ubep_launch_count.argtypes = u64, []
+    lib.ubep_debug_withhold_flag.restype, lib.ubep_debug_withhold_flag.argtypes = ctypes.c_int, [vp, i32]
+    lib.ubep_last_cuda_error.restype, lib.ubep_last_cuda_error.argtypes = ctypes.c_char_p, [vp]
+    lib.ubep_strerror.restype, lib.ubep_strerror.argtypes = ctypes.c_char_p, [ctypes.c_int]
+    _lib = lib
+    return lib
+
+
+class UbepError(RuntimeError):
+    def __init__(self, code: int, where: str, detail: str = ""):
+        self.code = code
+        msg = load().ubep_strerror(code).decode()
+        super().__init__(f"{where}: {msg} ({code}){' - ' + detail if detail else ''}")
+
+
+def _check(code: int, where: str, buf=None):
+    if code != UBEP_OK:
+        detail = load().ubep_last_cuda_error(buf).decode() if (buf and code == UBEP_ERR_CUDA) else ""
+        raise UbepError(code, where, detail)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    assert t.is_contiguous()
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+# ------------------------------------------------------------------ the C entry points
+
+def ubep_strerror(code: int) -> str:
+    return load().ubep_strerror(code).decode()
+
+
+def ubep_buffer_bytes(cfg: ubep_config_t) -> int:
+    return int(load().ubep_buffer_bytes(ctypes.byref(cfg)))
+
+
+def ubep_buffer_create(cfg: ubep_config_t, arena: torch.Tensor) -> ctypes.c_void_p:
+    out = ctypes.c_void_p()
+    _check(load().ubep_buffer_create(ctypes.byref(cfg), _ptr(arena), arena.numel() * arena.element_size(),
+                                     ctypes.byref(out)), "ubep_buffer_create")
+    return out
+
+
+def ubep_buffer_destroy(buf) -> None:
+    _check(load().ubep_buffer_destroy(buf), "ubep_buffer_destroy")
+
+
+def ubep_set_replicas(buf, phys: Optional[torch.Tensor], ncopies: Optional[torch.Tensor]) -> None:
+    if phys is None:
+        _check(load().ubep_set_replicas(buf, None, None, 0, 0), "ubep_set_replicas", buf)
+        return
+    assert phys.dtype == torch.int32 and ncopies.dtype == torch.int32 and phys.is_cuda
+    _check(load().ubep_set_replicas(buf, _ptr(phys), _ptr(ncopies), phys.shape[0], phys.shape[1]),
+           "ubep_set_replicas", buf)
+
+
+def ubep_set_dest_order(buf, order) -> None:
+    if order is None:
+        _check(load().ubep_set_dest_order(buf, None), "ubep_set_dest_order", buf)
+        return
+    arr = (ctypes.c_int32 * len(order))(*[int(v) for v in order])
+    _check(load().ubep_set_dest_order(buf, ctypes.cast(arr, ctypes.c_void_p)), "ubep_set_dest_order", buf)
+
+
+def ubep_get_dispatch_layout(buf, topk_idx: torch.Tensor, T: int, num_tokens_per_rank, num_tokens_per_expert,
+                             is_token_in_rank, stream=None) -> None:
+    _check(load().ubep_get_dispatch_layout(buf, _ptr(topk_idx), T, _ptr(num_tokens_per_rank),
+                                           _ptr(num_tokens_per_expert), _ptr(is_token_in_rank), _stream(stream)),
+           "ubep_get_dispatch_layout", buf)
+
+
+def ubep_dispatch(buf, x: torch.Tensor, topk_idx: torch.Tensor, topk_w: torch.Tensor, T: int, stream=None) -> None:
+    _check(load().ubep_dispatch(buf, _ptr(x), _ptr(topk_idx), _ptr(topk_w), T, _stream(stream)),
+           "ubep_dispatch", buf)
+
+
+def ubep_combine(buf, y: torch.Tensor, topk_w: torch.Tensor, T: int, out: torch.Tensor, stream=None) -> None:
+    _check(load().ubep_combine(buf, _ptr(y), _ptr(topk_w), T, _ptr(out), _stream(stream)), "ubep_combine", buf)
+
+
+def ubep_view(buf, which: int):
+    ptr = ctypes.c_void_p()
+    shape = (ctypes.c_int64 * 4)()
+    _check(load().ubep_view(buf, which, ctypes.byref(ptr), shape), "ubep_view", buf)
+    return ptr.value, list(shape)
+
+
+def ubep_status(buf) -> int:
+    st = ctypes.c_int32(0)
+    _check(load().ubep_status(buf, ctypes.byref(st)), "ubep_status", buf)
+    return st.value
+
+
+def ubep_epoch(buf) -> int:
+    return int(load().ubep_epoch(buf))
+
+
+def ubep_launch_count() -> int:
+    return int(load().ubep_launch_count())
+
+
+def ubep_debug_withhold_flag(buf, chunk: int) -> None:
+    _check(load().ubep_debug_withhold_flag(buf, chunk), "ubep_debug_withhold_flag", buf)
+
+
+# ------------------------------------------------------------------------ convenience
+
+class Buffer:
+    """An arena tensor plus the library handle laid out inside it."""
+
+    def __init__(self, *, num_ranks, num_experts, hidden, topk, max_tokens, rows_per_rank_cap,
+                 num_src_ranks=0, payload=0, dedup=0, device=0, pipeline=0, num_ctas=0, fill: Optional[int] = None):
+        self.cfg = ubep_config_t(num_ranks, num_experts, hidden, topk, max_tokens, rows_per_rank_cap,
+                                 num_src_ranks, payload, dedup, device, pipeline, num_ctas)
+        nbytes = ubep_buffer_bytes(self.cfg)
+        if nbytes == 0:
+            raise UbepError(UBEP_ERR_ARG, "ubep_buffer_bytes")
+        dev = torch.device("cuda", device)
+        self.arena = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+        if fill is not None:
+            self.arena.fill_(fill)
+        self.handle = ubep_buffer_create(self.cfg, self.arena)
+        self.views = {}
+        base = self.arena.data_ptr()
+        for which, (name, dt) in enumerate(zip(VIEW_NAMES, _VIEW_DTYPES)):
+            ptr, shape = ubep_view(self.handle, which)
+            if not ptr:
+                self.views[name] = None
+                continue
+            shape = [s for s in shape if s > 0]
+            rank = {"recv_x": 3, "recv_scale": 3, "recv_topk_idx": 3, "recv_topk_w": 3}.get(name)
+            if rank is None:
+                rank = 1 if name in ("expert_offset", "num_tokens_per_expert", "num_rows_per_rank",
+                                     "num_tokens_per_rank", "epoch") else 2
+            shape = shape[:rank]
+            n = 1
+            for s in shape:
+                n *= s
+            esz = torch.empty(0, dtype=dt).element_size()
+            self.views[name] = self.arena[ptr - base: ptr - base + n * esz].view(dt).view(shape)
+
+    def __getattr__(self, name):
+        views = self.__dict__.get("views", {})
+        if name in views:
+            return views[name]
+        raise AttributeError(name)
+
+    def set_replicas(self, phys, ncopies):
+        self._phys, self._ncopies = phys, ncopies     # keep the tensors alive
+        ubep_set_replicas(self.handle, phys, ncopies)
+
+    def set_dest_order(self, order):
+        ubep_set_dest_order(self.handle, order)
+
+    def get_dispatch_layout(self, topk_idx, stream=None):
+        T = topk_idx.shape[0]
+        R, E = self.cfg.num_ranks, self.cfg.num_experts
+        dev = self.arena.device
+        npr = torch.empty(R, dtype=torch.int32, device=dev)
+        npe = torch.empty(E, dtype=torch.int32, device=dev)
+        itr = torch.empty((T, R), dtype=torch.uint8, device=dev)
+        ubep_get_dispatch_layout(self.handle, topk_idx, T, npr, npe, itr, stream)
+        return npr, npe, itr
+
+    def dispatch(self, x, topk_idx, topk_w, stream=None):
+        ubep_dispatch(self.handle, x, topk_idx, topk_w, x.shape[0], stream)
+
+    def combine(self, y, topk_w, out=None, stream=None):
+        T = topk_w.shape[0]
+        if out is None:
+            out = torch.empty((T, self.cfg.hidden), dtype=torch.bfloat16, device=self.arena.device)
+        ubep_combine(self.handle, y, topk_w, T, out, stream)
+        return out
+
+    def status(self) -> int:
+        return ubep_status(self.handle)
+
+    def close(self):
+        if getattr(self, "handle", None):
+            ubep_buffer_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,212 @@
+// Shared device-side definitions of the dispatch / combine kernels (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace ubep {
+
+// Error codes mirrored from the public header (kept numerically identical).
+constexpr int kErrCapacity = -3;
+constexpr int kErrTimeout = -4;
+constexpr int kErrBadIndex = -5;
+
+constexpr int kThreads = 512;          // threads per persistent CTA
+constexpr int kWarps = kThreads / 32;
+constexpr int kMaxTopk = 32;
+constexpr int kMaxChunks = 320;        // scan keeps chunks/32 values per lane in registers
+constexpr int kMaxStages = 16;         // rows in the shared-memory ring
+constexpr int kModePhased = 1, kModeFused = 2, kModeLocal = 3;
+// Every wait in the kernels gives up after this many nanoseconds of wall time.
+constexpr unsigned long long kWaitLimitNs = 1500000000ull;
+
+// Everything a dispatch kernel needs, passed by value.
+struct Params {
+    // problem
+    int T, H, E, R, L, k, S, cap, payload, dedup;
+    int rowB;        // payload bytes per row: 2H (bf16) or H (FP8)
+    int G;           // H / 128 scale groups (FP8)
+    int B;           // histogram bins: E expert bins followed by R rank bins
+    int nchunks;     // token chunks == persistent CTAs of the fused kernel
+    int er_cap;      // entries per rank in expert_rows
+    unsigned* epoch_ctr;    // device word: dispatches completed on this buffer
+    unsigned* done_ticket;  // CTAs of the running dispatch kernel that have finished
+    int withhold;    // test hook: chunk whose hist flag is not published (-1 = none)
+    // inputs
+    const uint16_t* x;
+    const int32_t* topk_idx;
+    const float* topk_w;
+    const int32_t* phys;     // replica table [E_log, C] or null
+    const int32_t* ncopies;  // [E_log]
+    int E_log, C;
+    const int32_t* order_pos;  // [R] position of each rank in the destination-ordering table
+    // arena outputs
+    uint8_t* recv_x;
+    float* recv_scale;
+    int32_t* recv_src_idx;
+    float* recv_weight;
+    int32_t* recv_topk_idx;
+    float* recv_topk_w;
+    int32_t* expert_rows;
+    int32_t* cnt;
+    int32_t* src_offset;
+    int32_t* expert_offset;
+    int32_t* num_tokens_per_expert;
+    int32_t* num_rows_per_rank;
+    int32_t* num_tokens_per_rank;
+    int32_t* slot_row;   // [T, k] region-local row (chunk-local count until finalised)
+    int32_t* slot_aux;   // [T, k] dedup: chunk-local index into the expert's row list
+    int32_t* slot_pos;   // [T, k] global row (rank * cap + row) of each slot, -1 if none
+    // scratch
+    int32_t* chunk_hist;  // [nchunks, B]
+    int32_t* partial;     // [S, B] running chunk histogram at each source-rank boundary
+    int32_t* chunk_base;  // [nchunks, B] final base of every bin for every chunk
+    unsigned* hist_flag;  // [nchunks]
+    unsigned* scan_flag;  // [R]
+    unsigned* arrival;    // [2, R]
+    int32_t* status;
+};
+
+// ------------------------------------------------------------------ small helpers
+
+__device__ __forceinline__ int64_t chunk_begin(int c, int T, int n) { return (int64_t)c * T / n; }
+__device__ __forceinline__ int src_begin(int s, int T, int S) { return (int)((int64_t)s * T / S); }
+// Chunk that owns token b: the c with chunk_begin(c) <= b < chunk_begin(c + 1).
+__device__ __forceinline__ int chunk_of(int b, int T, int n) {
+    return (int)((((int64_t)b + 1) * n - 1) / T);
+}
+
+__device__ __forceinline__ void report(int32_t* status, int code) { atomicCAS(status, 0, code); }
+
+// Epoch of the running dispatch: one more than the number of completed dispatches.  Flags
+// must hold this value to count as set, so nothing is ever reset between calls, and a
+// captured CUDA graph can be replayed because the value lives on the device.  The word is
+// only advanced by the last CTA of a dispatch to finish, after every CTA has read it.
+__device__ __forceinline__ unsigned current_epoch(const Params& p) {
+    unsigned e = __ldcg(p.epoch_ctr) + 1u;
+    return e == 0u ? 1u : e;
+}
+__device__ __forceinline__ void finish_dispatch(const Params& p, unsigned epoch) {
+    __threadfence();
+    if (atomicAdd(p.done_ticket, 1u) == (unsigned)p.nchunks - 1u) {
+        *p.done_ticket = 0u;
+        __threadfence();
+        *p.epoch_ctr = epoch;
+    }
+}
+
+__device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release(unsigned* p, unsigned v) {
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void red_release_add(unsigned* p, unsigned v) {
+    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Wait until *flag == epoch.  Gives up after kWaitLimitNs (or as soon as *abort is set) and
+// returns false; the caller records the timeout and leaves.
+__device__ __forceinline__ bool wait_flag(const unsigned* flag, unsigned epoch, volatile int* abort) {
+    if (ld_acquire(flag) == epoch) return true;
+    const unsigned long long t_end = global_ns() + kWaitLimitNs;
+    unsigned ns = 32;
+    for (unsigned i = 1;; ++i) {
+        if (ld_acquire(flag) == epoch) return true;
+        if (abort && *abort) return false;
+        if ((i & 63u) == 0 && global_ns() > t_end) return false;
+        __nanosleep(ns);
+        if (ns < 256) ns <<= 1;
+    }
+}
+
+// ------------------------------------------------------------ TMA / mbarrier (PTX)
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_fence_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// Non-blocking test of an mbarrier phase.
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, unsigned parity) {
+    unsigned ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait on an mbarrier phase; false after kWaitLimitNs or on abort.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity, volatile int* abort) {
+    for (unsigned i = 0; i < 128; ++i)
+        if (mbar_test_wait(bar, parity)) return true;
+    const unsigned long long t_end = global_ns() + kWaitLimitNs;
+    for (unsigned i = 1;; ++i) {
+        if (mbar_test_wait(bar, parity)) return true;
+        if (abort && *abort) return false;
+        if ((i & 63u) == 0 && global_ns() > t_end) return false;
+        __nanosleep(40);
+    }
+}
+// global -> shared bulk copy, completion counted in bytes on `bar`.
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, unsigned bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_u32(smem_dst)),
+                 "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+// shared -> global bulk copy, tracked by the thread's bulk async-group.
+__device__ __forceinline__ void bulk_store(void* gdst, const void* smem_src, unsigned bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst),
+                 "r"(smem_u32(smem_src)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+template <int N>
+__device__ __forceinline__ void bulk_wait_all() {
+    asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
+// Barrier among a subset of the CTA's warps (id 1..15), `nthreads` a multiple of 32.
+__device__ __forceinline__ void group_sync(int id, int nthreads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+// The same barrier with an OR-reduction: every thread of the group gets the same answer.
+__device__ __forceinline__ bool group_or(int id, int nthreads, bool pred) {
+    unsigned r;
+    asm volatile(
+        "{\n .reg .pred p, q;\n setp.ne.u32 q, %3, 0;\n bar.red.or.pred p, %1, %2, q;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(r)
+        : "r"(id), "r"(nthreads), "r"((unsigned)pred)
+        : "memory");
+    return r != 0;
+}
+
+}  // namespace ubep

@@ -1,0 +1,405 @@
+// C ABI of the library (declared in include/ubep.h): argument checks, arena layout and
+// kernel launches.  No device memory is allocated here and no stream is created.
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/ubep.h"
+#include "ubep_kernels.h"
+
+using ubep::Params;
+
+namespace {
+
+std::atomic<uint64_t> g_launches{0};
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
+
+struct ArenaLayout {
+    size_t off[UBEP_VIEW_COUNT_];
+    size_t slot_aux, slot_pos, chunk_hist, partial, chunk_base;
+    size_t flags_begin, hist_flag, scan_flag, status, ticket, epoch_ctr, done_ticket, order_pos, flags_end;
+    size_t total;
+    int er_cap, nchunks, S, rowB, G, B;
+};
+
+bool valid_config(const ubep_config_t& c) {
+    if (c.num_ranks < 1 || c.num_experts < 1 || c.num_experts % c.num_ranks != 0) return false;
+    if (c.topk < 1 || c.topk > ubep::kMaxTopk) return false;
+    if (c.hidden < 8 || c.hidden % 8 != 0) return false;
+    if (c.payload != UBEP_PAYLOAD_BF16 && c.payload != UBEP_PAYLOAD_FP8_E4M3) return false;
+    if (c.payload == UBEP_PAYLOAD_FP8_E4M3 && c.hidden % 128 != 0) return false;
+    if (c.max_tokens < 1 || c.rows_per_rank_cap < 1 || c.num_src_ranks < 0) return false;
+    if (c.dedup != 0 && c.dedup != 1) return false;
+    if (c.pipeline < UBEP_PIPELINE_AUTO || c.pipeline > UBEP_PIPELINE_LOCAL) return false;
+    if (c.num_ctas < 0 || c.num_ctas > ubep::kMaxChunks) return false;
+    if ((int64_t)c.num_ranks * c.rows_per_rank_cap > INT32_MAX) return false;
+    if ((int64_t)c.max_tokens * c.topk > INT32_MAX) return false;
+    return true;
+}
+
+// nchunks == 0 means "not known yet": size for the largest value allowed.
+ArenaLayout make_layout(const ubep_config_t& c, int nchunks) {
+    ArenaLayout a{};
+    const size_t R = c.num_ranks, E = c.num_experts, H = c.hidden, k = c.topk, cap = c.rows_per_rank_cap;
+    const size_t L = E / R;
+    a.S = c.num_src_ranks > 0 ? c.num_src_ranks : c.num_ranks;
+    a.rowB = c.payload ? (int)H : (int)(2 * H);
+    a.G = (int)(H / 128);
+    a.B = (int)(E + R);
+    a.nchunks = nchunks > 0 ? nchunks : ubep::kMaxChunks;
+    a.er_cap = c.dedup ? (int)(cap * (k < L ? k : L)) : 0;
+    const size_t S = a.S, n = a.nchunks, B = a.B, Tk = (size_t)c.max_tokens * k;
+    size_t at = 0;
+    auto take = [&](size_t bytes) { size_t o = at; at = align_up(at + bytes); return o; };
+    a.off[UBEP_VIEW_RECV_X] = take(R * cap * a.rowB);
+    a.off[UBEP_VIEW_RECV_SCALE] = take(c.payload ? R * cap * a.G * 4 : 0);
+    a.off[UBEP_VIEW_RECV_SRC_IDX] = take(R * cap * 4);
+    a.off[UBEP_VIEW_RECV_WEIGHT] = take(c.dedup ? 0 : R * cap * 4);
+    a.off[UBEP_VIEW_RECV_TOPK_IDX] = take(c.dedup ? R * cap * k * 4 : 0);
+    a.off[UBEP_VIEW_RECV_TOPK_W] = take(c.dedup ? R * cap * k * 4 : 0);
+    a.off[UBEP_VIEW_EXPERT_ROWS] = take(R * (size_t)a.er_cap * 4);
+    a.off[UBEP_VIEW_CNT] = take(S * E * 4);
+    a.off[UBEP_VIEW_SRC_OFFSET] = take(S * E * 4);
+    a.off[UBEP_VIEW_EXPERT_OFFSET] = take(E * 4);
+    a.off[UBEP_VIEW_NUM_TOKENS_PER_EXPERT] = take(E * 4);
+    a.off[UBEP_VIEW_NUM_ROWS_PER_RANK] = take(R * 4);
+    a.off[UBEP_VIEW_NUM_TOKENS_PER_RANK] = take(R * 4);
+    a.off[UBEP_VIEW_SLOT_ROW] = take(Tk * 4);
+    a.slot_aux = take(Tk * 4);
+    a.slot_pos = take(Tk * 4);
+    a.chunk_hist = take(n * B * 4);
+    a.partial = take(S * B * 4);
+    a.chunk_base = take(n * B * 4);
+    a.flags_begin = at;
+    a.hist_flag = take(n * 4);
+    a.scan_flag = take(R * 4);
+    a.off[UBEP_VIEW_ARRIVAL] = take(2 * R * 4);
+    a.status = take(4);
+    a.ticket = take(4);
+    a.off[UBEP_VIEW_EPOCH] = a.epoch_ctr = take(4);
+    a.done_ticket = take(4);
+    a.flags_end = at;
+    a.order_pos = take(R * 4);
+    a.total = at;
+    return a;
+}
+
+}  // namespace
+
+struct ubep_buffer {
+    ubep_config_t cfg;
+    ArenaLayout lay;
+    uint8_t* arena;
+    int num_sms;
+    int max_smem;
+    uint32_t epoch;
+    int32_t withhold;
+    cudaStream_t last_stream;
+    const int32_t* phys;
+    const int32_t* ncopies;
+    int32_t E_log, C;
+    std::string cuda_error;
+};
+
+namespace {
+
+int cuda_fail(ubep_buffer* b, cudaError_t e) {
+    if (b) b->cuda_error = cudaGetErrorString(e);
+    return UBEP_ERR_CUDA;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+template <typename T>
+T* at(ubep_buffer* b, size_t off) { return reinterpret_cast<T*>(b->arena + off); }
+
+Params make_params(ubep_buffer* b, int T) {
+    const ubep_config_t& c = b->cfg;
+    const ArenaLayout& a = b->lay;
+    Params p{};
+    p.T = T; p.H = c.hidden; p.E = c.num_experts; p.R = c.num_ranks; p.L = p.E / p.R; p.k = c.topk;
+    p.S = a.S; p.cap = c.rows_per_rank_cap; p.payload = c.payload; p.dedup = c.dedup;
+    p.rowB = a.rowB; p.G = a.G; p.B = a.B; p.nchunks = a.nchunks; p.er_cap = a.er_cap;
+    p.epoch_ctr = at<unsigned>(b, a.epoch_ctr);
+    p.done_ticket = at<unsigned>(b, a.done_ticket);
+    p.withhold = -1;
+    p.phys = b->phys; p.ncopies = b->ncopies; p.E_log = b->E_log; p.C = b->C;
+    p.order_pos = at<int32_t>(b, a.order_pos);
+    p.recv_x = at<uint8_t>(b, a.off[UBEP_VIEW_RECV_X]);
+    p.recv_scale = at<float>(b, a.off[UBEP_VIEW_RECV_SCALE]);
+    p.recv_src_idx = at<int32_t>(b, a.off[UBEP_VIEW_RECV_SRC_IDX]);
+    p.recv_weight = at<float>(b, a.off[UBEP_VIEW_RECV_WEIGHT]);
+    p.recv_topk_idx = at<int32_t>(b, a.off[UBEP_VIEW_RECV_TOPK_IDX]);
+    p.recv_topk_w = at<float>(b, a.off[UBEP_VIEW_RECV_TOPK_W]);
+    p.expert_rows = at<int32_t>(b, a.off[UBEP_VIEW_EXPERT_ROWS]);
+    p.cnt = at<int32_t>(b, a.off[UBEP_VIEW_CNT]);
+    p.src_offset = at<int32_t>(b, a.off[UBEP_VIEW_SRC_OFFSET]);
+    p.expert_offset = at<int32_t>(b, a.off[UBEP_VIEW_EXPERT_OFFSET]);
+    p.num_tokens_per_expert = at<int32_t>(b, a.off[UBEP_VIEW_NUM_TOKENS_PER_EXPERT]);
+    p.num_rows_per_rank = at<int32_t>(b, a.off[UBEP_VIEW_NUM_ROWS_PER_RANK]);
+    p.num_tokens_per_rank = at<int32_t>(b, a.off[UBEP_VIEW_NUM_TOKENS_PER_RANK]);
+    p.slot_row = at<int32_t>(b, a.off[UBEP_VIEW_SLOT_ROW]);
+    p.slot_aux = at<int32_t>(b, a.slot_aux);
+    p.slot_pos = at<int32_t>(b, a.slot_pos);
+    p.chunk_hist = at<int32_t>(b, a.chunk_hist);
+    p.partial = at<int32_t>(b, a.partial);
+    p.chunk_base = at<int32_t>(b, a.chunk_base);
+    p.hist_flag = at<unsigned>(b, a.hist_flag);
+    p.scan_flag = at<unsigned>(b, a.scan_flag);
+    p.arrival = at<unsigned>(b, a.off[UBEP_VIEW_ARRIVAL]);
+    p.status = at<int32_t>(b, a.status);
+    return p;
+}
+
+// Makes the buffer's device current for the scope of one call.
+struct DeviceGuard {
+    int prev = -1;
+    bool switched = false;
+    cudaError_t err = cudaSuccess;
+    explicit DeviceGuard(int dev) {
+        err = cudaGetDevice(&prev);
+        if (err == cudaSuccess && prev != dev) {
+            err = cudaSetDevice(dev);
+            switched = err == cudaSuccess;
+        }
+    }
+    ~DeviceGuard() {
+        if (switched) cudaSetDevice(prev);
+    }
+};
+
+}  // namespace
+
+extern "C" {
+
+size_t ubep_buffer_bytes(const ubep_config_t* cfg) {
+    if (!cfg || !valid_config(*cfg)) return 0;
+    return make_layout(*cfg, cfg->num_ctas).total;
+}
+
+int ubep_buffer_create(const ubep_config_t* cfg, void* dev_arena, size_t bytes, ubep_buffer_t** out) {
+    if (!cfg || !out || !dev_arena || !valid_config(*cfg)) return UBEP_ERR_ARG;
+    *out = nullptr;
+    if ((reinterpret_cast<uintptr_t>(dev_arena) & (kAlign - 1)) != 0) return UBEP_ERR_ARENA;
+    if (bytes < make_layout(*cfg, cfg->num_ctas).total) return UBEP_ERR_ARENA;
+    DeviceGuard guard(cfg->device);
+    if (guard.err != cudaSuccess) return UBEP_ERR_CUDA;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, cfg->device) != cudaSuccess) return UBEP_ERR_CUDA;
+    ubep_buffer* b = new (std::nothrow) ubep_buffer();
+    if (!b) return UBEP_ERR_ARG;
+    b->cfg = *cfg;
+    b->num_sms = prop.multiProcessorCount;
+    b->max_smem = (int)prop.sharedMemPerBlockOptin;
+    int n = cfg->num_ctas > 0 ? cfg->num_ctas : b->num_sms;
+    if (n > b->num_sms) n = b->num_sms;  // all CTAs of the persistent kernel must be resident
+    if (n > ubep::kMaxChunks) n = ubep::kMaxChunks;
+    b->lay = make_layout(*cfg, n);
+    b->arena = static_cast<uint8_t*>(dev_arena);
+    b->epoch = 0;
+    b->withhold = -1;
+    b->last_stream = nullptr;
+    b->phys = nullptr;
+    b->ncopies = nullptr;
+    b->E_log = 0;
+    b->C = 0;
+    cudaError_t e = cudaMemset(b->arena + b->lay.flags_begin, 0, b->lay.flags_end - b->lay.flags_begin);
+    if (e == cudaSuccess) {
+        std::vector<int32_t> ident(cfg->num_ranks);
+        for (int r = 0; r < cfg->num_ranks; ++r) ident[r] = r;
+        e = cudaMemcpy(b->arena + b->lay.order_pos, ident.data(), sizeof(int32_t) * ident.size(),
+                       cudaMemcpyHostToDevice);
+    }
+    if (e != cudaSuccess) {
+        delete b;
+        return UBEP_ERR_CUDA;
+    }
+    *out = b;
+    return UBEP_OK;
+}
+
+int ubep_buffer_destroy(ubep_buffer_t* buf) {
+    if (!buf) return UBEP_ERR_ARG;
+    delete buf;
+    return UBEP_OK;
+}
+
+int ubep_set_replicas(ubep_buffer_t* buf, const int32_t* phys, const int32_t* ncopies, int32_t E_log, int32_t C) {
+    if (!buf) return UBEP_ERR_ARG;
+    if (!phys && !ncopies) {
+        buf->phys = nullptr; buf->ncopies = nullptr; buf->E_log = 0; buf->C = 0;
+        return UBEP_OK;
+    }
+    if (!phys || !ncopies || E_log < 1 || C < 1) return UBEP_ERR_ARG;
+    buf->phys = phys; buf->ncopies = ncopies; buf->E_log = E_log; buf->C = C;
+    return UBEP_OK;
+}
+
+int ubep_set_dest_order(ubep_buffer_t* buf, const int32_t* order) {
+    if (!buf) return UBEP_ERR_ARG;
+    const int R = buf->cfg.num_ranks;
+    std::vector<int32_t> posv(R, -1);
+    for (int i = 0; i < R; ++i) {
+        const int r = order ? order[i] : i;
+        if (r < 0 || r >= R || posv[r] != -1) return UBEP_ERR_ARG;  // not a permutation
+        posv[r] = i;
+    }
+    DeviceGuard guard(buf->cfg.device);
+    if (guard.err != cudaSuccess) return cuda_fail(buf, guard.err);
+    // ordered after earlier work on the stream of the last call, then waited for
+    cudaError_t e = cudaMemcpyAsync(buf->arena + buf->lay.order_pos, posv.data(), sizeof(int32_t) * R,
+                                    cudaMemcpyHostToDevice, buf->last_stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(buf->last_stream);
+    return e == cudaSuccess ? UBEP_OK : cuda_fail(buf, e);
+}
+
+int ubep_get_dispatch_layout(ubep_buffer_t* buf, const int32_t* topk_idx, int32_t T, int32_t* num_tokens_per_rank,
+                             int32_t* num_tokens_per_expert, uint8_t* is_token_in_rank, void* cuda_stream) {
+    if (!buf || T < 0 || T > buf->cfg.max_tokens || (T > 0 && !topk_idx) || !aligned16(topk_idx)) return UBEP_ERR_ARG;
+    DeviceGuard guard(buf->cfg.device);
+    if (guard.err != cudaSuccess) return cuda_fail(buf, guard.err);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    buf->last_stream = st;
+    Params p = make_params(buf, T);
+    p.topk_idx = topk_idx;
+    cudaError_t e = ubep::launch_layout(p, num_tokens_per_rank, num_tokens_per_expert, is_token_in_rank,
+                                        p.chunk_hist, at<unsigned>(buf, buf->lay.ticket), st);
+    if (e != cudaSuccess) return cuda_fail(buf, e);
+    g_launches += 1;
+    return UBEP_OK;
+}
+
+int ubep_dispatch(ubep_buffer_t* buf, const void* x, const int32_t* topk_idx, const float* topk_w, int32_t T,
+                  void* cuda_stream) {
+    if (!buf || T < 0 || T > buf->cfg.max_tokens) return UBEP_ERR_ARG;
+    if (T > 0 && (!x || !topk_idx || !topk_w)) return UBEP_ERR_ARG;
+    if (!aligned16(x) || !aligned16(topk_idx) || !aligned16(topk_w)) return UBEP_ERR_ARG;
+    DeviceGuard guard(buf->cfg.device);
+    if (guard.err != cudaSuccess) return cuda_fail(buf, guard.err);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    buf->last_stream = st;
+    if (T == 0) {
+        // nothing to route: every count and offset is zero (one contiguous block of the arena)
+        const size_t lo = buf->lay.off[UBEP_VIEW_CNT], hi = buf->lay.off[UBEP_VIEW_SLOT_ROW];
+        cudaError_t e0 = cudaMemsetAsync(buf->arena + lo, 0, hi - lo, st);
+        return e0 == cudaSuccess ? UBEP_OK : cuda_fail(buf, e0);
+    }
+    buf->epoch += 1;
+    Params p = make_params(buf, T);
+    p.x = static_cast<const uint16_t*>(x);
+    p.topk_idx = topk_idx;
+    p.topk_w = topk_w;
+    p.withhold = buf->withhold;
+    buf->withhold = -1;
+    int mode = buf->cfg.pipeline == UBEP_PIPELINE_AUTO ? UBEP_PIPELINE_FUSED : buf->cfg.pipeline;
+    if (mode == UBEP_PIPELINE_LOCAL) mode = UBEP_PIPELINE_FUSED;
+    int stages = 0, stage_bytes = 0, launches = 0;
+    size_t smem = 0;
+    if (ubep::plan_dispatch(p, buf->max_smem, &stages, &stage_bytes, &smem) != 0) return UBEP_ERR_ARG;
+    cudaError_t e = ubep::launch_dispatch(p, mode, stages, stage_bytes, smem, st, &launches);
+    if (e != cudaSuccess) return cuda_fail(buf, e);
+    g_launches += launches;
+    return UBEP_OK;
+}
+
+int ubep_combine(ubep_buffer_t* buf, const void* y, const float* topk_w, int32_t T, void* out, void* cuda_stream) {
+    if (!buf || T < 0 || T > buf->cfg.max_tokens) return UBEP_ERR_ARG;
+    if (T > 0 && (!y || !topk_w || !out)) return UBEP_ERR_ARG;
+    if (!aligned16(y) || !aligned16(topk_w) || !aligned16(out)) return UBEP_ERR_ARG;
+    if (T == 0) return UBEP_OK;
+    DeviceGuard guard(buf->cfg.device);
+    if (guard.err != cudaSuccess) return cuda_fail(buf, guard.err);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    buf->last_stream = st;
+    cudaError_t e = ubep::launch_combine(static_cast<const uint16_t*>(y), at<int32_t>(buf, buf->lay.slot_pos), topk_w,
+                                         T, buf->cfg.hidden, buf->cfg.topk, static_cast<uint16_t*>(out),
+                                         buf->num_sms, st);
+    if (e != cudaSuccess) return cuda_fail(buf, e);
+    g_launches += 1;
+    return UBEP_OK;
+}
+
+int ubep_view(ubep_buffer_t* buf, int which, void** dev_ptr, int64_t shape[4]) {
+    if (!buf || !dev_ptr || !shape || which < 0 || which >= UBEP_VIEW_COUNT_) return UBEP_ERR_ARG;
+    const ubep_config_t& c = buf->cfg;
+    const ArenaLayout& a = buf->lay;
+    const int64_t R = c.num_ranks, E = c.num_experts, cap = c.rows_per_rank_cap, k = c.topk, S = a.S;
+    int64_t s[4] = {1, 1, 1, 1};
+    bool present = true;
+    switch (which) {
+        case UBEP_VIEW_RECV_X: s[0] = R; s[1] = cap; s[2] = a.rowB; break;
+        case UBEP_VIEW_RECV_SCALE: s[0] = R; s[1] = cap; s[2] = a.G; present = c.payload != 0; break;
+        case UBEP_VIEW_RECV_SRC_IDX: s[0] = R; s[1] = cap; break;
+        case UBEP_VIEW_RECV_WEIGHT: s[0] = R; s[1] = cap; present = !c.dedup; break;
+        case UBEP_VIEW_RECV_TOPK_IDX:
+        case UBEP_VIEW_RECV_TOPK_W: s[0] = R; s[1] = cap; s[2] = k; present = c.dedup != 0; break;
+        case UBEP_VIEW_EXPERT_ROWS: s[0] = R; s[1] = a.er_cap; present = c.dedup != 0; break;
+        case UBEP_VIEW_CNT:
+        case UBEP_VIEW_SRC_OFFSET: s[0] = S; s[1] = E; break;
+        case UBEP_VIEW_EXPERT_OFFSET:
+        case UBEP_VIEW_NUM_TOKENS_PER_EXPERT: s[0] = E; break;
+        case UBEP_VIEW_NUM_ROWS_PER_RANK:
+        case UBEP_VIEW_NUM_TOKENS_PER_RANK: s[0] = R; break;
+        case UBEP_VIEW_SLOT_ROW: s[0] = c.max_tokens; s[1] = k; break;
+        case UBEP_VIEW_ARRIVAL: s[0] = 2; s[1] = R; break;
+        case UBEP_VIEW_EPOCH: s[0] = 1; break;
+        default: return UBEP_ERR_ARG;
+    }
+    if (!present) {
+        *dev_ptr = nullptr;
+        for (int i = 0; i < 4; ++i) shape[i] = 0;
+        return UBEP_OK;
+    }
+    *dev_ptr = buf->arena + a.off[which];
+    for (int i = 0; i < 4; ++i) shape[i] = s[i];
+    return UBEP_OK;
+}
+
+int ubep_status(ubep_buffer_t* buf, int32_t* last_async_status) {
+    if (!buf || !last_async_status) return UBEP_ERR_ARG;
+    DeviceGuard guard(buf->cfg.device);
+    if (guard.err != cudaSuccess) return cuda_fail(buf, guard.err);
+    int32_t v = 0;
+    cudaError_t e = cudaMemcpyAsync(&v, buf->arena + buf->lay.status, sizeof(v), cudaMemcpyDeviceToHost,
+                                    buf->last_stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(buf->last_stream);
+    if (e == cudaSuccess && v != 0) {
+        e = cudaMemsetAsync(buf->arena + buf->lay.status, 0, sizeof(v), buf->last_stream);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(buf->last_stream);
+    }
+    if (e != cudaSuccess) return cuda_fail(buf, e);
+    *last_async_status = v;
+    return UBEP_OK;
+}
+
+uint32_t ubep_epoch(const ubep_buffer_t* buf) { return buf ? buf->epoch : 0; }
+
+uint64_t ubep_launch_count(void) { return g_launches.load(); }
+
+int ubep_debug_withhold_flag(ubep_buffer_t* buf, int32_t chunk) {
+    if (!buf || chunk < -1 || chunk >= buf->lay.nchunks) return UBEP_ERR_ARG;
+    buf->withhold = chunk;
+    return UBEP_OK;
+}
+
+const char* ubep_last_cuda_error(const ubep_buffer_t* buf) { return buf ? buf->cuda_error.c_str() : ""; }
+
+const char* ubep_strerror(int code) {
+    switch (code) {
+        case UBEP_OK: return "ok";
+        case UBEP_ERR_ARG: return "invalid argument";
+        case UBEP_ERR_CUDA: return "CUDA runtime error";
+        case UBEP_ERR_CAPACITY: return "a receive region needs more rows than rows_per_rank_cap";
+        case UBEP_ERR_TIMEOUT: return "a bounded wait on a readiness flag ran out";
+        case UBEP_ERR_BAD_INDEX: return "expert id out of range";
+        case UBEP_ERR_ARENA: return "arena too small or misaligned";
+        default: return "unknown error";
+    }
+}
+
+}  // extern "C"
