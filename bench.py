@@ -205,7 +205,7 @@ def run_ours(args, cfg, rank: int, world: int, local_rank: int):
 
     # one CUDA graph holds one pass over all sets; the epoch lives on the device, so replays are valid
     graph = None
-    if not args.no_graph:
+    if not args.no_graph and not args.profile:
         with torch.cuda.stream(stream):
             for s in sets:
                 step(s)
@@ -231,7 +231,7 @@ def run_ours(args, cfg, rank: int, world: int, local_rank: int):
             dist.barrier()
         torch.cuda.synchronize()
 
-    run_steps(max(args.warmup, 3))
+    run_steps(args.warmup if args.profile else max(args.warmup, 3))
     barrier()
     sampler = ClockSampler(physical_gpu_index(local_rank))
     sampler.start()
@@ -256,6 +256,12 @@ def run_ours(args, cfg, rank: int, world: int, local_rank: int):
         total_ms = float(t.item())
     ms_per_step = total_ms / args.steps
     value = world * (disp_b + comb_b) / (ms_per_step * 1e-3) / 1e9
+
+    if args.profile:
+        if rank == 0:
+            print(json.dumps({"profile_run": True, "workload": cfg.name, "steps": args.steps,
+                              "ms_per_step": ms_per_step, "pipeline": args.pipeline}), flush=True)
+        return
 
     # per-kernel durations, CUDA events on the launching stream, same rotating sets
     n_k = min(args.steps, 400)
@@ -382,6 +388,8 @@ def main():
     ap.add_argument("--workload", default="decode")
     ap.add_argument("--pipeline", type=int, default=0)
     ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--profile", action="store_true",
+                    help="plain launches of the timed steps only (for ncu): no graph, no e2e, no CPU leg")
     args = ap.parse_args()
 
     from paper_2607_06202_b200 import workload as W

@@ -163,7 +163,7 @@ def test_bad_arguments_are_rejected_synchronously():
     with pytest.raises(B.UbepError):
         B.ubep_dispatch(buf.handle, x, idx, w, 65)                 # T > max_tokens
     with pytest.raises(B.UbepError):
-        B.ubep_dispatch(buf.handle, x.view(torch.uint8)[2:].view(torch.bfloat16), idx, w, 32)   # misaligned
+        B.ubep_dispatch(buf.handle, x.view(torch.uint8).flatten()[2:-14].view(torch.bfloat16), idx, w, 32)  # misaligned
     with pytest.raises(B.UbepError):
         B.ubep_dispatch(buf.handle, None, idx, w, 64)
     assert B.ubep_launch_count() == n0
