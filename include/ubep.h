@@ -43,7 +43,7 @@ enum { UBEP_PAYLOAD_BF16 = 0, UBEP_PAYLOAD_FP8_E4M3 = 1 };
 
 /* How ubep_dispatch schedules its steps. */
 enum {
-    UBEP_PIPELINE_AUTO = 0,   /* FUSED                                                        */
+    UBEP_PIPELINE_AUTO = 0,   /* LOCAL while T*k <= 8192, else FUSED                           */
     UBEP_PIPELINE_PHASED = 1, /* count -> prefix sums -> scatter as three launches; the        */
                               /* kernel boundaries play the role of the global barriers of    */
                               /* the bulk-synchronous dispatch (Sec. 2.3, phases 2-5)         */
@@ -88,13 +88,17 @@ enum {
     UBEP_VIEW_NUM_TOKENS_PER_RANK = 12,   /* i32 [R]    distinct tokens routed to each rank    */
     UBEP_VIEW_SLOT_ROW = 13,     /* i32 [max_tokens, k] region-local row of each slot, or -1;  */
                                  /*                     the handle ubep_combine uses           */
-    UBEP_VIEW_ARRIVAL = 14,      /* u32 [2, R]          rows landed per region; the half the   */
-                                 /*                     n-th dispatch uses is (n & 1)          */
+    UBEP_VIEW_ARRIVAL = 14,      /* u32 [2, R]          eighths of rows landed per region (a   */
+                                 /*                     region is complete at 8 * its row      */
+                                 /*                     count); the n-th dispatch uses half    */
+                                 /*                     (n & 1)                                */
     UBEP_VIEW_EPOCH = 15,        /* u32 [1]             dispatches completed on this buffer;   */
                                  /*                     readiness flags hold this count + 1    */
                                  /*                     while a dispatch runs, so replaying a  */
                                  /*                     captured CUDA graph needs no reset     */
-    UBEP_VIEW_COUNT_ = 16
+    UBEP_VIEW_TRACE = 16,        /* u64 [chunks, 16]    per-CTA phase time stamps in ns of the */
+                                 /*                     last traced dispatch (ubep_debug_trace)*/
+    UBEP_VIEW_COUNT_ = 17
 };
 
 /*
@@ -190,6 +194,16 @@ uint64_t ubep_launch_count(void);
  * after about a second, the kernel returns and ubep_status reports UBEP_ERR_TIMEOUT.
  */
 int ubep_debug_withhold_flag(ubep_buffer_t *buf, int32_t chunk);
+
+/*
+ * Tracing (the paper reports per-task latency breakdowns, Sec. 5.3): when enabled, every
+ * CTA of the following dispatches stamps the device nanosecond timer at its phase
+ * boundaries into UBEP_VIEW_TRACE: 0 start, 1 counted, 2 all counts seen, 3 prefix sums
+ * published, 4 all offsets seen, 5 rows assigned, 6 movers released, 7 first row in shared
+ * memory, 8 last copy issued, 9 copies complete, 10 end.  Slots a CTA does not pass keep
+ * their old value.
+ */
+int ubep_debug_trace(ubep_buffer_t *buf, int32_t enable);
 
 /* Text of the last CUDA runtime error seen by this buffer's calls ("" if none). */
 const char *ubep_last_cuda_error(const ubep_buffer_t *buf);

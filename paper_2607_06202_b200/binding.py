@@ -25,15 +25,15 @@ UBEP_PIPELINE_AUTO, UBEP_PIPELINE_PHASED, UBEP_PIPELINE_FUSED, UBEP_PIPELINE_LOC
 
 VIEW_NAMES = ["recv_x", "recv_scale", "recv_src_idx", "recv_weight", "recv_topk_idx", "recv_topk_w",
               "expert_rows", "cnt", "src_offset", "expert_offset", "num_tokens_per_expert",
-              "num_rows_per_rank", "num_tokens_per_rank", "slot_row", "arrival", "epoch"]
+              "num_rows_per_rank", "num_tokens_per_rank", "slot_row", "arrival", "epoch", "trace"]
 _VIEW_DTYPES = [torch.uint8, torch.float32, torch.int32, torch.float32, torch.int32, torch.float32,
                 torch.int32, torch.int32, torch.int32, torch.int32, torch.int32, torch.int32, torch.int32,
-                torch.int32, torch.int32, torch.int32]
+                torch.int32, torch.int32, torch.int32, torch.int64]
 
 # every symbol include/ubep.h declares
 EXPORTS = ["ubep_buffer_bytes", "ubep_buffer_create", "ubep_buffer_destroy", "ubep_set_replicas",
            "ubep_set_dest_order", "ubep_get_dispatch_layout", "ubep_dispatch", "ubep_combine", "ubep_view",
-           "ubep_status", "ubep_epoch", "ubep_launch_count", "ubep_debug_withhold_flag",
+           "ubep_status", "ubep_epoch", "ubep_launch_count", "ubep_debug_withhold_flag", "ubep_debug_trace",
            "ubep_last_cuda_error", "ubep_strerror"]
 
 
@@ -72,6 +72,7 @@ def load() -> ctypes.CDLL:
     lib.ubep_epoch.restype, lib.ubep_epoch.argtypes = u32, [vp]
     lib.ubep_launch_count.restype, lib.ubep_launch_count.argtypes = u64, []
     lib.ubep_debug_withhold_flag.restype, lib.ubep_debug_withhold_flag.argtypes = ctypes.c_int, [vp, i32]
+    lib.ubep_debug_trace.restype, lib.ubep_debug_trace.argtypes = ctypes.c_int, [vp, i32]
     lib.ubep_last_cuda_error.restype, lib.ubep_last_cuda_error.argtypes = ctypes.c_char_p, [vp]
     lib.ubep_strerror.restype, lib.ubep_strerror.argtypes = ctypes.c_char_p, [ctypes.c_int]
     _lib = lib
@@ -177,6 +178,10 @@ def ubep_epoch(buf) -> int:
 
 def ubep_launch_count() -> int:
     return int(load().ubep_launch_count())
+
+
+def ubep_debug_trace(buf, enable: bool) -> None:
+    _check(load().ubep_debug_trace(buf, int(bool(enable))), "ubep_debug_trace", buf)
 
 
 def ubep_debug_withhold_flag(buf, chunk: int) -> None:

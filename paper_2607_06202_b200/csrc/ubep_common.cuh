@@ -17,6 +17,8 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kMaxTopk = 32;
 constexpr int kMaxChunks = 320;        // scan keeps chunks/32 values per lane in registers
 constexpr int kMaxStages = 16;         // rows in the shared-memory ring
+constexpr int kOutStages = 4;          // quantised rows waiting for their bulk stores (FP8)
+constexpr int kTraceSlots = 16;        // per-CTA phase time stamps (optional tracing)
 constexpr int kModePhased = 1, kModeFused = 2, kModeLocal = 3;
 // Every wait in the kernels gives up after this many nanoseconds of wall time.
 constexpr unsigned long long kWaitLimitNs = 1500000000ull;
@@ -28,7 +30,9 @@ struct Params {
     int rowB;        // payload bytes per row: 2H (bf16) or H (FP8)
     int G;           // H / 128 scale groups (FP8)
     int B;           // histogram bins: E expert bins followed by R rank bins
-    int nchunks;     // token chunks == persistent CTAs of the fused kernel
+    int nchunks;     // token chunks (contiguous, equal to +-1 token)
+    int parts;       // column parts per row: CTA c moves part c % parts of chunk c / parts
+    int grid;        // CTAs of the dispatch kernel = nchunks * parts
     int er_cap;      // entries per rank in expert_rows
     unsigned* epoch_ctr;    // device word: dispatches completed on this buffer
     unsigned* done_ticket;  // CTAs of the running dispatch kernel that have finished
@@ -66,6 +70,7 @@ struct Params {
     unsigned* scan_flag;  // [R]
     unsigned* arrival;    // [2, R]
     int32_t* status;
+    unsigned long long* trace;  // optional [nchunks, kTraceSlots] globaltimer stamps, or null
 };
 
 // ------------------------------------------------------------------ small helpers
@@ -89,7 +94,7 @@ __device__ __forceinline__ unsigned current_epoch(const Params& p) {
 }
 __device__ __forceinline__ void finish_dispatch(const Params& p, unsigned epoch) {
     __threadfence();
-    if (atomicAdd(p.done_ticket, 1u) == (unsigned)p.nchunks - 1u) {
+    if (atomicAdd(p.done_ticket, 1u) == (unsigned)p.grid - 1u) {
         *p.done_ticket = 0u;
         __threadfence();
         *p.epoch_ctr = epoch;
@@ -112,6 +117,13 @@ __device__ __forceinline__ unsigned long long global_ns() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
     return t;
+}
+
+// Optional tracing: per-CTA %globaltimer stamp of a phase boundary.
+enum TracePhase { kTrStart = 0, kTrCounted, kTrHistSeen, kTrScanned, kTrScanSeen, kTrFinalized, kTrReady,
+                  kTrFirstRow, kTrIssued, kTrStored, kTrEnd };
+__device__ __forceinline__ void trace(const Params& p, int cta, int phase) {
+    if (p.trace) p.trace[(size_t)cta * kTraceSlots + phase] = global_ns();
 }
 
 // Wait until *flag == epoch.  Gives up after kWaitLimitNs (or as soon as *abort is set) and
@@ -192,6 +204,17 @@ __device__ __forceinline__ void bulk_wait_all() {
     asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory");
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async_smem() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+// Where the dispatch kernel keeps things in dynamic shared memory (byte offsets).
+struct SmemPlan {
+    int stages, stage_bytes;          // input row ring
+    int out_stage_bytes;              // FP8: kOutStages quantised rows
+    int off_out, off_ids, off_loc_e, off_loc_r, off_pos, off_hist, off_arr, off_order;
+    int total;
+};
 
 // Barrier among a subset of the CTA's warps (id 1..15), `nthreads` a multiple of 32.
 __device__ __forceinline__ void group_sync(int id, int nthreads) {

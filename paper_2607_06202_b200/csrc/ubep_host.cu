@@ -17,11 +17,12 @@ namespace {
 std::atomic<uint64_t> g_launches{0};
 
 constexpr size_t kAlign = 256;
+constexpr int64_t kLocalMaxSlots = 8192;  // AUTO uses the flag-free kernel up to this many (token, slot) pairs
 inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 
 struct ArenaLayout {
     size_t off[UBEP_VIEW_COUNT_];
-    size_t slot_aux, slot_pos, chunk_hist, partial, chunk_base;
+    size_t slot_aux, slot_pos, chunk_hist, partial, chunk_base, trace;
     size_t flags_begin, hist_flag, scan_flag, status, ticket, epoch_ctr, done_ticket, order_pos, flags_end;
     size_t total;
     int er_cap, nchunks, S, rowB, G, B;
@@ -75,6 +76,7 @@ ArenaLayout make_layout(const ubep_config_t& c, int nchunks) {
     a.chunk_hist = take(n * B * 4);
     a.partial = take(S * B * 4);
     a.chunk_base = take(n * B * 4);
+    a.off[UBEP_VIEW_TRACE] = a.trace = take(n * ubep::kTraceSlots * 8);
     a.flags_begin = at;
     a.hist_flag = take(n * 4);
     a.scan_flag = take(R * 4);
@@ -99,6 +101,7 @@ struct ubep_buffer {
     int max_smem;
     uint32_t epoch;
     int32_t withhold;
+    int32_t tracing;
     cudaStream_t last_stream;
     const int32_t* phys;
     const int32_t* ncopies;
@@ -125,6 +128,7 @@ Params make_params(ubep_buffer* b, int T) {
     p.T = T; p.H = c.hidden; p.E = c.num_experts; p.R = c.num_ranks; p.L = p.E / p.R; p.k = c.topk;
     p.S = a.S; p.cap = c.rows_per_rank_cap; p.payload = c.payload; p.dedup = c.dedup;
     p.rowB = a.rowB; p.G = a.G; p.B = a.B; p.nchunks = a.nchunks; p.er_cap = a.er_cap;
+    p.parts = 1; p.grid = a.nchunks;
     p.epoch_ctr = at<unsigned>(b, a.epoch_ctr);
     p.done_ticket = at<unsigned>(b, a.done_ticket);
     p.withhold = -1;
@@ -153,6 +157,7 @@ Params make_params(ubep_buffer* b, int T) {
     p.scan_flag = at<unsigned>(b, a.scan_flag);
     p.arrival = at<unsigned>(b, a.off[UBEP_VIEW_ARRIVAL]);
     p.status = at<int32_t>(b, a.status);
+    p.trace = b->tracing ? at<unsigned long long>(b, a.trace) : nullptr;
     return p;
 }
 
@@ -203,6 +208,7 @@ int ubep_buffer_create(const ubep_config_t* cfg, void* dev_arena, size_t bytes, 
     b->arena = static_cast<uint8_t*>(dev_arena);
     b->epoch = 0;
     b->withhold = -1;
+    b->tracing = 0;
     b->last_stream = nullptr;
     b->phys = nullptr;
     b->ncopies = nullptr;
@@ -296,12 +302,40 @@ int ubep_dispatch(ubep_buffer_t* buf, const void* x, const int32_t* topk_idx, co
     p.topk_w = topk_w;
     p.withhold = buf->withhold;
     buf->withhold = -1;
-    int mode = buf->cfg.pipeline == UBEP_PIPELINE_AUTO ? UBEP_PIPELINE_FUSED : buf->cfg.pipeline;
-    if (mode == UBEP_PIPELINE_LOCAL) mode = UBEP_PIPELINE_FUSED;
-    int stages = 0, stage_bytes = 0, launches = 0;
-    size_t smem = 0;
-    if (ubep::plan_dispatch(p, buf->max_smem, &stages, &stage_bytes, &smem) != 0) return UBEP_ERR_ARG;
-    cudaError_t e = ubep::launch_dispatch(p, mode, stages, stage_bytes, smem, st, &launches);
+    // AUTO: a routing table that fits in shared memory is cheaper to recount in every CTA
+    // than to exchange through flags; larger ones use the decomposed kernel.
+    int mode = buf->cfg.pipeline;
+    if (mode == UBEP_PIPELINE_AUTO)
+        mode = (int64_t)T * p.k <= kLocalMaxSlots ? UBEP_PIPELINE_LOCAL : UBEP_PIPELINE_FUSED;
+    ubep::SmemPlan pl{};
+    int launches = 0;
+    p.parts = 1;
+    p.grid = p.nchunks;
+    if (mode == UBEP_PIPELINE_LOCAL) {
+        // split rows into column parts until the slices of work are balanced to ~5 %
+        const int n = buf->lay.nchunks;
+        int best = 1;
+        for (int parts = 1; parts <= 8; parts *= 2) {
+            const int chunks = n / parts;
+            if (chunks < 1 || (p.H * 2 / parts) % 16 != 0 || (p.H * 2) % parts != 0) break;
+            if (p.payload && ((p.H / parts) % 128 != 0 || p.H % parts != 0)) break;
+            best = parts;
+            const double per = (double)T / chunks;
+            if (per / (double)((T + chunks - 1) / chunks) >= 0.95) break;
+        }
+        p.parts = best;
+        p.nchunks = n / best;
+        p.grid = p.nchunks * best;
+        if (ubep::plan_dispatch(p, mode, buf->max_smem, &pl) != 0) {
+            if (buf->cfg.pipeline == UBEP_PIPELINE_LOCAL) return UBEP_ERR_ARG;
+            mode = UBEP_PIPELINE_FUSED;   // table too large for shared memory
+            p.parts = 1;
+            p.nchunks = n;
+            p.grid = n;
+        }
+    }
+    if (mode != UBEP_PIPELINE_LOCAL && ubep::plan_dispatch(p, mode, buf->max_smem, &pl) != 0) return UBEP_ERR_ARG;
+    cudaError_t e = ubep::launch_dispatch(p, mode, pl, st, &launches);
     if (e != cudaSuccess) return cuda_fail(buf, e);
     g_launches += launches;
     return UBEP_OK;
@@ -348,6 +382,7 @@ int ubep_view(ubep_buffer_t* buf, int which, void** dev_ptr, int64_t shape[4]) {
         case UBEP_VIEW_SLOT_ROW: s[0] = c.max_tokens; s[1] = k; break;
         case UBEP_VIEW_ARRIVAL: s[0] = 2; s[1] = R; break;
         case UBEP_VIEW_EPOCH: s[0] = 1; break;
+        case UBEP_VIEW_TRACE: s[0] = a.nchunks; s[1] = ubep::kTraceSlots; break;
         default: return UBEP_ERR_ARG;
     }
     if (!present) {
@@ -384,6 +419,12 @@ uint64_t ubep_launch_count(void) { return g_launches.load(); }
 int ubep_debug_withhold_flag(ubep_buffer_t* buf, int32_t chunk) {
     if (!buf || chunk < -1 || chunk >= buf->lay.nchunks) return UBEP_ERR_ARG;
     buf->withhold = chunk;
+    return UBEP_OK;
+}
+
+int ubep_debug_trace(ubep_buffer_t* buf, int32_t enable) {
+    if (!buf) return UBEP_ERR_ARG;
+    buf->tracing = enable != 0;
     return UBEP_OK;
 }
 

@@ -2,10 +2,12 @@
 //
 //   count_kernel / scan_kernel        TokenCnt and CalCumSum as separate launches (the
 //                                     bulk-synchronous pipeline; kernel boundaries = barriers)
-//   dispatch_kernel<mode, fp8>        persistent CTA per token chunk: layout warps + a mover
-//                                     warp that streams rows with TMA bulk copies; in fused
-//                                     mode the layout steps are ordered by release/acquire
-//                                     flags instead of launches (kernel decomposition)
+//   dispatch_kernel<mode, fp8>        persistent CTA per work slice: layout warps plus a mover
+//                                     warp that streams rows with TMA bulk copies.  FUSED: the
+//                                     layout steps of different CTAs are ordered by
+//                                     release/acquire flags instead of launches (kernel
+//                                     decomposition).  LOCAL: every CTA derives its offsets
+//                                     from the whole routing table (small T*k, no flags).
 //   combine_kernel<K>                 gather + fp32 weighted sum + one bf16 rounding
 //   layout_kernel                     counts only (ubep_get_dispatch_layout)
 #include <cuda_fp8.h>
@@ -17,14 +19,23 @@ namespace ubep {
 
 // --------------------------------------------------------------- phased: count / scan
 
+// One warp per token chunk; chunk-local counts go to slot_aux (expert) / slot_row (rank).
 __global__ void __launch_bounds__(32) count_kernel(const Params p) {
     extern __shared__ int sm_i[];
-    count_chunk(p, blockIdx.x, sm_i, threadIdx.x);
+    const int c = blockIdx.x, lane = threadIdx.x;
+    const int t0 = (int)chunk_begin(c, p.T, p.nchunks), t1 = (int)chunk_begin(c + 1, p.T, p.nchunks);
+    int* hist = sm_i;
+    int* ids = sm_i + p.B;
+    stage_ids(p, t0, t1, ids, lane, 32);
+    __syncwarp();
+    count_slots(p, t0, t1, ids, hist, p.slot_aux + (size_t)t0 * p.k, p.slot_row + (size_t)t0 * p.k, p.partial, lane);
+    for (int b = lane; b < p.B; b += 32) p.chunk_hist[(size_t)c * p.B + b] = hist[b];
 }
 
 __global__ void __launch_bounds__(256) scan_kernel(const Params p) {
     extern __shared__ int sm_i[];
-    scan_rank(p, blockIdx.x, sm_i, threadIdx.x / 32, 8, threadIdx.x % 32, 1);
+    scan_rank_publish(p, blockIdx.x, sm_i, threadIdx.x / 32, 8, threadIdx.x % 32, 1);
+    scan_rank_sources(p, blockIdx.x, sm_i, threadIdx.x, 256);
 }
 
 // ------------------------------------------------------------------ FP8 quantisation
@@ -60,47 +71,67 @@ __device__ __forceinline__ void quantize8(const uint4 in, bool valid, uint2& out
 }
 
 // --------------------------------------------------------------------- dispatch kernel
-// Shared memory carve-up (dynamic): [stages * stage_bytes] row ring, then int arrays
-// hist[B] (also scratch of scan_rank), arr[R], pos[chunk_slots].
+// Warp roles: warp 0 = mover (one elected thread issues the TMA loads and, for bf16 rows,
+// the TMA stores); warps 1..15 = layout group (count, prefix sums, row assignment); with
+// FP8 rows warp 1 then becomes the store issuer and warps 2..15 quantise.
 template <int kMode, bool kFp8>
-__global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, int stages, int stage_bytes) {
+__global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, const SmemPlan pl) {
     extern __shared__ __align__(128) uint8_t smem[];
-    __shared__ __align__(8) uint64_t full_bar[kMaxStages];
-    __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
-    __shared__ __align__(8) uint64_t ready_bar;
+    __shared__ __align__(8) uint64_t full_bar[kMaxStages];    // input row landed
+    __shared__ __align__(8) uint64_t empty_bar[kMaxStages];   // FP8: input row consumed
+    __shared__ __align__(8) uint64_t out_full[kOutStages];    // FP8: quantised row written
+    __shared__ __align__(8) uint64_t out_empty[kOutStages];   // FP8: its stores have read it
+    __shared__ __align__(8) uint64_t ready_bar;               // rows assigned, movers may go
     __shared__ int abort_flag;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int c = blockIdx.x;
-    const int t0 = (int)chunk_begin(c, p.T, p.nchunks), t1 = (int)chunk_begin(c + 1, p.T, p.nchunks);
+    const int part = c % p.parts, ch = c / p.parts;
+    const int t0 = (int)chunk_begin(ch, p.T, p.nchunks), t1 = (int)chunk_begin(ch + 1, p.T, p.nchunks);
     const int ntok = t1 - t0;
-    int* hist = reinterpret_cast<int*>(smem + (size_t)stages * stage_bytes);
-    int* arr = hist + p.B;
-    int* pos = arr + p.R;
+    const int stages = pl.stages;
+    int* ids_sm = reinterpret_cast<int*>(smem + pl.off_ids);
+    int* loc_e_sm = reinterpret_cast<int*>(smem + pl.off_loc_e);
+    int* loc_r_sm = reinterpret_cast<int*>(smem + pl.off_loc_r);
+    int* pos = reinterpret_cast<int*>(smem + pl.off_pos);
+    int* hist = reinterpret_cast<int*>(smem + pl.off_hist);
+    int* arr = reinterpret_cast<int*>(smem + pl.off_arr);
+    int* order_sm = reinterpret_cast<int*>(smem + pl.off_order);
     volatile int* abortp = &abort_flag;
     int issued = 0;  // rows whose load thread 0 has started
     const unsigned epoch = current_epoch(p);
 
     constexpr int gn = kThreads - 32;  // layout group: warps 1..15
     constexpr int nw = kWarps - 1;
+    constexpr int nq = kWarps - 2;     // FP8: quantising warps 2..15
     const int gtid = tid - 32, gw = warp - 1;
 
     if (tid == 0) {
         for (int s = 0; s < stages; ++s) {
             mbar_init(&full_bar[s], 1);
-            mbar_init(&empty_bar[s], nw);
+            mbar_init(&empty_bar[s], nq);
+        }
+        for (int s = 0; s < kOutStages; ++s) {
+            mbar_init(&out_full[s], nq);
+            mbar_init(&out_empty[s], 1);
         }
         mbar_init(&ready_bar, 1);
         abort_flag = 0;
         mbar_fence_init();
     }
-    for (int r = tid; r < p.R; r += kThreads) arr[r] = 0;
+    for (int r = tid; r < p.R; r += kThreads) {
+        arr[r] = 0;
+        order_sm[r] = __ldg(p.order_pos + r);
+    }
     // the arrival counters of the next call live in the other half; clear them now
     if (c == 0)
         for (int r = tid; r < p.R; r += kThreads) p.arrival[((epoch + 1) & 1) * p.R + r] = 0;
     __syncthreads();
+    if (tid == 0) trace(p, c, kTrStart);
 
-    const unsigned row_in_bytes = (unsigned)p.H * 2u;
+    const unsigned in_bytes = (unsigned)(p.H * 2 / p.parts);   // this CTA's piece of a bf16 row
+    const unsigned out_bytes = (unsigned)(p.rowB / p.parts);   // and of a payload row
+    const size_t in_off = (size_t)part * in_bytes, out_off = (size_t)part * out_bytes;
 
     if (warp == 0) {
         // ------------------------------------------------ mover warp (one elected thread)
@@ -108,8 +139,10 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, i
             bool ok = true;
             auto issue_load = [&](int n) {
                 const int s = n % stages;
-                mbar_arrive_expect_tx(&full_bar[s], row_in_bytes);
-                bulk_load(smem + (size_t)s * stage_bytes, p.x + (size_t)(t0 + n) * p.H, row_in_bytes, &full_bar[s]);
+                mbar_arrive_expect_tx(&full_bar[s], in_bytes);
+                bulk_load(smem + (size_t)s * pl.stage_bytes,
+                          reinterpret_cast<const uint8_t*>(p.x) + (size_t)(t0 + n) * p.H * 2 + in_off, in_bytes,
+                          &full_bar[s]);
             };
             if (!kFp8) {
                 // loads run (stages - 3) rows ahead; up to 3 rows' stores stay in flight
@@ -120,10 +153,11 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, i
                     const int s = n % stages;
                     ok = mbar_wait(&full_bar[s], (n / stages) & 1, abortp);
                     if (!ok) break;
-                    const uint8_t* src = smem + (size_t)s * stage_bytes;
+                    if (n == 0) trace(p, c, kTrFirstRow);
+                    const uint8_t* src = smem + (size_t)s * pl.stage_bytes;
                     for (int j = 0; j < p.k; ++j) {
                         const int where = pos[n * p.k + j];
-                        if (where >= 0) bulk_store(p.recv_x + (size_t)where * p.rowB, src, (unsigned)p.rowB);
+                        if (where >= 0) bulk_store(p.recv_x + (size_t)where * p.rowB + out_off, src, out_bytes);
                     }
                     bulk_commit();
                     if (issued < ntok) {
@@ -133,7 +167,7 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, i
                     }
                 }
             } else {
-                // loader only; the layout group quantises and stores, and frees the stages
+                // loader only; the quantising warps free the stages
                 for (int n = 0; ok && n < ntok; ++n) {
                     const int s = n % stages;
                     if (n >= stages) ok = mbar_wait(&empty_bar[s], ((n / stages) - 1) & 1, abortp);
@@ -143,98 +177,249 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, i
                 }
             }
             if (!ok) {
-                // a wait gave up: record it and let everybody leave
-                report(p.status, kErrTimeout);
+                report(p.status, kErrTimeout);  // a wait gave up: record it and let everybody leave
                 abort_flag = 1;
             }
+            trace(p, c, kTrIssued);
             bulk_wait_all<0>();
+            trace(p, c, kTrStored);
         }
     } else {
         // ------------------------------------------------------------- layout group
         bool ok = true;
-        if (kMode == kModeFused) {
-            if (gw == 0) count_chunk(p, c, hist, lane);
+        const int* ids = ids_sm;           // resolved ids of this CTA's tokens
+        const int* loc_e = loc_e_sm;
+        const int* loc_r = loc_r_sm;
+        if (kMode == kModeLocal) {
+            // every CTA: whole routing table -> totals and the prefix before its own tokens
+            int* tot = hist;
+            int* pre = hist + p.B;
+            int* spre = hist + 2 * p.B;
+            int* scnt = hist + 3 * p.B;
+            int* scratch = hist + 4 * p.B;
+            int* eo = hist + 5 * p.B;
+            stage_ids(p, 0, p.T, ids_sm, gtid, gn);
+            for (int b = gtid; b < 4 * p.B; b += gn) hist[b] = 0;
             group_sync(1, gn);
-            if (gtid == 0 && c != p.withhold) {
-                __threadfence();
-                st_release(p.hist_flag + c, epoch);
+            int duty_s = (part == 0 && ch < p.S) ? ch : -1;
+            local_histograms(p, ids_sm, t0, duty_s, tot, pre, spre, scnt, gtid, gn);
+            group_sync(1, gn);
+            for (int e = gtid; e < p.E; e += gn) {
+                int o = 0;
+                for (int q = (e / p.L) * p.L; q < e; ++q) o += tot[q];
+                eo[e] = o;
             }
-            // CalCumSum duty: this CTA serves rank c (and c + nchunks, ...)
-            bool lost = false;  // a wait of this thread ran out
-            for (int r = c; r < p.R; r += p.nchunks) {
-                for (int cc = gtid; cc < p.nchunks; cc += gn)
-                    if (!wait_flag(p.hist_flag + cc, epoch, abortp)) lost = true;
-                if (group_or(1, gn, lost || *abortp)) { lost = true; break; }  // same answer for all
-                scan_rank(p, r, hist, gw, nw, lane, 1);
-                group_sync(1, gn);
-                if (gtid == 0) {
-                    __threadfence();
-                    st_release(p.scan_flag + r, epoch);
+            ids = ids_sm + (size_t)t0 * p.k;
+            if (gw == 0) count_slots(p, t0, t1, ids, scratch, loc_e_sm, loc_r_sm, nullptr, lane);
+            group_sync(1, gn);
+            if (gtid == 0) trace(p, c, kTrScanSeen);
+            finalize_chunk(p, t0, t1, ids, loc_e, loc_r, [&](int e) { return eo[e] + pre[e]; },
+                           [&](int r) { return pre[p.E + r]; }, part == 0, pos, arr, gtid, gn);
+            group_sync(1, gn);
+            if (gtid == 0) trace(p, c, kTrFinalized);
+            order_destinations(p, c, order_sm, pos, ntok, gtid, gn);
+            group_sync(1, gn);
+            if (gtid == 0) {
+                mbar_arrive(&ready_bar);
+                trace(p, c, kTrReady);
+            }
+            // outputs nobody inside this kernel waits for
+            if (c == 0) {
+                for (int e = gtid; e < p.E; e += gn) {
+                    p.expert_offset[e] = eo[e];
+                    p.num_tokens_per_expert[e] = tot[e];
+                }
+                for (int r = gtid; r < p.R; r += gn) {
+                    p.num_tokens_per_rank[r] = tot[p.E + r];
+                    int rows = tot[p.E + r];
+                    if (!p.dedup) {
+                        rows = 0;
+                        for (int q = r * p.L; q < (r + 1) * p.L; ++q) rows += tot[q];
+                    }
+                    p.num_rows_per_rank[r] = rows;
                 }
             }
-            // every slot of this chunk may need any rank's bases
-            if (!lost)
-                for (int r = gtid; r < p.R; r += gn)
-                    if (!wait_flag(p.scan_flag + r, epoch, abortp)) lost = true;
-            ok = !group_or(1, gn, lost || *abortp);
-            if (!ok && gtid == 0) {
-                report(p.status, kErrTimeout);
-                abort_flag = 1;
+            while (duty_s >= 0) {
+                for (int e = gtid; e < p.E; e += gn) {
+                    p.cnt[(size_t)duty_s * p.E + e] = scnt[e];
+                    p.src_offset[(size_t)duty_s * p.E + e] = eo[e] + spre[e];
+                }
+                duty_s += p.nchunks;   // more source ranks than chunks: another pass per extra rank
+                if (duty_s >= p.S) break;
+                group_sync(1, gn);
+                for (int b = gtid; b < 2 * p.B; b += gn) spre[b] = 0;   // spre and scnt are adjacent
+                group_sync(1, gn);
+                local_histograms(p, ids_sm, 0, duty_s, scratch, scratch, spre, scnt, gtid, gn);
+                group_sync(1, gn);
             }
-        }
-        if (ok) {
-            finalize_chunk(p, c, pos, arr, gtid, gn);
+        } else {
+            stage_ids(p, t0, t1, ids_sm, gtid, gn);
             group_sync(1, gn);
-            order_destinations(p, c, pos, ntok, gtid, gn);
-            group_sync(1, gn);
-        }
-        if (gtid == 0) mbar_arrive(&ready_bar);
-        if (kFp8 && ok) {
-            const int nvec = p.H / 8;
-            for (int n = 0; n < ntok; ++n) {
-                const int s = n % stages;
-                if (!mbar_wait(&full_bar[s], (n / stages) & 1, abortp)) break;
-                const uint8_t* src = smem + (size_t)s * stage_bytes;
-                for (int vb = gw * 32; vb < nvec; vb += gn) {
-                    const int v = vb + lane;
-                    const bool valid = v < nvec;
-                    uint4 in = make_uint4(0, 0, 0, 0);
-                    if (valid) in = *reinterpret_cast<const uint4*>(src + (size_t)v * 16);
-                    uint2 q;
-                    float scale;
-                    quantize8(in, valid, q, scale);
-                    if (valid) {
-                        for (int j = 0; j < p.k; ++j) {
-                            const int where = pos[n * p.k + j];
-                            if (where < 0) continue;
-                            *reinterpret_cast<uint2*>(p.recv_x + (size_t)where * p.rowB + (size_t)v * 8) = q;
-                            if ((lane & 15) == 0) p.recv_scale[(size_t)where * p.G + (v >> 4)] = scale;
-                        }
+            if (kMode == kModeFused) {
+                if (gw == 0) {
+                    count_slots(p, t0, t1, ids_sm, hist, loc_e_sm, loc_r_sm, p.partial, lane);
+                    for (int b = lane; b < p.B; b += 32) p.chunk_hist[(size_t)ch * p.B + b] = hist[b];
+                    __syncwarp();
+                    if (lane == 0 && ch != p.withhold) {
+                        __threadfence();
+                        st_release(p.hist_flag + ch, epoch);
+                    }
+                    if (lane == 0) trace(p, c, kTrCounted);
+                }
+                group_sync(1, gn);
+                // CalCumSum duty: this CTA serves rank c (and c + nchunks, ...)
+                bool lost = false;  // a wait of this thread ran out
+                int deferred = -1;
+                for (int r = ch; r < p.R; r += p.nchunks) {
+                    for (int cc = gtid; cc < p.nchunks; cc += gn)
+                        if (!wait_flag(p.hist_flag + cc, epoch, abortp)) lost = true;
+                    if (group_or(1, gn, lost || *abortp)) { lost = true; break; }  // same answer for all
+                    if (gtid == 0) trace(p, c, kTrHistSeen);
+                    scan_rank_publish(p, r, hist, gw, nw, lane, 1);
+                    if (gtid == 0) {
+                        __threadfence();
+                        st_release(p.scan_flag + r, epoch);
+                        trace(p, c, kTrScanned);
+                    }
+                    if (r + p.nchunks < p.R) {
+                        scan_rank_sources(p, r, hist, gtid, gn);
+                        group_sync(1, gn);
+                    } else {
+                        deferred = r;   // cnt / src_offset: after our own movers are released
                     }
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&empty_bar[s]);
+                // every slot of this chunk may need any rank's bases
+                if (!lost)
+                    for (int r = gtid; r < p.R; r += gn)
+                        if (!wait_flag(p.scan_flag + r, epoch, abortp)) lost = true;
+                ok = !group_or(1, gn, lost || *abortp);
+                if (gtid == 0) trace(p, c, kTrScanSeen);
+                if (!ok && gtid == 0) {
+                    report(p.status, kErrTimeout);
+                    abort_flag = 1;
+                }
+                if (ok) {
+                    const int32_t* cb = p.chunk_base + (size_t)ch * p.B;
+                    finalize_chunk(p, t0, t1, ids, loc_e, loc_r,
+                                   [&](int e) { return __ldcg(p.expert_offset + e) + __ldcg(cb + e); },
+                                   [&](int r) { return __ldcg(cb + p.E + r); }, true, pos, arr, gtid, gn);
+                    group_sync(1, gn);
+                    if (gtid == 0) trace(p, c, kTrFinalized);
+                    order_destinations(p, c, order_sm, pos, ntok, gtid, gn);
+                    group_sync(1, gn);
+                }
+                if (gtid == 0) {
+                    mbar_arrive(&ready_bar);
+                    trace(p, c, kTrReady);
+                }
+                if (ok && deferred >= 0) scan_rank_sources(p, deferred, hist, gtid, gn);
+            } else {
+                // phased: counts and prefix sums were separate launches; local counts are in
+                // slot_aux (expert) / slot_row (rank)
+                loc_e = p.slot_aux + (size_t)t0 * p.k;
+                loc_r = p.slot_row + (size_t)t0 * p.k;
+                const int32_t* cb = p.chunk_base + (size_t)ch * p.B;
+                finalize_chunk(p, t0, t1, ids, loc_e, loc_r,
+                               [&](int e) { return __ldcg(p.expert_offset + e) + __ldcg(cb + e); },
+                               [&](int r) { return __ldcg(cb + p.E + r); }, true, pos, arr, gtid, gn);
+                group_sync(1, gn);
+                if (gtid == 0) trace(p, c, kTrFinalized);
+                order_destinations(p, c, order_sm, pos, ntok, gtid, gn);
+                group_sync(1, gn);
+                if (gtid == 0) {
+                    mbar_arrive(&ready_bar);
+                    trace(p, c, kTrReady);
+                }
+            }
+        }
+        if (kFp8 && ok) {
+            uint8_t* out_ring = smem + pl.off_out;
+            if (warp == 1) {
+                // ---------------------------------------- store issuer (one elected thread)
+                if (lane == 0) {
+                    bool sok = true;
+                    for (int n = 0; n < ntok; ++n) {
+                        const int os = n % kOutStages;
+                        sok = mbar_wait(&out_full[os], (n / kOutStages) & 1, abortp);
+                        if (!sok) break;
+                        if (n == 0) trace(p, c, kTrFirstRow);
+                        const uint8_t* src = out_ring + (size_t)os * pl.out_stage_bytes;
+                        for (int j = 0; j < p.k; ++j) {
+                            const int where = pos[n * p.k + j];
+                            if (where >= 0) bulk_store(p.recv_x + (size_t)where * p.rowB + out_off, src, out_bytes);
+                        }
+                        bulk_commit();
+                        if (n + 1 >= kOutStages) {
+                            bulk_wait_read<kOutStages - 1>();          // the oldest row's stores have read it
+                            mbar_arrive(&out_empty[(n + 1) % kOutStages]);
+                        }
+                    }
+                    if (!sok) {
+                        report(p.status, kErrTimeout);
+                        abort_flag = 1;
+                    }
+                    bulk_wait_all<0>();
+                }
+            } else {
+                // ------------------------------------------------- quantising warps 2..15
+                const int qw = warp - 2;
+                const int nvec = (int)in_bytes / 16;          // 8-channel vectors in this CTA's piece
+                const int g0 = part * (p.G / p.parts);        // first scale group of the piece
+                for (int n = 0; n < ntok; ++n) {
+                    const int s = n % stages, os = n % kOutStages;
+                    if (!mbar_wait(&full_bar[s], (n / stages) & 1, abortp)) break;
+                    if (n >= kOutStages && !mbar_wait(&out_empty[os], ((n / kOutStages) - 1) & 1, abortp)) break;
+                    const uint8_t* src = smem + (size_t)s * pl.stage_bytes;
+                    uint8_t* dst = out_ring + (size_t)os * pl.out_stage_bytes;
+                    for (int vb = qw * 32; vb < nvec; vb += nq * 32) {
+                        const int v = vb + lane;
+                        const bool valid = v < nvec;
+                        uint4 in = make_uint4(0, 0, 0, 0);
+                        if (valid) in = *reinterpret_cast<const uint4*>(src + (size_t)v * 16);
+                        uint2 q;
+                        float scale;
+                        quantize8(in, valid, q, scale);
+                        if (valid) {
+                            *reinterpret_cast<uint2*>(dst + (size_t)v * 8) = q;
+                            if ((lane & 15) == 0) {
+                                for (int j = 0; j < p.k; ++j) {
+                                    const int where = pos[n * p.k + j];
+                                    if (where >= 0) p.recv_scale[(size_t)where * p.G + g0 + (v >> 4)] = scale;
+                                }
+                            }
+                        }
+                    }
+                    fence_proxy_async_smem();   // the bulk stores read what we just wrote
+                    __syncwarp();
+                    if (lane == 0) {
+                        mbar_arrive(&out_full[os]);
+                        mbar_arrive(&empty_bar[s]);
+                    }
+                }
             }
         }
     }
     __syncthreads();
     if (abort_flag) {
         // leaving early: the newest load of every ring stage may still be landing
-        if (tid == 0)
+        if (tid == 0) {
             for (int n = max(0, issued - stages); n < issued; ++n)
                 (void)mbar_wait(&full_bar[n % stages], (n / stages) & 1, nullptr);
-        if (tid == 0) finish_dispatch(p, epoch);
+            finish_dispatch(p, epoch);
+        }
         return;
     }
-    // rows of this chunk have landed: add them to the per-region arrival counters
-    {
-        __threadfence();
-        fence_proxy_async();
-        for (int r = tid; r < p.R; r += kThreads)
-            if (arr[r]) red_release_add(p.arrival + (epoch & 1) * p.R + r, (unsigned)arr[r]);
-    }
+    // pieces of this CTA's rows have landed: add them to the per-region arrival counters
+    // (unit: eighths of a row, so that the total does not depend on the column split)
+    __threadfence();
+    fence_proxy_async();
+    for (int r = tid; r < p.R; r += kThreads)
+        if (arr[r]) red_release_add(p.arrival + (epoch & 1) * p.R + r, (unsigned)(arr[r] * (8 / p.parts)));
     __syncthreads();
-    if (tid == 0) finish_dispatch(p, epoch);
+    if (tid == 0) {
+        trace(p, c, kTrEnd);
+        finish_dispatch(p, epoch);
+    }
 }
 
 // ---------------------------------------------------------------------------- combine
@@ -360,48 +545,63 @@ __global__ void __launch_bounds__(256) layout_kernel(const Params p, int32_t* nu
 
 // ------------------------------------------------------------------------- launchers
 
-static size_t dispatch_smem_bytes(const Params& p, int stages, int stage_bytes) {
-    const int chunk_tokens = (p.T + p.nchunks - 1) / p.nchunks;
-    return (size_t)stages * stage_bytes + sizeof(int) * ((size_t)p.B + p.R + (size_t)chunk_tokens * p.k) + 16;
-}
+static int round_up_i(int v, int m) { return (v + m - 1) / m * m; }
 
-int plan_dispatch(const Params& p, int max_smem, int* stages, int* stage_bytes, size_t* smem) {
-    const int sb = ((p.H * 2 + 127) / 128) * 128;
+// Shared-memory plan of the dispatch kernel for one call; -1 if it cannot fit.
+int plan_dispatch(const Params& p, int mode, int max_smem, SmemPlan* out) {
+    SmemPlan pl{};
     const int chunk_tokens = (p.T + p.nchunks - 1) / p.nchunks;
-    const size_t fixed = sizeof(int) * ((size_t)p.B + p.R + (size_t)chunk_tokens * p.k) + 16 + 1024;
-    if (fixed + 4 * (size_t)sb > (size_t)max_smem) return -1;
-    int st = (int)(((size_t)max_smem - fixed) / sb);
-    if (st > kMaxStages) st = kMaxStages;
-    *stages = st;
-    *stage_bytes = sb;
-    *smem = dispatch_smem_bytes(p, st, sb);
+    const int chunk_slots = chunk_tokens * p.k;
+    const int64_t ids_ints = mode == kModeLocal ? (int64_t)p.T * p.k : chunk_slots;
+    const int hist_ints = mode == kModeLocal ? 5 * p.B + p.E : p.B;
+    pl.stage_bytes = round_up_i(p.H * 2 / p.parts, 128);
+    pl.out_stage_bytes = p.payload ? round_up_i(p.rowB / p.parts, 128) : 0;
+    const int64_t ints = ids_ints + 3 * (int64_t)chunk_slots + hist_ints + 2 * p.R;
+    const int64_t fixed = (int64_t)kOutStages * pl.out_stage_bytes + ints * 4 + 128 + 1024;  // 1 KB: static smem
+    if (fixed + 4 * (int64_t)pl.stage_bytes > max_smem) return -1;
+    pl.stages = (int)((max_smem - fixed) / pl.stage_bytes);
+    if (pl.stages > kMaxStages) pl.stages = kMaxStages;
+    int at = pl.stages * pl.stage_bytes;
+    pl.off_out = at; at += kOutStages * pl.out_stage_bytes;
+    pl.off_ids = at; at += (int)ids_ints * 4;
+    pl.off_loc_e = at; at += chunk_slots * 4;
+    pl.off_loc_r = at; at += chunk_slots * 4;
+    pl.off_pos = at; at += chunk_slots * 4;
+    pl.off_hist = at; at += hist_ints * 4;
+    pl.off_arr = at; at += p.R * 4;
+    pl.off_order = at; at += p.R * 4;
+    pl.total = round_up_i(at, 128);
+    *out = pl;
     return 0;
 }
 
 template <int kMode, bool kFp8>
-static cudaError_t launch_dispatch_t(const Params& p, int stages, int stage_bytes, size_t smem, cudaStream_t st) {
+static cudaError_t launch_dispatch_t(const Params& p, const SmemPlan& pl, cudaStream_t st) {
     auto kern = dispatch_kernel<kMode, kFp8>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.total);
     if (e != cudaSuccess) return e;
-    kern<<<p.nchunks, kThreads, smem, st>>>(p, stages, stage_bytes);
+    kern<<<p.grid, kThreads, pl.total, st>>>(p, pl);
     return cudaGetLastError();
 }
 
-cudaError_t launch_dispatch(const Params& p, int mode, int stages, int stage_bytes, size_t smem, cudaStream_t st,
-                            int* launches) {
+cudaError_t launch_dispatch(const Params& p, int mode, const SmemPlan& pl, cudaStream_t st, int* launches) {
     cudaError_t e;
+    *launches = 1;
     if (mode == kModePhased) {
-        count_kernel<<<p.nchunks, 32, sizeof(int) * p.B, st>>>(p);
+        const int chunk_slots = ((p.T + p.nchunks - 1) / p.nchunks) * p.k;
+        count_kernel<<<p.nchunks, 32, sizeof(int) * (p.B + chunk_slots), st>>>(p);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
         scan_kernel<<<p.R, 256, sizeof(int) * (p.L + 1), st>>>(p);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
         *launches = 3;
-        return p.payload ? launch_dispatch_t<kModePhased, true>(p, stages, stage_bytes, smem, st)
-                         : launch_dispatch_t<kModePhased, false>(p, stages, stage_bytes, smem, st);
+        return p.payload ? launch_dispatch_t<kModePhased, true>(p, pl, st)
+                         : launch_dispatch_t<kModePhased, false>(p, pl, st);
     }
-    *launches = 1;
-    return p.payload ? launch_dispatch_t<kModeFused, true>(p, stages, stage_bytes, smem, st)
-                     : launch_dispatch_t<kModeFused, false>(p, stages, stage_bytes, smem, st);
+    if (mode == kModeLocal)
+        return p.payload ? launch_dispatch_t<kModeLocal, true>(p, pl, st)
+                         : launch_dispatch_t<kModeLocal, false>(p, pl, st);
+    return p.payload ? launch_dispatch_t<kModeFused, true>(p, pl, st)
+                     : launch_dispatch_t<kModeFused, false>(p, pl, st);
 }
 
 cudaError_t launch_combine(const uint16_t* y, const int32_t* slot_pos, const float* topk_w, int T, int H, int k,

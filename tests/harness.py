@@ -97,7 +97,7 @@ def check_dispatch(buf: B.Buffer, wl: W.Workload, lay, cap: int, recv, check_tai
             n = int(lay.num_tokens_per_expert[r * cfg.L:(r + 1) * cfg.L].sum())
             assert np.array_equal(er[r, :n], lay.expert_rows[r, :n]), f"expert_rows[{r}]"
     arrival = buf.arrival.cpu().numpy()[int(buf.epoch.item()) & 1]
-    assert np.array_equal(arrival, lay.num_rows_per_rank), "arrival counters"
+    assert np.array_equal(arrival, 8 * lay.num_rows_per_rank), "arrival counters"
 
 
 def bf16_ulp_distance(a_bits: np.ndarray, b_bits: np.ndarray) -> np.ndarray:
