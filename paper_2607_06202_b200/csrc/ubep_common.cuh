@@ -17,6 +17,7 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kMaxTopk = 32;
 constexpr int kMaxChunks = 320;        // scan keeps chunks/32 values per lane in registers
 constexpr int kMaxStages = 16;         // rows in the shared-memory ring
+constexpr int kRankWordsHost = 4;      // the rank-level fast path handles up to 128 ranks
 constexpr int kOutStages = 4;          // quantised rows waiting for their bulk stores (FP8)
 constexpr int kTraceSlots = 16;        // per-CTA phase time stamps (optional tracing)
 constexpr int kModePhased = 1, kModeFused = 2, kModeLocal = 3;
@@ -33,6 +34,8 @@ struct Params {
     int nchunks;     // token chunks (contiguous, equal to +-1 token)
     int parts;       // column parts per row: CTA c moves part c % parts of chunk c / parts
     int grid;        // CTAs of the dispatch kernel = nchunks * parts
+    unsigned L_magic;  // ceil(2^32 / L): e / L == umulhi(e, L_magic) for e < 65536
+    int local_fast;    // flag-free kernel: rank-level fast path (dedup, L < 32, R <= 128)
     int er_cap;      // entries per rank in expert_rows
     unsigned* epoch_ctr;    // device word: dispatches completed on this buffer
     unsigned* done_ticket;  // CTAs of the running dispatch kernel that have finished
@@ -212,7 +215,8 @@ __device__ __forceinline__ void fence_proxy_async_smem() {
 struct SmemPlan {
     int stages, stage_bytes;          // input row ring
     int out_stage_bytes;              // FP8: kOutStages quantised rows
-    int off_out, off_ids, off_loc_e, off_loc_r, off_pos, off_hist, off_arr, off_order;
+    int map_groups, map_wb, map_wbs, map_bp;  // bin bitmaps: 32-token groups, words, stride, padded bins
+    int off_out, off_ids, off_mask, off_bm, off_pos, off_key, off_ord, off_w, off_hist, off_arr, off_order;
     int total;
 };
 

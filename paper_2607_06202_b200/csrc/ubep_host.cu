@@ -30,6 +30,7 @@ struct ArenaLayout {
 
 bool valid_config(const ubep_config_t& c) {
     if (c.num_ranks < 1 || c.num_experts < 1 || c.num_experts % c.num_ranks != 0) return false;
+    if (c.num_experts > 65535) return false;  // staged slots pack the expert id into 16 bits
     if (c.topk < 1 || c.topk > ubep::kMaxTopk) return false;
     if (c.hidden < 8 || c.hidden % 8 != 0) return false;
     if (c.payload != UBEP_PAYLOAD_BF16 && c.payload != UBEP_PAYLOAD_FP8_E4M3) return false;
@@ -129,6 +130,8 @@ Params make_params(ubep_buffer* b, int T) {
     p.S = a.S; p.cap = c.rows_per_rank_cap; p.payload = c.payload; p.dedup = c.dedup;
     p.rowB = a.rowB; p.G = a.G; p.B = a.B; p.nchunks = a.nchunks; p.er_cap = a.er_cap;
     p.parts = 1; p.grid = a.nchunks;
+    p.L_magic = p.L == 1 ? 0xffffffffu : (unsigned)((0x100000000ull + (uint64_t)p.L - 1) / (uint64_t)p.L);
+    p.local_fast = (c.dedup && p.L < 32 && p.L > 1 && p.R <= 32 * ubep::kRankWordsHost) ? 1 : 0;
     p.epoch_ctr = at<unsigned>(b, a.epoch_ctr);
     p.done_ticket = at<unsigned>(b, a.done_ticket);
     p.withhold = -1;

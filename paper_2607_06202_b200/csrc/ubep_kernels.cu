@@ -19,17 +19,20 @@ namespace ubep {
 
 // --------------------------------------------------------------- phased: count / scan
 
-// One warp per token chunk; chunk-local counts go to slot_aux (expert) / slot_row (rank).
-__global__ void __launch_bounds__(32) count_kernel(const Params p) {
-    extern __shared__ int sm_i[];
-    const int c = blockIdx.x, lane = threadIdx.x;
+// TokenCnt of one token chunk per CTA: bin bitmaps -> chunk histogram and boundary snapshots.
+__global__ void __launch_bounds__(256) count_kernel(const Params p, const SmemPlan pl) {
+    extern __shared__ __align__(16) uint8_t sm_c[];
+    const int c = blockIdx.x, tid = threadIdx.x;
     const int t0 = (int)chunk_begin(c, p.T, p.nchunks), t1 = (int)chunk_begin(c + 1, p.T, p.nchunks);
-    int* hist = sm_i;
-    int* ids = sm_i + p.B;
-    stage_ids(p, t0, t1, ids, lane, 32);
-    __syncwarp();
-    count_slots(p, t0, t1, ids, hist, p.slot_aux + (size_t)t0 * p.k, p.slot_row + (size_t)t0 * p.k, p.partial, lane);
-    for (int b = lane; b < p.B; b += 32) p.chunk_hist[(size_t)c * p.B + b] = hist[b];
+    int* ids = reinterpret_cast<int*>(sm_c + (pl.off_ids - pl.off_ids));
+    BinMaps bmaps{reinterpret_cast<unsigned*>(sm_c + (pl.off_mask - pl.off_ids)),
+                  reinterpret_cast<unsigned*>(sm_c + (pl.off_bm - pl.off_ids)), pl.map_wb, pl.map_wbs, pl.map_bp,
+                  pl.map_groups};
+    stage_ids(p, t0, t1, ids, tid, 256);
+    __syncthreads();
+    build_bin_maps(p, ids, t1 - t0, bmaps, tid / 32, 8, tid % 32);
+    __syncthreads();
+    publish_chunk_counts(p, c, t0, t1, bmaps, tid, 256);
 }
 
 __global__ void __launch_bounds__(256) scan_kernel(const Params p) {
@@ -91,9 +94,13 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
     const int ntok = t1 - t0;
     const int stages = pl.stages;
     int* ids_sm = reinterpret_cast<int*>(smem + pl.off_ids);
-    int* loc_e_sm = reinterpret_cast<int*>(smem + pl.off_loc_e);
-    int* loc_r_sm = reinterpret_cast<int*>(smem + pl.off_loc_r);
-    int* pos = reinterpret_cast<int*>(smem + pl.off_pos);
+    int* pos = reinterpret_cast<int*>(smem + pl.off_ord);     // destinations in issue order
+    int* pos_raw = reinterpret_cast<int*>(smem + pl.off_pos);  // destinations in slot order
+    int* key = reinterpret_cast<int*>(smem + pl.off_key);
+    float* w_sm = reinterpret_cast<float*>(smem + pl.off_w);
+    const BinMaps bmaps{reinterpret_cast<unsigned*>(smem + pl.off_mask),
+                        reinterpret_cast<unsigned*>(smem + pl.off_bm), pl.map_wb, pl.map_wbs, pl.map_bp,
+                        pl.map_groups};
     int* hist = reinterpret_cast<int*>(smem + pl.off_hist);
     int* arr = reinterpret_cast<int*>(smem + pl.off_arr);
     int* order_sm = reinterpret_cast<int*>(smem + pl.off_order);
@@ -187,37 +194,60 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
     } else {
         // ------------------------------------------------------------- layout group
         bool ok = true;
-        const int* ids = ids_sm;           // resolved ids of this CTA's tokens
-        const int* loc_e = loc_e_sm;
-        const int* loc_r = loc_r_sm;
-        if (kMode == kModeLocal) {
-            // every CTA: whole routing table -> totals and the prefix before its own tokens
+        const int* ids = ids_sm;  // staged slots of this CTA's tokens
+        if (!(kMode == kModeLocal && p.local_fast))
+            for (int i = gtid; i < ntok * p.k; i += gn) w_sm[i] = __ldg(p.topk_w + (size_t)t0 * p.k + i);
+        if (kMode == kModeLocal && p.local_fast) {
+            // rank-level rows first, movers released, expert-level outputs afterwards
+            const RankMaps rm{bmaps.bm, bmaps.mask_t, (p.R + 31) / 32, ((p.R + 31) / 32) * 32, (p.T + 31) / 32};
+            int* row_sm = reinterpret_cast<int*>(w_sm);
+            local_stage_and_rank_maps(p, ids_sm, rm, gw, nw, lane);
+            group_sync(1, gn);
+            if (gtid == 0) trace(p, c, kTrCounted);
+            local_rows_dedup(p, t0, t1, ids_sm, rm, pos_raw, key, row_sm, arr, gtid, gn);
+            group_sync(1, gn);
+            if (gtid == 0) trace(p, c, kTrFinalized);
+            order_destinations(p, c, order_sm, pos_raw, key, pos, ntok * p.k, gtid, gn);
+            group_sync(1, gn);
+            if (gtid == 0) {
+                mbar_arrive(&ready_bar);
+                trace(p, c, kTrReady);
+            }
+            if (part == 0) local_meta_dedup(p, t0, t1, ids_sm, pos_raw, row_sm, gtid, gn);
+            for (int r = c; r < p.R; r += p.grid) local_rank_duty(p, r, ids_sm, rm, hist, gw, nw, lane, gtid, gn, 1);
+        } else if (kMode == kModeLocal) {
+            // every CTA: bitmaps over the whole routing table -> totals, the rows before its
+            // own tokens, and (CTAs with a source-rank duty) that rank's counts
             int* tot = hist;
             int* pre = hist + p.B;
-            int* spre = hist + 2 * p.B;
-            int* scnt = hist + 3 * p.B;
-            int* scratch = hist + 4 * p.B;
-            int* eo = hist + 5 * p.B;
+            int* eo = hist + 2 * p.B;
             stage_ids(p, 0, p.T, ids_sm, gtid, gn);
-            for (int b = gtid; b < 4 * p.B; b += gn) hist[b] = 0;
             group_sync(1, gn);
-            int duty_s = (part == 0 && ch < p.S) ? ch : -1;
-            local_histograms(p, ids_sm, t0, duty_s, tot, pre, spre, scnt, gtid, gn);
+            if (gtid == 0) trace(p, c, kTrCounted);
+            build_bin_maps(p, ids_sm, p.T, bmaps, gw, nw, lane);
+            group_sync(1, gn);
+            if (gtid == 0) trace(p, c, kTrHistSeen);
+            for (int b = gtid; b < p.B; b += gn) {
+                const int before = bits_in_range(bmaps, b, 0, t0);
+                pre[b] = before;
+                tot[b] = before + bits_in_range(bmaps, b, t0, p.T);
+            }
             group_sync(1, gn);
             for (int e = gtid; e < p.E; e += gn) {
                 int o = 0;
                 for (int q = (e / p.L) * p.L; q < e; ++q) o += tot[q];
                 eo[e] = o;
             }
-            ids = ids_sm + (size_t)t0 * p.k;
-            if (gw == 0) count_slots(p, t0, t1, ids, scratch, loc_e_sm, loc_r_sm, nullptr, lane);
             group_sync(1, gn);
             if (gtid == 0) trace(p, c, kTrScanSeen);
-            finalize_chunk(p, t0, t1, ids, loc_e, loc_r, [&](int e) { return eo[e] + pre[e]; },
-                           [&](int r) { return pre[p.E + r]; }, part == 0, pos, arr, gtid, gn);
+            ids = ids_sm + (size_t)t0 * p.k;
+            finalize_chunk(p, t0, t1, ids, w_sm,
+                           [&](int e, int tl) { return eo[e] + pre[e] + bits_in_range(bmaps, e, t0, t0 + tl); },
+                           [&](int r, int tl) { return pre[p.E + r] + bits_in_range(bmaps, p.E + r, t0, t0 + tl); },
+                           part == 0, pos_raw, key, arr, gtid, gn);
             group_sync(1, gn);
             if (gtid == 0) trace(p, c, kTrFinalized);
-            order_destinations(p, c, order_sm, pos, ntok, gtid, gn);
+            order_destinations(p, c, order_sm, pos_raw, key, pos, ntok * p.k, gtid, gn);
             group_sync(1, gn);
             if (gtid == 0) {
                 mbar_arrive(&ready_bar);
@@ -239,37 +269,32 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
                     p.num_rows_per_rank[r] = rows;
                 }
             }
-            while (duty_s >= 0) {
-                for (int e = gtid; e < p.E; e += gn) {
-                    p.cnt[(size_t)duty_s * p.E + e] = scnt[e];
-                    p.src_offset[(size_t)duty_s * p.E + e] = eo[e] + spre[e];
+            if (part == 0)
+                for (int s = ch; s < p.S; s += p.nchunks) {   // source ranks this CTA reports
+                    const int b0 = src_begin(s, p.T, p.S), b1 = src_begin(s + 1, p.T, p.S);
+                    for (int e = gtid; e < p.E; e += gn) {
+                        p.cnt[(size_t)s * p.E + e] = bits_in_range(bmaps, e, b0, b1);
+                        p.src_offset[(size_t)s * p.E + e] = eo[e] + bits_in_range(bmaps, e, 0, b0);
+                    }
                 }
-                duty_s += p.nchunks;   // more source ranks than chunks: another pass per extra rank
-                if (duty_s >= p.S) break;
-                group_sync(1, gn);
-                for (int b = gtid; b < 2 * p.B; b += gn) spre[b] = 0;   // spre and scnt are adjacent
-                group_sync(1, gn);
-                local_histograms(p, ids_sm, 0, duty_s, scratch, scratch, spre, scnt, gtid, gn);
-                group_sync(1, gn);
-            }
         } else {
             stage_ids(p, t0, t1, ids_sm, gtid, gn);
             group_sync(1, gn);
+            build_bin_maps(p, ids_sm, ntok, bmaps, gw, nw, lane);
+            group_sync(1, gn);
+            int deferred = -1;
             if (kMode == kModeFused) {
-                if (gw == 0) {
-                    count_slots(p, t0, t1, ids_sm, hist, loc_e_sm, loc_r_sm, p.partial, lane);
-                    for (int b = lane; b < p.B; b += 32) p.chunk_hist[(size_t)ch * p.B + b] = hist[b];
-                    __syncwarp();
-                    if (lane == 0 && ch != p.withhold) {
+                publish_chunk_counts(p, ch, t0, t1, bmaps, gtid, gn);
+                group_sync(1, gn);
+                if (gtid == 0) {
+                    if (ch != p.withhold) {
                         __threadfence();
                         st_release(p.hist_flag + ch, epoch);
                     }
-                    if (lane == 0) trace(p, c, kTrCounted);
+                    trace(p, c, kTrCounted);
                 }
-                group_sync(1, gn);
-                // CalCumSum duty: this CTA serves rank c (and c + nchunks, ...)
+                // CalCumSum duty: this CTA serves rank ch (and ch + nchunks, ...)
                 bool lost = false;  // a wait of this thread ran out
-                int deferred = -1;
                 for (int r = ch; r < p.R; r += p.nchunks) {
                     for (int cc = gtid; cc < p.nchunks; cc += gn)
                         if (!wait_flag(p.hist_flag + cc, epoch, abortp)) lost = true;
@@ -298,39 +323,29 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
                     report(p.status, kErrTimeout);
                     abort_flag = 1;
                 }
-                if (ok) {
-                    const int32_t* cb = p.chunk_base + (size_t)ch * p.B;
-                    finalize_chunk(p, t0, t1, ids, loc_e, loc_r,
-                                   [&](int e) { return __ldcg(p.expert_offset + e) + __ldcg(cb + e); },
-                                   [&](int r) { return __ldcg(cb + p.E + r); }, true, pos, arr, gtid, gn);
-                    group_sync(1, gn);
-                    if (gtid == 0) trace(p, c, kTrFinalized);
-                    order_destinations(p, c, order_sm, pos, ntok, gtid, gn);
-                    group_sync(1, gn);
-                }
-                if (gtid == 0) {
-                    mbar_arrive(&ready_bar);
-                    trace(p, c, kTrReady);
-                }
-                if (ok && deferred >= 0) scan_rank_sources(p, deferred, hist, gtid, gn);
-            } else {
-                // phased: counts and prefix sums were separate launches; local counts are in
-                // slot_aux (expert) / slot_row (rank)
-                loc_e = p.slot_aux + (size_t)t0 * p.k;
-                loc_r = p.slot_row + (size_t)t0 * p.k;
+            }
+            if (ok) {
+                // rows before a token = rows of earlier chunks (+ the expert's offset in its
+                // region), published by the prefix-sum step, + earlier tokens of this chunk
                 const int32_t* cb = p.chunk_base + (size_t)ch * p.B;
-                finalize_chunk(p, t0, t1, ids, loc_e, loc_r,
-                               [&](int e) { return __ldcg(p.expert_offset + e) + __ldcg(cb + e); },
-                               [&](int r) { return __ldcg(cb + p.E + r); }, true, pos, arr, gtid, gn);
+                finalize_chunk(p, t0, t1, ids, w_sm,
+                               [&](int e, int tl) {
+                                   return __ldcg(p.expert_offset + e) + __ldcg(cb + e) + bits_in_range(bmaps, e, 0, tl);
+                               },
+                               [&](int r, int tl) {
+                                   return __ldcg(cb + p.E + r) + bits_in_range(bmaps, p.E + r, 0, tl);
+                               },
+                               true, pos_raw, key, arr, gtid, gn);
                 group_sync(1, gn);
                 if (gtid == 0) trace(p, c, kTrFinalized);
-                order_destinations(p, c, order_sm, pos, ntok, gtid, gn);
+                order_destinations(p, c, order_sm, pos_raw, key, pos, ntok * p.k, gtid, gn);
                 group_sync(1, gn);
-                if (gtid == 0) {
-                    mbar_arrive(&ready_bar);
-                    trace(p, c, kTrReady);
-                }
             }
+            if (gtid == 0) {
+                mbar_arrive(&ready_bar);
+                trace(p, c, kTrReady);
+            }
+            if (ok && deferred >= 0) scan_rank_sources(p, deferred, hist, gtid, gn);
         }
         if (kFp8 && ok) {
             uint8_t* out_ring = smem + pl.off_out;
@@ -552,11 +567,19 @@ int plan_dispatch(const Params& p, int mode, int max_smem, SmemPlan* out) {
     SmemPlan pl{};
     const int chunk_tokens = (p.T + p.nchunks - 1) / p.nchunks;
     const int chunk_slots = chunk_tokens * p.k;
-    const int64_t ids_ints = mode == kModeLocal ? (int64_t)p.T * p.k : chunk_slots;
-    const int hist_ints = mode == kModeLocal ? 5 * p.B + p.E : p.B;
+    const int map_tokens = mode == kModeLocal ? p.T : chunk_tokens;   // tokens the bitmaps cover
+    const int64_t ids_ints = (int64_t)map_tokens * p.k;
+    int hist_ints = mode == kModeLocal ? 2 * p.B + p.E : p.B;
+    if (hist_ints < 64) hist_ints = 64;   // the per-rank duty of the flag-free kernel keeps 2 x 32 ints here
+    pl.map_groups = (map_tokens + 31) / 32;
+    pl.map_wb = (p.B + 31) / 32;
+    pl.map_wbs = pl.map_wb | 1;
+    pl.map_bp = pl.map_wb * 32;
     pl.stage_bytes = round_up_i(p.H * 2 / p.parts, 128);
     pl.out_stage_bytes = p.payload ? round_up_i(p.rowB / p.parts, 128) : 0;
-    const int64_t ints = ids_ints + 3 * (int64_t)chunk_slots + hist_ints + 2 * p.R;
+    const int64_t mask_ints = (int64_t)pl.map_groups * 32 * pl.map_wbs;
+    const int64_t bm_ints = (int64_t)pl.map_groups * pl.map_bp;
+    const int64_t ints = ids_ints + mask_ints + bm_ints + 4 * (int64_t)chunk_slots + hist_ints + 2 * p.R;
     const int64_t fixed = (int64_t)kOutStages * pl.out_stage_bytes + ints * 4 + 128 + 1024;  // 1 KB: static smem
     if (fixed + 4 * (int64_t)pl.stage_bytes > max_smem) return -1;
     pl.stages = (int)((max_smem - fixed) / pl.stage_bytes);
@@ -564,9 +587,12 @@ int plan_dispatch(const Params& p, int mode, int max_smem, SmemPlan* out) {
     int at = pl.stages * pl.stage_bytes;
     pl.off_out = at; at += kOutStages * pl.out_stage_bytes;
     pl.off_ids = at; at += (int)ids_ints * 4;
-    pl.off_loc_e = at; at += chunk_slots * 4;
-    pl.off_loc_r = at; at += chunk_slots * 4;
+    pl.off_mask = at; at += (int)mask_ints * 4;
+    pl.off_bm = at; at += (int)bm_ints * 4;
     pl.off_pos = at; at += chunk_slots * 4;
+    pl.off_key = at; at += chunk_slots * 4;
+    pl.off_ord = at; at += chunk_slots * 4;
+    pl.off_w = at; at += chunk_slots * 4;
     pl.off_hist = at; at += hist_ints * 4;
     pl.off_arr = at; at += p.R * 4;
     pl.off_order = at; at += p.R * 4;
@@ -588,8 +614,11 @@ cudaError_t launch_dispatch(const Params& p, int mode, const SmemPlan& pl, cudaS
     cudaError_t e;
     *launches = 1;
     if (mode == kModePhased) {
-        const int chunk_slots = ((p.T + p.nchunks - 1) / p.nchunks) * p.k;
-        count_kernel<<<p.nchunks, 32, sizeof(int) * (p.B + chunk_slots), st>>>(p);
+        const int count_smem = pl.off_pos - pl.off_ids;   // ids + both bitmap arrays
+        if ((e = cudaFuncSetAttribute(count_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, count_smem)) !=
+            cudaSuccess)
+            return e;
+        count_kernel<<<p.nchunks, 256, count_smem, st>>>(p, pl);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
         scan_kernel<<<p.R, 256, sizeof(int) * (p.L + 1), st>>>(p);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;

@@ -1,6 +1,6 @@
-// Layout steps of dispatch as device functions: TokenCnt (stage_ids + count_slots),
-// CalCumSum (scan_rank, or local_layout when every CTA derives it from the whole routing
-// table) and slot -> row assignment (finalize_chunk).  They are shared by the three-launch
+// Layout steps of dispatch as device functions: TokenCnt (stage_ids + build_bin_maps),
+// CalCumSum (scan_rank_*, or bit counts over the whole routing table when every CTA derives
+// it alone) and slot -> row assignment (finalize_chunk).  They are shared by the three-launch
 // pipeline, where kernel boundaries order them, and by the persistent kernel, where
 // readiness flags do (Sec. 3.2 of the paper: kernel decomposition).
 #pragma once
@@ -38,80 +38,171 @@ __device__ __forceinline__ int warp_incl_scan(int v, int lane) {
     return v;
 }
 
-// Resolved expert ids of tokens [t0, t1) into shared memory, one coalesced pass.
+// Staged slot: physical expert id in the low 16 bits, its rank above; -1 = empty slot.
+__device__ __forceinline__ int slot_expert(int v) { return v & 0xffff; }
+__device__ __forceinline__ int slot_rank(int v) { return v >> 16; }
+
+// Resolved expert ids (with their ranks) of tokens [t0, t1) into shared memory.  The raw ids
+// are gathered eight at a time before any of them is resolved, so that the loads overlap.
 __device__ __forceinline__ void stage_ids(const Params& p, int t0, int t1, int* ids, int tid, int nthreads) {
     const int k = p.k, n = (t1 - t0) * k;
     const int32_t* src = p.topk_idx + (size_t)t0 * k;
-    for (int i = tid; i < n; i += nthreads) ids[i] = resolve_expert(p, t0 + i / k, __ldg(src + i));
+    if ((((size_t)t0 * k) & 3) == 0 && (n & 3) == 0) {
+        // 16-byte loads, four of them in flight per thread
+        const int4* src4 = reinterpret_cast<const int4*>(src);
+        const int n4 = n >> 2;
+        for (int i0 = tid; i0 < n4; i0 += 4 * nthreads) {
+            int4 raw[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int i = i0 + u * nthreads;
+                raw[u] = i < n4 ? __ldg(src4 + i) : make_int4(-1, -1, -1, -1);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int i = i0 + u * nthreads;
+                if (i < n4) {
+                    const int r4[4] = {raw[u].x, raw[u].y, raw[u].z, raw[u].w};
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int e = resolve_expert(p, t0 + (4 * i + q) / k, r4[q]);
+                        ids[4 * i + q] = e < 0 ? -1 : (e | ((e / p.L) << 16));
+                    }
+                }
+            }
+        }
+        return;
+    }
+    for (int i0 = tid; i0 < n; i0 += 8 * nthreads) {
+        int raw[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int i = i0 + u * nthreads;
+            raw[u] = i < n ? __ldg(src + i) : -1;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int i = i0 + u * nthreads;
+            if (i < n) {
+                const int e = resolve_expert(p, t0 + i / k, raw[u]);
+                ids[i] = e < 0 ? -1 : (e | ((e / p.L) << 16));
+            }
+        }
+    }
 }
 
 // ------------------------------------------------------------------- TokenCnt
-// One warp walks the slots of tokens [t0, t1) in token order (ids staged in shared memory,
-// index 0 = slot (t0, 0)).  For every slot it records how many earlier slots of the range
-// chose the same expert (loc_e) and, for the first slot a token has on a rank, how many
-// earlier tokens of the range visit that rank (loc_r; later slots of the token on that rank
-// copy it).  hist[B] receives the range's histogram.  When `partial` is given, the running
-// histogram is also written out at every source-rank boundary inside the range.  Equal ids
-// inside a batch of 32 slots are ranked with match_any / popc.
-__device__ void count_slots(const Params& p, int t0, int t1, const int* ids, int* hist, int* loc_e, int* loc_r,
-                            int32_t* partial, int lane) {
-    const int T = p.T, k = p.k, B = p.B, S = p.S;
-    for (int b = lane; b < B; b += 32) hist[b] = 0;
-    __syncwarp();
-    const int tpb = 32 / k;  // whole tokens per batch
-    int s_next = partial ? (int)(((int64_t)t0 * S + T - 1) / T) : S;  // smallest s with src_begin(s) >= t0
-    const unsigned lt = (1u << lane) - 1u;
-    const int tok = lane / k, j = lane - tok * k;
-    const int base_lane = lane - j;
-    int t = t0;
-    while (true) {
-        while (t < t1 && s_next < S && src_begin(s_next, T, S) == t) {
-            for (int b = lane; b < B; b += 32) partial[(size_t)s_next * B + b] = hist[b];
-            ++s_next;
-        }
-        if (t >= t1) break;
-        int lim = t1;
-        if (s_next < S) lim = min(lim, src_begin(s_next, T, S));
-        const int nb = min(tpb, lim - t);
-        const bool active = lane < nb * k;
-        const int li = (t - t0 + tok) * k + j;
-        const int e = active ? ids[li] : -1;
-        const int r = e >= 0 ? e / p.L : -1;
-        // is this the first slot of its token on rank r?
-        bool first = e >= 0;
-        int jf = j;
-        for (int jj = 0; jj < k; ++jj) {
-            int rr = __shfl_sync(0xffffffffu, r, min(base_lane + jj, 31));
-            if (jj < j && first && rr == r) { first = false; jf = jj; }
-        }
-        // expert bins
-        unsigned m = __match_any_sync(0xffffffffu, e >= 0 ? (unsigned)e : (0x40000000u | lane));
-        int le = -1;
-        if (e >= 0) le = hist[e] + __popc(m & lt);
-        __syncwarp();
-        if (e >= 0 && (m & lt) == 0) hist[e] += __popc(m);
-        // rank bins, first slots only
-        unsigned m2 = __match_any_sync(0xffffffffu, first ? (unsigned)r : (0x40000000u | lane));
-        int lr = -1;
-        if (first) lr = hist[p.E + r] + __popc(m2 & lt);
-        __syncwarp();
-        if (first && (m2 & lt) == 0) hist[p.E + r] += __popc(m2);
-        __syncwarp();
-        int lr_first = __shfl_sync(0xffffffffu, lr, min(base_lane + jf, 31));
-        if (e >= 0 && !first) lr = lr_first;
-        if (active) {
-            loc_e[li] = le;
-            loc_r[li] = first ? lr : (e >= 0 ? -2 - lr : -1);  // later slots on a rank: -2 - row
-        }
-        t += nb;
+// Counting without ordered atomics: for a range of tokens, every bin (E expert bins then R
+// rank bins) gets a bitmap with one bit per token of the range.  A token selects an expert
+// at most once, so "how many earlier tokens of the range chose this bin" -- the stable rank
+// the row placement needs -- is a population count of the bits below the token, and the
+// range's histogram is the population count of all bits.
+//
+// Built per group of 32 tokens: each lane ORs the bins of its own token into a private row
+// of words (mask_t), then the warp transposes each 32x32 bit tile (lane = token, bit = bin
+// -> lane = bin, bit = token) with five shuffle steps and stores it bin-major (bm).
+struct BinMaps {
+    unsigned* mask_t;  // [groups * 32, wbs] token-major scratch rows
+    unsigned* bm;      // [groups, bp] bit (token & 31) of word [token >> 5][bin]
+    int wb;            // words per token row that carry bins: ceil(B / 32)
+    int wbs;           // row stride in words (odd, keeps the rows bank-conflict free)
+    int bp;            // bins padded to a multiple of 32
+    int groups;        // 32-token groups of the range
+};
+
+__device__ __forceinline__ unsigned transpose32(unsigned x, int lane) {
+    unsigned m = 0x0000ffffu;
+#pragma unroll
+    for (int j = 16; j != 0; j >>= 1) {
+        const unsigned y = __shfl_xor_sync(0xffffffffu, x, j);
+        if ((lane & j) == 0) x ^= ((((x >> j) ^ y) & m) << j);
+        else x ^= (((y >> j) ^ x) & m);
+        m ^= m << (j >> 1);
     }
-    __syncwarp();
+    return x;  // bit b of lane i before == bit i of lane b after
 }
 
-// loc_r encoding: >= 0 first slot of its token on that rank (value = local row count);
-// <= -2 a later slot sharing the row -2 - value; -1 empty slot.
-__device__ __forceinline__ bool locr_first(int v) { return v >= 0; }
-__device__ __forceinline__ int locr_value(int v) { return v >= 0 ? v : -2 - v; }
+// ids: staged slots of the range (index 0 = first token's slot 0); run by nw warps.
+constexpr int kRegWords = 12;  // up to 384 bins are masked in registers
+__device__ void build_bin_maps(const Params& p, const int* ids, int ntok, const BinMaps& bmaps, int gw, int nw,
+                               int lane) {
+    const int k = p.k;
+    if (bmaps.wb <= kRegWords) {
+        for (int g = gw; g < bmaps.groups; g += nw) {
+            const int tl = g * 32 + lane;
+            unsigned m[kRegWords];
+#pragma unroll
+            for (int w = 0; w < kRegWords; ++w) m[w] = 0u;
+            if (tl < ntok) {
+                for (int j = 0; j < k; ++j) {
+                    const int v = ids[tl * k + j];
+                    if (v < 0) continue;
+                    const int e = slot_expert(v), rb = p.E + slot_rank(v);
+                    const unsigned be = 1u << (e & 31), br = 1u << (rb & 31);
+                    const int we = e >> 5, wr = rb >> 5;
+#pragma unroll
+                    for (int w = 0; w < kRegWords; ++w) m[w] |= (w == we ? be : 0u) | (w == wr ? br : 0u);
+                }
+            }
+#pragma unroll
+            for (int w = 0; w < kRegWords; ++w)
+                if (w < bmaps.wb) bmaps.bm[(size_t)g * bmaps.bp + w * 32 + lane] = transpose32(m[w], lane);
+        }
+        return;
+    }
+    for (int g = gw; g < bmaps.groups; g += nw) {
+        const int tl = g * 32 + lane;
+        unsigned* row = bmaps.mask_t + (size_t)tl * bmaps.wbs;
+        for (int w = 0; w < bmaps.wb; ++w) row[w] = 0u;
+        if (tl < ntok) {
+            for (int j = 0; j < k; ++j) {
+                const int v = ids[tl * k + j];
+                if (v < 0) continue;
+                const int e = slot_expert(v), rb = p.E + slot_rank(v);
+                row[e >> 5] |= 1u << (e & 31);
+                row[rb >> 5] |= 1u << (rb & 31);
+            }
+        }
+        for (int w = 0; w < bmaps.wb; ++w)
+            bmaps.bm[(size_t)g * bmaps.bp + w * 32 + lane] = transpose32(row[w], lane);
+    }
+}
+
+// Tokens with local index in [lo, hi) that selected `bin`.
+__device__ __forceinline__ int bits_in_range(const BinMaps& bmaps, int bin, int lo, int hi) {
+    if (hi <= lo) return 0;
+    const int g0 = lo >> 5, g1 = (hi - 1) >> 5;
+    int c = 0;
+    for (int g = g0; g <= g1; ++g) {
+        unsigned w = bmaps.bm[(size_t)g * bmaps.bp + bin];
+        if (g == g0) w &= 0xffffffffu << (lo & 31);
+        if (g == g1 && (hi & 31) != 0) w &= (1u << (hi & 31)) - 1u;
+        c += __popc(w);
+    }
+    return c;
+}
+
+// Chunk histogram and its running value at the source-rank boundaries inside the chunk
+// (tokens [t0, t1), bitmaps over the chunk), written to chunk_hist[ch] and partial[s].
+__device__ void publish_chunk_counts(const Params& p, int ch, int t0, int t1, const BinMaps& bmaps, int gtid,
+                                     int gn) {
+    const int T = p.T, S = p.S, B = p.B;
+    const int s_lo = (int)(((int64_t)t0 * S + T - 1) / T);  // smallest s with src_begin(s) >= t0
+    int nbnd = 0, bnd[4];                                    // boundaries inside the chunk (first four cached)
+    for (int s = s_lo; s < S; ++s) {
+        const int bs = src_begin(s, T, S);
+        if (bs >= t1) break;
+        if (nbnd < 4) bnd[nbnd] = bs;
+        ++nbnd;
+    }
+    for (int b = gtid; b < B; b += gn) {
+        p.chunk_hist[(size_t)ch * B + b] = bits_in_range(bmaps, b, 0, t1 - t0);
+        for (int q = 0; q < nbnd; ++q) {
+            const int bs = q < 4 ? bnd[q] : src_begin(s_lo + q, T, S);
+            p.partial[(size_t)(s_lo + q) * B + b] = bits_in_range(bmaps, b, 0, bs - t0);
+        }
+    }
+}
 
 // ------------------------------------------------------------------ CalCumSum
 // Prefix sums for the bins of rank r (its L experts and its rank bin), run by a group of
@@ -125,13 +216,21 @@ __device__ void scan_rank_publish(const Params& p, int r, int* sm, int gw, int n
     const int nb = L + 1;
     for (int bi = gw; bi < nb; bi += nw) {
         const int bin = bi < L ? r * L + bi : E + r;
+        int v[kMaxChunks / 32];
+#pragma unroll
+        for (int i = 0; i < kMaxChunks / 32; ++i) {   // all loads first: one round trip to L2
+            const int c = i * 32 + lane;
+            v[i] = c < n ? __ldcg(p.chunk_hist + (size_t)c * B + bin) : 0;
+        }
         int carry = 0;
-        for (int c0 = 0; c0 < n; c0 += 32) {
-            const int c = c0 + lane;
-            const int v = c < n ? __ldcg(p.chunk_hist + (size_t)c * B + bin) : 0;
-            const int incl = warp_incl_scan(v, lane);
-            if (c < n) p.chunk_base[(size_t)c * B + bin] = carry + incl - v;
-            carry += __shfl_sync(0xffffffffu, incl, 31);
+#pragma unroll
+        for (int i = 0; i < kMaxChunks / 32; ++i) {
+            const int c = i * 32 + lane;
+            if (i * 32 < n) {
+                const int incl = warp_incl_scan(v[i], lane);
+                if (c < n) p.chunk_base[(size_t)c * B + bin] = carry + incl - v[i];
+                carry += __shfl_sync(0xffffffffu, incl, 31);
+            }
         }
         if (lane == 0) sm[bi] = carry;
     }
@@ -177,67 +276,38 @@ __device__ void scan_rank_sources(const Params& p, int r, const int* sm, int gti
     }
 }
 
-// ------------------------------------------------ CalCumSum without communication
-// Every CTA histograms the whole routing table (ids of all T tokens staged in shared
-// memory): tot[B] over all tokens, pre[B] over tokens before t0.  CTA `duty_s` (< S) also
-// gets the per-source numbers of source rank duty_s: spre (tokens before its first token)
-// and scnt (its own tokens), expert bins only.  Run by gn threads between barriers.
-__device__ void local_histograms(const Params& p, const int* ids, int t0, int duty_s, int* tot, int* pre, int* spre,
-                                 int* scnt, int gtid, int gn) {
-    const int k = p.k, L = p.L, E = p.E, T = p.T;
-    const int b0 = duty_s >= 0 ? src_begin(duty_s, T, p.S) : 0;
-    const int b1 = duty_s >= 0 ? src_begin(duty_s + 1, T, p.S) : 0;
-    for (int t = gtid; t < T; t += gn) {
-        const int* row = ids + (size_t)t * k;
-        const bool before = t < t0;
-        for (int j = 0; j < k; ++j) {
-            const int e = row[j];
-            if (e < 0) continue;
-            const int r = e / L;
-            bool first = true;
-            for (int jj = 0; jj < j; ++jj) {
-                const int e2 = row[jj];
-                if (e2 >= 0 && e2 / L == r) { first = false; break; }
-            }
-            atomicAdd(&tot[e], 1);
-            if (before) atomicAdd(&pre[e], 1);
-            if (first) {
-                atomicAdd(&tot[E + r], 1);
-                if (before) atomicAdd(&pre[E + r], 1);
-            }
-            if (duty_s >= 0) {
-                if (t < b0) atomicAdd(&spre[e], 1);
-                else if (t < b1) atomicAdd(&scnt[e], 1);
-            }
-        }
-    }
-}
-
 // -------------------------------------------------------- slot -> row assignment
-// Turns the range-local counts of this CTA's tokens [t0, t1) into final rows.  base_e(e) /
-// base_r(r) give the rows taken by earlier tokens (plus the expert's offset in its region).
-// Writes slot_row / slot_pos, the per-row metadata (only when `write_meta`; with column
-// parts one CTA of the group does it) and leaves in pos[] the global row to copy to
-// (rank * cap + row), or -1.  arr[r] counts the rows this CTA sends to rank r.
-template <typename BaseE, typename BaseR>
-__device__ void finalize_chunk(const Params& p, int t0, int t1, const int* ids, const int* loc_e, const int* loc_r,
-                               BaseE base_e, BaseR base_r, bool write_meta, int* pos, int* arr, int gtid, int gn) {
+// Final rows of this CTA's tokens [t0, t1).  rows_e(e, tl) / rows_r(r, tl) return how many
+// rows precede local token tl in expert e's segment (offset of the segment included) / in
+// rank r's region.  Writes slot_row / slot_pos and the per-row metadata (only when
+// `write_meta`; with column parts one CTA of the group does it) and leaves in pos[] the
+// global row to copy to (rank * cap + row), or -1, and in dst_rank[] that row's rank.
+// arr[r] counts the rows this CTA sends to rank r.  w_sm: the tokens' gate weights, staged.
+template <typename RowsE, typename RowsR>
+__device__ void finalize_chunk(const Params& p, int t0, int t1, const int* ids, const float* w_sm, RowsE rows_e,
+                               RowsR rows_r, bool write_meta, int* pos, int* dst_rank, int* arr, int gtid, int gn) {
     const int k = p.k, L = p.L;
     const int nslots = (t1 - t0) * k;
     for (int li = gtid; li < nslots; li += gn) {
-        const int t = t0 + li / k;
+        const int tl = li / k, j = li - tl * k;
+        const int t = t0 + tl;
         const size_t i = (size_t)t0 * k + li;
-        const int e = ids[li];
-        int where = -1, row = -1, gpos = -1;
-        if (e >= 0) {
-            const int r = e / L;
-            const bool first = !p.dedup || locr_first(loc_r[li]);
+        const int packed = ids[li];
+        int where = -1, row = -1, gpos = -1, r = 0;
+        if (packed >= 0) {
+            const int e = slot_expert(packed);
+            r = slot_rank(packed);
+            bool first = true;
             if (!p.dedup) {
-                row = base_e(e) + loc_e[li];
+                row = rows_e(e, tl);
             } else {
-                row = base_r(r) + locr_value(loc_r[li]);
+                for (int jj = 0; jj < j; ++jj) {
+                    const int v2 = ids[li - j + jj];
+                    if (v2 >= 0 && slot_rank(v2) == r) { first = false; break; }
+                }
+                row = rows_r(r, tl);
                 if (write_meta) {
-                    const int at = base_e(e) + loc_e[li];
+                    const int at = rows_e(e, tl);
                     if (at < p.er_cap) p.expert_rows[(size_t)r * p.er_cap + at] = row;
                     else report(p.status, kErrCapacity);
                 }
@@ -252,15 +322,15 @@ __device__ void finalize_chunk(const Params& p, int t0, int t1, const int* ids, 
                     if (write_meta) {
                         p.recv_src_idx[where] = t;
                         if (!p.dedup) {
-                            p.recv_weight[where] = __ldg(p.topk_w + i);
+                            p.recv_weight[where] = w_sm[li];
                         } else {
-                            const int* row_ids = ids + (li / k) * k;
+                            const int* row_ids = ids + tl * k;
                             for (int jj = 0; jj < k; ++jj) {
-                                const int e2 = row_ids[jj];
-                                const bool here = e2 >= 0 && e2 / L == r;
-                                p.recv_topk_idx[(size_t)where * k + jj] = here ? e2 % L : -1;
+                                const int v2 = row_ids[jj];
+                                const bool here = v2 >= 0 && slot_rank(v2) == r;
+                                p.recv_topk_idx[(size_t)where * k + jj] = here ? slot_expert(v2) - r * L : -1;
                                 p.recv_topk_w[(size_t)where * k + jj] =
-                                    here ? __ldg(p.topk_w + (size_t)t * k + jj) : 0.0f;
+                                    here ? w_sm[tl * k + jj] : 0.0f;
                             }
                         }
                     }
@@ -272,37 +342,216 @@ __device__ void finalize_chunk(const Params& p, int t0, int t1, const int* ids, 
             p.slot_pos[i] = gpos;
         }
         pos[li] = where;
+        dst_rank[li] = r;
     }
+}
+
+// --------------------------------------------- flag-free layout, dedup fast path
+// With one row per (token, rank) the movers only need rank-level rows: row of token t in
+// region r = number of earlier tokens that visit r.  One 32-bit word per token and 32 ranks
+// says which ranks it visits; transposed per group of 32 tokens it becomes, per rank, a
+// bitmap over tokens, and the row is a population count.  Everything expert-level (offsets,
+// counts per source, the per-expert row lists) is produced after the movers are released,
+// each rank's share by one CTA.
+struct RankMaps {
+    unsigned* rbm;  // [groups, rp] rank bitmaps over all T tokens
+    unsigned* dbm;  // [groups, 32] duty bitmaps: bit l < L = local expert l, bit L = the rank itself
+    int wr;         // words of ranks per token: ceil(R / 32), at most kRankWords
+    int rp;         // wr * 32
+    int groups;     // ceil(T / 32)
+};
+constexpr int kRankWords = 4;
+
+__device__ __forceinline__ int fast_div(int v, unsigned magic) { return (int)__umulhi((unsigned)v, magic); }
+
+// Stage all T*k slots (packed id | rank << 16) and build the rank bitmaps; lane = token.
+__device__ void local_stage_and_rank_maps(const Params& p, int* ids, const RankMaps& rm, int gw, int nw, int lane) {
+    const int k = p.k, T = p.T;
+    for (int g = gw; g < rm.groups; g += nw) {
+        const int t = g * 32 + lane;
+        unsigned m[kRankWords];
+#pragma unroll
+        for (int w = 0; w < kRankWords; ++w) m[w] = 0u;
+        if (t < T) {
+            const int32_t* src = p.topk_idx + (size_t)t * k;
+            for (int j0 = 0; j0 < k; j0 += 8) {       // up to eight ids in flight
+                int raw[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) raw[u] = j0 + u < k ? __ldg(src + j0 + u) : -1;
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    if (j0 + u >= k) break;
+                    const int e = resolve_expert(p, t, raw[u]);
+                    int packed = -1;
+                    if (e >= 0) {
+                        const int r = fast_div(e, p.L_magic);
+                        packed = e | (r << 16);
+#pragma unroll
+                        for (int w = 0; w < kRankWords; ++w) m[w] |= (w == (r >> 5)) ? 1u << (r & 31) : 0u;
+                    }
+                    ids[t * k + j0 + u] = packed;
+                }
+            }
+        }
+#pragma unroll
+        for (int w = 0; w < kRankWords; ++w)
+            if (w < rm.wr) rm.rbm[(size_t)g * rm.rp + w * 32 + lane] = transpose32(m[w], lane);
+    }
+}
+
+// Tokens below t that visit rank r.
+__device__ __forceinline__ int rank_rows_before(const RankMaps& rm, int r, int t) {
+    int c = 0;
+    const int g1 = t >> 5;
+    for (int g = 0; g < g1; ++g) c += __popc(rm.rbm[(size_t)g * rm.rp + r]);
+    if (t & 31) c += __popc(rm.rbm[(size_t)g1 * rm.rp + r] & ((1u << (t & 31)) - 1u));
+    return c;
+}
+
+// Destinations of this CTA's tokens [t0, t1): pos_raw (slot order), dst_rank, row_sm, arr.
+__device__ void local_rows_dedup(const Params& p, int t0, int t1, const int* ids_all, const RankMaps& rm,
+                                 int* pos_raw, int* dst_rank, int* row_sm, int* arr, int gtid, int gn) {
+    const int k = p.k;
+    const int nslots = (t1 - t0) * k;
+    for (int li = gtid; li < nslots; li += gn) {
+        const int tl = li / k, j = li - tl * k, t = t0 + tl;
+        const int packed = ids_all[(size_t)t * k + j];
+        int where = -1, row = -1, r = 0;
+        if (packed >= 0) {
+            r = slot_rank(packed);
+            bool first = true;
+            for (int jj = 0; jj < j; ++jj) {
+                const int v2 = ids_all[(size_t)t * k + jj];
+                if (v2 >= 0 && slot_rank(v2) == r) { first = false; break; }
+            }
+            row = rank_rows_before(rm, r, t);
+            if (row >= p.cap) {
+                report(p.status, kErrCapacity);
+            } else if (first) {
+                where = r * p.cap + row;
+                atomicAdd(&arr[r], 1);
+            }
+        }
+        pos_raw[li] = where;
+        dst_rank[li] = r;
+        row_sm[li] = row;
+    }
+}
+
+// Metadata of this CTA's own tokens (after the movers were released).
+__device__ void local_meta_dedup(const Params& p, int t0, int t1, const int* ids_all, const int* pos_raw,
+                                 const int* row_sm, int gtid, int gn) {
+    const int k = p.k, L = p.L;
+    const int nslots = (t1 - t0) * k;
+    for (int li = gtid; li < nslots; li += gn) {
+        const int tl = li / k, t = t0 + tl;
+        const size_t i = (size_t)t0 * k + li;
+        const int packed = ids_all[i];
+        const int row = row_sm[li];
+        p.slot_row[i] = row;
+        p.slot_pos[i] = (packed >= 0 && row >= 0 && row < p.cap) ? slot_rank(packed) * p.cap + row : -1;
+        const int where = pos_raw[li];
+        if (where >= 0) {
+            const int r = slot_rank(packed);
+            p.recv_src_idx[where] = t;
+            for (int jj = 0; jj < k; ++jj) {
+                const int v2 = ids_all[(size_t)t * k + jj];
+                const bool here = v2 >= 0 && slot_rank(v2) == r;
+                p.recv_topk_idx[(size_t)where * k + jj] = here ? slot_expert(v2) - r * L : -1;
+                p.recv_topk_w[(size_t)where * k + jj] = here ? __ldg(p.topk_w + (size_t)t * k + jj) : 0.0f;
+            }
+        }
+    }
+}
+
+// Everything about rank r that nobody inside the kernel waits for: expert totals and
+// offsets, tokens per rank, counts and offsets per source rank, the per-expert row lists.
+// Needs L < 32.  `sm` holds 2 * 32 ints.  Run by the whole layout group (barrier bar_id).
+__device__ void local_rank_duty(const Params& p, int r, const int* ids_all, const RankMaps& rm, int* sm, int gw,
+                                int nw, int lane, int gtid, int gn, int bar_id) {
+    const int k = p.k, L = p.L, T = p.T, S = p.S, E = p.E;
+    for (int g = gw; g < rm.groups; g += nw) {
+        const int t = g * 32 + lane;
+        unsigned m = 0u;
+        if (t < T)
+            for (int j = 0; j < k; ++j) {
+                const int v = ids_all[(size_t)t * k + j];
+                if (v >= 0 && slot_rank(v) == r) m |= (1u << (slot_expert(v) - r * L)) | (1u << L);
+            }
+        rm.dbm[(size_t)g * 32 + lane] = transpose32(m, lane);
+    }
+    group_sync(bar_id, gn);
+    auto bits = [&](int l, int lo, int hi) {   // tokens in [lo, hi) with bit l
+        if (hi <= lo) return 0;
+        const int g0 = lo >> 5, g1 = (hi - 1) >> 5;
+        int c = 0;
+        for (int g = g0; g <= g1; ++g) {
+            unsigned w = rm.dbm[(size_t)g * 32 + l];
+            if (g == g0) w &= 0xffffffffu << (lo & 31);
+            if (g == g1 && (hi & 31) != 0) w &= (1u << (hi & 31)) - 1u;
+            c += __popc(w);
+        }
+        return c;
+    };
+    int* tot = sm;
+    int* eo = sm + 32;
+    if (gtid <= L) tot[gtid] = bits(gtid, 0, T);
+    group_sync(bar_id, gn);
+    if (gtid <= L) {
+        int o = 0;
+        for (int q = 0; q < gtid; ++q) o += tot[q];
+        eo[gtid] = o;
+        if (gtid < L) {
+            p.expert_offset[r * L + gtid] = o;
+            p.num_tokens_per_expert[r * L + gtid] = tot[gtid];
+        } else {
+            p.num_tokens_per_rank[r] = tot[L];
+            p.num_rows_per_rank[r] = tot[L];
+        }
+    }
+    group_sync(bar_id, gn);
+    for (int i = gtid; i < S * L; i += gn) {
+        const int s = i / L, l = i - s * L;
+        const int b0 = src_begin(s, T, S), b1 = src_begin(s + 1, T, S);
+        p.cnt[(size_t)s * E + r * L + l] = bits(l, b0, b1);
+        p.src_offset[(size_t)s * E + r * L + l] = eo[l] + bits(l, 0, b0);
+    }
+    for (int i = gtid; i < T * k; i += gn) {
+        const int v = ids_all[i];
+        if (v < 0 || slot_rank(v) != r) continue;
+        const int t = i / k, l = slot_expert(v) - r * L;
+        const int at = eo[l] + bits(l, 0, t);
+        if (at < p.er_cap) p.expert_rows[(size_t)r * p.er_cap + at] = bits(L, 0, t);
+        else report(p.status, kErrCapacity);
+    }
+    group_sync(bar_id, gn);   // sm and dbm are reused by the next rank
 }
 
 // Per token, put the destinations into the order of the destination-ordering table rotated
 // by the worker id (Sec. 3.3: each worker visits a re-mapped destination sequence).  Only
-// the issue order of the copies changes.  order_sm[R] is the table in shared memory.  One
-// thread per token, insertion sort on <= 32 keys.
-__device__ void order_destinations(const Params& p, int worker, const int* order_sm, int* pos, int ntok, int gtid,
-                                   int gn) {
+// the issue order of the copies changes.  One thread per slot: its place is the number of
+// the token's destinations that come earlier in the rotated table (ties keep slot order);
+// empty slots go last.  Reads pos / dst_rank, writes pos_out.
+__device__ void order_destinations(const Params& p, int worker, const int* order_sm, const int* pos,
+                                   const int* dst_rank, int* pos_out, int nslots, int gtid, int gn) {
     const int k = p.k, R = p.R;
     const int rot = worker % R;
-    for (int n = gtid; n < ntok; n += gn) {
-        int* q = pos + n * k;
-        int m = 0;
-        for (int j = 0; j < k; ++j)
-            if (q[j] >= 0) q[m++] = q[j];
-        for (int j = m; j < k; ++j) q[j] = -1;
-        for (int a = 1; a < m; ++a) {
-            const int v = q[a];
-            int kv = order_sm[v / p.cap] - rot;
-            kv += kv < 0 ? R : 0;
-            int b = a - 1;
-            while (b >= 0) {
-                int kb = order_sm[q[b] / p.cap] - rot;
-                kb += kb < 0 ? R : 0;
-                if (kb <= kv) break;
-                q[b + 1] = q[b];
-                --b;
-            }
-            q[b + 1] = v;
+    for (int li = gtid; li < nslots; li += gn) {
+        const int tl = li / k, j = li - tl * k;
+        const int* q = pos + tl * k;
+        const int* rk = dst_rank + tl * k;
+        const int mine = q[j];
+        int kv = order_sm[rk[j]] - rot;
+        kv += kv < 0 ? R : 0;
+        if (mine < 0) kv = R;   // after every real destination
+        int place = 0;
+        for (int jj = 0; jj < k; ++jj) {
+            int ko = order_sm[rk[jj]] - rot;
+            ko += ko < 0 ? R : 0;
+            if (q[jj] < 0) ko = R;
+            place += (ko < kv || (ko == kv && jj < j)) ? 1 : 0;
         }
+        pos_out[tl * k + place] = mine;
     }
 }
 
