@@ -11,6 +11,7 @@
 //   combine_kernel<K>                 gather + fp32 weighted sum + one bf16 rounding
 //   layout_kernel                     counts only (ubep_get_dispatch_layout)
 #include <cuda_fp8.h>
+#include <cstdlib>
 
 #include "ubep_kernels.h"
 #include "ubep_layout.cuh"
@@ -126,13 +127,7 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
         abort_flag = 0;
         mbar_fence_init();
     }
-    for (int r = tid; r < p.R; r += kThreads) {
-        arr[r] = 0;
-        order_sm[r] = __ldg(p.order_pos + r);
-    }
-    // the arrival counters of the next call live in the other half; clear them now
-    if (c == 0)
-        for (int r = tid; r < p.R; r += kThreads) p.arrival[((epoch + 1) & 1) * p.R + r] = 0;
+    for (int r = tid; r < p.R; r += kThreads) arr[r] = 0;
     __syncthreads();
     if (tid == 0) trace(p, c, kTrStart);
 
@@ -140,42 +135,63 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
     const unsigned out_bytes = (unsigned)(p.rowB / p.parts);   // and of a payload row
     const size_t in_off = (size_t)part * in_bytes, out_off = (size_t)part * out_bytes;
 
+    const bool fast_local = kMode == kModeLocal && p.local_fast;
     if (warp == 0) {
-        // ------------------------------------------------ mover warp (one elected thread)
-        if (lane == 0) {
-            bool ok = true;
-            auto issue_load = [&](int n) {
+        // ------------------------------------------------------------------ mover warp
+        // Lane 0 issues the TMA loads; for bf16 rows lane j issues the TMA store of slot j,
+        // so the k copies of a row are issued side by side.
+        bool ok = true;
+        auto issue_load = [&](int n) {
+            const int s = n % stages;
+            mbar_arrive_expect_tx(&full_bar[s], in_bytes);
+            bulk_load(smem + (size_t)s * pl.stage_bytes,
+                      reinterpret_cast<const uint8_t*>(p.x) + (size_t)(t0 + n) * p.H * 2 + in_off, in_bytes,
+                      &full_bar[s]);
+        };
+        if (!kFp8) {
+            // loads run (stages - 3) rows ahead; up to 3 rows' stores stay in flight
+            const int pf = min(stages - 3, ntok);
+            if (lane == 0)
+                for (int n = 0; n < pf; ++n) issue_load(n);
+            issued = pf;
+            if (fast_local) {
+                // lend a hand with the routing table, then wait for the layout group
+                const RankMaps rm{bmaps.bm, bmaps.mask_t, (p.R + 31) / 32, ((p.R + 31) / 32) * 32, (p.T + 31) / 32};
+                local_stage_and_rank_maps(p, ids_sm, rm, 0, kWarps, lane);
+                group_sync(2, kThreads);
+            }
+            ok = mbar_wait(&ready_bar, 0, abortp) && !*abortp;  // no rows without a layout
+            for (int n = 0; ok && n < ntok; ++n) {
                 const int s = n % stages;
-                mbar_arrive_expect_tx(&full_bar[s], in_bytes);
-                bulk_load(smem + (size_t)s * pl.stage_bytes,
-                          reinterpret_cast<const uint8_t*>(p.x) + (size_t)(t0 + n) * p.H * 2 + in_off, in_bytes,
-                          &full_bar[s]);
-            };
-            if (!kFp8) {
-                // loads run (stages - 3) rows ahead; up to 3 rows' stores stay in flight
-                const int pf = stages - 3;
-                for (; issued < min(pf, ntok); ++issued) issue_load(issued);
-                ok = mbar_wait(&ready_bar, 0, abortp) && !*abortp;  // no rows without a layout
-                for (int n = 0; ok && n < ntok; ++n) {
-                    const int s = n % stages;
-                    ok = mbar_wait(&full_bar[s], (n / stages) & 1, abortp);
-                    if (!ok) break;
-                    if (n == 0) trace(p, c, kTrFirstRow);
-                    const uint8_t* src = smem + (size_t)s * pl.stage_bytes;
-                    for (int j = 0; j < p.k; ++j) {
-                        const int where = pos[n * p.k + j];
-                        if (where >= 0) bulk_store(p.recv_x + (size_t)where * p.rowB + out_off, src, out_bytes);
-                    }
-                    bulk_commit();
-                    if (issued < ntok) {
-                        bulk_wait_read<3>();
-                        issue_load(issued);
-                        ++issued;
-                    }
+                ok = mbar_wait(&full_bar[s], (n / stages) & 1, abortp);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                if (n == 0 && lane == 0) trace(p, c, kTrFirstRow);
+                const uint8_t* src = smem + (size_t)s * pl.stage_bytes;
+                for (int j = lane; j < p.k; j += 32) {
+                    const int where = pos[n * p.k + j];
+                    if (where >= 0) bulk_store(p.recv_x + (size_t)where * p.rowB + out_off, src, out_bytes);
                 }
-            } else {
-                // loader only; the quantising warps free the stages
-                for (int n = 0; ok && n < ntok; ++n) {
+                bulk_commit();
+                if (issued < ntok) {
+                    bulk_wait_read<3>();     // every lane: its copies of the row 3 back have read the stage
+                    __syncwarp();
+                    if (lane == 0) issue_load(issued);
+                    ++issued;
+                }
+            }
+        } else {
+            if (fast_local) {
+                const RankMaps rm{bmaps.bm, bmaps.mask_t, (p.R + 31) / 32, ((p.R + 31) / 32) * 32, (p.T + 31) / 32};
+                if (lane == 0)
+                    for (; issued < min(stages, ntok); ++issued) issue_load(issued);
+                issued = __shfl_sync(0xffffffffu, issued, 0);
+                local_stage_and_rank_maps(p, ids_sm, rm, 0, kWarps, lane);
+                group_sync(2, kThreads);
+            }
+            // loader only (lane 0); the quantising warps free the stages
+            if (lane == 0) {
+                for (int n = issued; ok && n < ntok; ++n) {
                     const int s = n % stages;
                     if (n >= stages) ok = mbar_wait(&empty_bar[s], ((n / stages) - 1) & 1, abortp);
                     if (!ok) break;
@@ -183,26 +199,40 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
                     issued = n + 1;
                 }
             }
-            if (!ok) {
-                report(p.status, kErrTimeout);  // a wait gave up: record it and let everybody leave
-                abort_flag = 1;
-            }
-            trace(p, c, kTrIssued);
-            bulk_wait_all<0>();
-            trace(p, c, kTrStored);
+            issued = __shfl_sync(0xffffffffu, issued, 0);
+            ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
         }
+        if (!ok && lane == 0) {
+            report(p.status, kErrTimeout);  // a wait gave up: record it and let everybody leave
+            abort_flag = 1;
+        }
+        if (lane == 0) trace(p, c, kTrIssued);
+        bulk_wait_all<0>();
+        if (lane == 0) trace(p, c, kTrStored);
     } else {
         // ------------------------------------------------------------- layout group
         bool ok = true;
         const int* ids = ids_sm;  // staged slots of this CTA's tokens
-        if (!(kMode == kModeLocal && p.local_fast))
-            for (int i = gtid; i < ntok * p.k; i += gn) w_sm[i] = __ldg(p.topk_w + (size_t)t0 * p.k + i);
+        // Small global reads whose values are needed only after the first barriers: issue the
+        // loads now (first trip of each loop), store to shared memory after the ids are staged.
+        const int order_r = gtid < p.R ? __ldg(p.order_pos + gtid) : 0;
+        const bool stage_w = !(kMode == kModeLocal && p.local_fast);
+        const float w_first = (stage_w && gtid < ntok * p.k) ? __ldg(p.topk_w + (size_t)t0 * p.k + gtid) : 0.0f;
+        auto stage_small = [&]() {
+            if (gtid < p.R) order_sm[gtid] = order_r;
+            for (int r = gtid + gn; r < p.R; r += gn) order_sm[r] = __ldg(p.order_pos + r);
+            if (stage_w) {
+                if (gtid < ntok * p.k) w_sm[gtid] = w_first;
+                for (int i = gtid + gn; i < ntok * p.k; i += gn) w_sm[i] = __ldg(p.topk_w + (size_t)t0 * p.k + i);
+            }
+        };
         if (kMode == kModeLocal && p.local_fast) {
             // rank-level rows first, movers released, expert-level outputs afterwards
             const RankMaps rm{bmaps.bm, bmaps.mask_t, (p.R + 31) / 32, ((p.R + 31) / 32) * 32, (p.T + 31) / 32};
             int* row_sm = reinterpret_cast<int*>(w_sm);
-            local_stage_and_rank_maps(p, ids_sm, rm, gw, nw, lane);
-            group_sync(1, gn);
+            local_stage_and_rank_maps(p, ids_sm, rm, warp, kWarps, lane);   // with the mover warp
+            stage_small();
+            group_sync(2, kThreads);
             if (gtid == 0) trace(p, c, kTrCounted);
             local_rows_dedup(p, t0, t1, ids_sm, rm, pos_raw, key, row_sm, arr, gtid, gn);
             group_sync(1, gn);
@@ -222,6 +252,7 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
             int* pre = hist + p.B;
             int* eo = hist + 2 * p.B;
             stage_ids(p, 0, p.T, ids_sm, gtid, gn);
+            stage_small();
             group_sync(1, gn);
             if (gtid == 0) trace(p, c, kTrCounted);
             build_bin_maps(p, ids_sm, p.T, bmaps, gw, nw, lane);
@@ -279,6 +310,7 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
                 }
         } else {
             stage_ids(p, t0, t1, ids_sm, gtid, gn);
+            stage_small();
             group_sync(1, gn);
             build_bin_maps(p, ids_sm, ntok, bmaps, gw, nw, lane);
             group_sync(1, gn);
@@ -349,57 +381,88 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
         }
         if (kFp8 && ok) {
             uint8_t* out_ring = smem + pl.off_out;
+            const int g0 = part * (p.G / p.parts);                      // first scale group of this CTA's piece
+            const unsigned scale_bytes = (unsigned)(p.G / p.parts) * 4u;  // its scales travel with the payload
+            const bool scale_bulk = (scale_bytes & 15u) == 0;             // when a bulk copy can carry them
             if (warp == 1) {
-                // ---------------------------------------- store issuer (one elected thread)
-                if (lane == 0) {
-                    bool sok = true;
-                    for (int n = 0; n < ntok; ++n) {
-                        const int os = n % kOutStages;
-                        sok = mbar_wait(&out_full[os], (n / kOutStages) & 1, abortp);
-                        if (!sok) break;
-                        if (n == 0) trace(p, c, kTrFirstRow);
-                        const uint8_t* src = out_ring + (size_t)os * pl.out_stage_bytes;
-                        for (int j = 0; j < p.k; ++j) {
-                            const int where = pos[n * p.k + j];
-                            if (where >= 0) bulk_store(p.recv_x + (size_t)where * p.rowB + out_off, src, out_bytes);
-                        }
-                        bulk_commit();
-                        if (n + 1 >= kOutStages) {
-                            bulk_wait_read<kOutStages - 1>();          // the oldest row's stores have read it
-                            mbar_arrive(&out_empty[(n + 1) % kOutStages]);
-                        }
+                // ------------------------------ store issuer: lane j issues the copy of slot j
+                bool sok = true;
+                unsigned long long w_full = 0, w_read = 0, tq = 0;
+                for (int n = 0; n < ntok; ++n) {
+                    const int os = n % kOutStages;
+                    if (p.trace) tq = global_ns();
+                    sok = mbar_wait(&out_full[os], (n / kOutStages) & 1, abortp);
+                    if (p.trace) w_full += global_ns() - tq;
+                    sok = __all_sync(0xffffffffu, sok);
+                    if (!sok) break;
+                    if (n == 0 && lane == 0) trace(p, c, kTrFirstRow);
+                    const uint8_t* src = out_ring + (size_t)os * pl.out_stage_bytes;
+                    // lanes 0..k-1: payload of slot j; lanes k..2k-1: its scales (when bulk-storable)
+                    for (int j = lane; j < (scale_bulk ? 2 * p.k : p.k); j += 32) {
+                        const int jj = j < p.k ? j : j - p.k;
+                        const int where = pos[n * p.k + jj];
+                        if (where < 0) continue;
+                        if (j < p.k)
+                            bulk_store(p.recv_x + (size_t)where * p.rowB + out_off, src, out_bytes);
+                        else
+                            bulk_store(p.recv_scale + (size_t)where * p.G + g0, src + out_bytes, scale_bytes);
                     }
-                    if (!sok) {
-                        report(p.status, kErrTimeout);
-                        abort_flag = 1;
+                    bulk_commit();
+                    if (n + 1 >= kOutStages) {
+                        if (p.trace) tq = global_ns();
+                        bulk_wait_read<kOutStages - 1>();   // every lane: the oldest row's copies have read it
+                        if (p.trace) w_read += global_ns() - tq;
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&out_empty[(n + 1) % kOutStages]);
                     }
-                    bulk_wait_all<0>();
+                }
+                if (!sok && lane == 0) {
+                    report(p.status, kErrTimeout);
+                    abort_flag = 1;
+                }
+                bulk_wait_all<0>();
+                if (p.trace && lane == 0) {
+                    p.trace[(size_t)c * kTraceSlots + 14] = w_full;
+                    p.trace[(size_t)c * kTraceSlots + 15] = w_read;
                 }
             } else {
                 // ------------------------------------------------- quantising warps 2..15
                 const int qw = warp - 2;
                 const int nvec = (int)in_bytes / 16;          // 8-channel vectors in this CTA's piece
-                const int g0 = part * (p.G / p.parts);        // first scale group of the piece
+                unsigned long long w_in = 0, w_out = 0, t_cmp = 0, tq = 0;
                 for (int n = 0; n < ntok; ++n) {
                     const int s = n % stages, os = n % kOutStages;
+                    if (p.trace) tq = global_ns();
                     if (!mbar_wait(&full_bar[s], (n / stages) & 1, abortp)) break;
+                    if (p.trace) { unsigned long long t2 = global_ns(); w_in += t2 - tq; tq = t2; }
                     if (n >= kOutStages && !mbar_wait(&out_empty[os], ((n / kOutStages) - 1) & 1, abortp)) break;
+                    if (p.trace) { unsigned long long t2 = global_ns(); w_out += t2 - tq; tq = t2; }
                     const uint8_t* src = smem + (size_t)s * pl.stage_bytes;
                     uint8_t* dst = out_ring + (size_t)os * pl.out_stage_bytes;
-                    for (int vb = qw * 32; vb < nvec; vb += nq * 32) {
-                        const int v = vb + lane;
-                        const bool valid = v < nvec;
-                        uint4 in = make_uint4(0, 0, 0, 0);
-                        if (valid) in = *reinterpret_cast<const uint4*>(src + (size_t)v * 16);
-                        uint2 q;
-                        float scale;
-                        quantize8(in, valid, q, scale);
-                        if (valid) {
-                            *reinterpret_cast<uint2*>(dst + (size_t)v * 8) = q;
-                            if ((lane & 15) == 0) {
+                    float* dst_scale = reinterpret_cast<float*>(dst + out_bytes);
+                    // two vectors per thread and trip, independent of each other
+                    for (int vb = qw * 32; vb < nvec; vb += 2 * nq * 32) {
+                        const int v0 = vb + lane, v1 = v0 + nq * 32;
+                        const bool ok0 = v0 < nvec, ok1 = v1 < nvec;
+                        uint4 in0 = make_uint4(0, 0, 0, 0), in1 = make_uint4(0, 0, 0, 0);
+                        if (ok0) in0 = *reinterpret_cast<const uint4*>(src + (size_t)v0 * 16);
+                        if (ok1) in1 = *reinterpret_cast<const uint4*>(src + (size_t)v1 * 16);
+                        uint2 q0, q1;
+                        float sc0, sc1;
+                        quantize8(in0, ok0, q0, sc0);
+                        quantize8(in1, ok1, q1, sc1);
+                        if (ok0) *reinterpret_cast<uint2*>(dst + (size_t)v0 * 8) = q0;
+                        if (ok1) *reinterpret_cast<uint2*>(dst + (size_t)v1 * 8) = q1;
+                        if ((lane & 15) == 0) {
+                            if (scale_bulk) {
+                                if (ok0) dst_scale[v0 >> 4] = sc0;
+                                if (ok1) dst_scale[v1 >> 4] = sc1;
+                            } else {
                                 for (int j = 0; j < p.k; ++j) {
                                     const int where = pos[n * p.k + j];
-                                    if (where >= 0) p.recv_scale[(size_t)where * p.G + g0 + (v >> 4)] = scale;
+                                    if (where < 0) continue;
+                                    if (ok0) p.recv_scale[(size_t)where * p.G + g0 + (v0 >> 4)] = sc0;
+                                    if (ok1) p.recv_scale[(size_t)where * p.G + g0 + (v1 >> 4)] = sc1;
                                 }
                             }
                         }
@@ -410,6 +473,12 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
                         mbar_arrive(&out_full[os]);
                         mbar_arrive(&empty_bar[s]);
                     }
+                    if (p.trace) t_cmp += global_ns() - tq;
+                }
+                if (p.trace && warp == 2 && lane == 0) {
+                    p.trace[(size_t)c * kTraceSlots + 11] = w_in;
+                    p.trace[(size_t)c * kTraceSlots + 12] = w_out;
+                    p.trace[(size_t)c * kTraceSlots + 13] = t_cmp;
                 }
             }
         }
@@ -430,6 +499,9 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
     fence_proxy_async();
     for (int r = tid; r < p.R; r += kThreads)
         if (arr[r]) red_release_add(p.arrival + (epoch & 1) * p.R + r, (unsigned)(arr[r] * (8 / p.parts)));
+    // the arrival counters of the next call live in the other half; clear them now
+    if (c == 0)
+        for (int r = tid; r < p.R; r += kThreads) p.arrival[((epoch + 1) & 1) * p.R + r] = 0;
     __syncthreads();
     if (tid == 0) {
         trace(p, c, kTrEnd);
@@ -576,8 +648,8 @@ int plan_dispatch(const Params& p, int mode, int max_smem, SmemPlan* out) {
     pl.map_wbs = pl.map_wb | 1;
     pl.map_bp = pl.map_wb * 32;
     pl.stage_bytes = round_up_i(p.H * 2 / p.parts, 128);
-    pl.out_stage_bytes = p.payload ? round_up_i(p.rowB / p.parts, 128) : 0;
-    const int64_t mask_ints = (int64_t)pl.map_groups * 32 * pl.map_wbs;
+    pl.out_stage_bytes = p.payload ? round_up_i(p.rowB / p.parts + (p.G / p.parts) * 4, 128) : 0;
+    const int64_t mask_ints = (int64_t)pl.map_groups * 32;
     const int64_t bm_ints = (int64_t)pl.map_groups * pl.map_bp;
     const int64_t ints = ids_ints + mask_ints + bm_ints + 4 * (int64_t)chunk_slots + hist_ints + 2 * p.R;
     const int64_t fixed = (int64_t)kOutStages * pl.out_stage_bytes + ints * 4 + 128 + 1024;  // 1 KB: static smem
@@ -637,7 +709,12 @@ cudaError_t launch_combine(const uint16_t* y, const int32_t* slot_pos, const flo
                            uint16_t* out, int num_sms, cudaStream_t st) {
     const int64_t total = (int64_t)T * (H / 8);
     int64_t blocks = (total + 255) / 256;
-    const int64_t cap = (int64_t)num_sms * 8;
+    static int knob_carve = getenv("UBEP_X_CARVE") ? atoi(getenv("UBEP_X_CARVE")) : -1;
+    static int knob_wave = getenv("UBEP_X_WAVE") ? atoi(getenv("UBEP_X_WAVE")) : 8;
+    if (knob_carve >= 0) {
+        cudaFuncSetAttribute(combine_kernel<8>, cudaFuncAttributePreferredSharedMemoryCarveout, knob_carve);
+    }
+    const int64_t cap = knob_wave > 0 ? (int64_t)num_sms * knob_wave : blocks;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
     switch (k) {

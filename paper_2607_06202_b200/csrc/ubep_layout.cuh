@@ -98,11 +98,11 @@ __device__ __forceinline__ void stage_ids(const Params& p, int t0, int t1, int* 
 // the row placement needs -- is a population count of the bits below the token, and the
 // range's histogram is the population count of all bits.
 //
-// Built per group of 32 tokens: each lane ORs the bins of its own token into a private row
-// of words (mask_t), then the warp transposes each 32x32 bit tile (lane = token, bit = bin
-// -> lane = bin, bit = token) with five shuffle steps and stores it bin-major (bm).
+// Built per group of 32 tokens and word of 32 bins: each lane ORs the bins of its own token
+// into a register, then the warp transposes the 32x32 bit tile (lane = token, bit = bin ->
+// lane = bin, bit = token) with five shuffle steps and stores it bin-major (bm).
 struct BinMaps {
-    unsigned* mask_t;  // [groups * 32, wbs] token-major scratch rows
+    unsigned* mask_t;  // [groups * 32] scratch words (duty bitmaps of the flag-free kernel)
     unsigned* bm;      // [groups, bp] bit (token & 31) of word [token >> 5][bin]
     int wb;            // words per token row that carry bins: ceil(B / 32)
     int wbs;           // row stride in words (odd, keeps the rows bank-conflict free)
@@ -122,49 +122,26 @@ __device__ __forceinline__ unsigned transpose32(unsigned x, int lane) {
     return x;  // bit b of lane i before == bit i of lane b after
 }
 
-// ids: staged slots of the range (index 0 = first token's slot 0); run by nw warps.
-constexpr int kRegWords = 12;  // up to 384 bins are masked in registers
+// ids: staged slots of the range (index 0 = first token's slot 0); run by nw warps.  One unit
+// of work = one 32-token group x one 32-bin word: the lane (= token) collects the bins of
+// that word its token selected, the warp transposes the tile and stores it bin-major.
 __device__ void build_bin_maps(const Params& p, const int* ids, int ntok, const BinMaps& bmaps, int gw, int nw,
                                int lane) {
     const int k = p.k;
-    if (bmaps.wb <= kRegWords) {
-        for (int g = gw; g < bmaps.groups; g += nw) {
-            const int tl = g * 32 + lane;
-            unsigned m[kRegWords];
-#pragma unroll
-            for (int w = 0; w < kRegWords; ++w) m[w] = 0u;
-            if (tl < ntok) {
-                for (int j = 0; j < k; ++j) {
-                    const int v = ids[tl * k + j];
-                    if (v < 0) continue;
-                    const int e = slot_expert(v), rb = p.E + slot_rank(v);
-                    const unsigned be = 1u << (e & 31), br = 1u << (rb & 31);
-                    const int we = e >> 5, wr = rb >> 5;
-#pragma unroll
-                    for (int w = 0; w < kRegWords; ++w) m[w] |= (w == we ? be : 0u) | (w == wr ? br : 0u);
-                }
-            }
-#pragma unroll
-            for (int w = 0; w < kRegWords; ++w)
-                if (w < bmaps.wb) bmaps.bm[(size_t)g * bmaps.bp + w * 32 + lane] = transpose32(m[w], lane);
-        }
-        return;
-    }
-    for (int g = gw; g < bmaps.groups; g += nw) {
+    const int units = bmaps.groups * bmaps.wb;
+    for (int u = gw; u < units; u += nw) {
+        const int g = u / bmaps.wb, w = u - g * bmaps.wb;
         const int tl = g * 32 + lane;
-        unsigned* row = bmaps.mask_t + (size_t)tl * bmaps.wbs;
-        for (int w = 0; w < bmaps.wb; ++w) row[w] = 0u;
+        unsigned m = 0u;
         if (tl < ntok) {
             for (int j = 0; j < k; ++j) {
                 const int v = ids[tl * k + j];
                 if (v < 0) continue;
                 const int e = slot_expert(v), rb = p.E + slot_rank(v);
-                row[e >> 5] |= 1u << (e & 31);
-                row[rb >> 5] |= 1u << (rb & 31);
+                m |= ((e >> 5) == w ? 1u << (e & 31) : 0u) | ((rb >> 5) == w ? 1u << (rb & 31) : 0u);
             }
         }
-        for (int w = 0; w < bmaps.wb; ++w)
-            bmaps.bm[(size_t)g * bmaps.bp + w * 32 + lane] = transpose32(row[w], lane);
+        bmaps.bm[(size_t)g * bmaps.bp + w * 32 + lane] = transpose32(m, lane);
     }
 }
 
@@ -216,22 +193,27 @@ __device__ void scan_rank_publish(const Params& p, int r, int* sm, int gw, int n
     const int nb = L + 1;
     for (int bi = gw; bi < nb; bi += nw) {
         const int bin = bi < L ? r * L + bi : E + r;
+        // lane l owns the `per` consecutive chunks starting at l * per: all loads first (one
+        // round trip to L2), a serial sum per lane, one warp scan, a serial prefix per lane
+        const int per = (n + 31) / 32;
         int v[kMaxChunks / 32];
-#pragma unroll
-        for (int i = 0; i < kMaxChunks / 32; ++i) {   // all loads first: one round trip to L2
-            const int c = i * 32 + lane;
-            v[i] = c < n ? __ldcg(p.chunk_hist + (size_t)c * B + bin) : 0;
-        }
-        int carry = 0;
+        int mine = 0;
 #pragma unroll
         for (int i = 0; i < kMaxChunks / 32; ++i) {
-            const int c = i * 32 + lane;
-            if (i * 32 < n) {
-                const int incl = warp_incl_scan(v[i], lane);
-                if (c < n) p.chunk_base[(size_t)c * B + bin] = carry + incl - v[i];
-                carry += __shfl_sync(0xffffffffu, incl, 31);
-            }
+            const int c = lane * per + i;
+            v[i] = (i < per && c < n) ? __ldcg(p.chunk_hist + (size_t)c * B + bin) : 0;
         }
+#pragma unroll
+        for (int i = 0; i < kMaxChunks / 32; ++i) mine += v[i];
+        const int incl = warp_incl_scan(mine, lane);
+        int run = incl - mine;
+#pragma unroll
+        for (int i = 0; i < kMaxChunks / 32; ++i) {
+            const int c = lane * per + i;
+            if (i < per && c < n) p.chunk_base[(size_t)c * B + bin] = run;
+            run += v[i];
+        }
+        const int carry = __shfl_sync(0xffffffffu, incl, 31);
         if (lane == 0) sm[bi] = carry;
     }
     group_sync(bar_id, nw * 32);
