@@ -79,7 +79,10 @@ struct Params {
 // ------------------------------------------------------------------ small helpers
 
 __device__ __forceinline__ int64_t chunk_begin(int c, int T, int n) { return (int64_t)c * T / n; }
-__device__ __forceinline__ int src_begin(int s, int T, int S) { return (int)((int64_t)s * T / S); }
+__device__ __forceinline__ int src_begin(int s, int T, int S) {
+    if ((int64_t)S * T < 0x7fffffffLL) return (int)((unsigned)s * (unsigned)T / (unsigned)S);  // the usual case
+    return (int)((int64_t)s * T / S);
+}
 // Chunk that owns token b: the c with chunk_begin(c) <= b < chunk_begin(c + 1).
 __device__ __forceinline__ int chunk_of(int b, int T, int n) {
     return (int)((((int64_t)b + 1) * n - 1) / T);
@@ -219,6 +222,15 @@ struct SmemPlan {
     int off_out, off_ids, off_mask, off_bm, off_pos, off_key, off_ord, off_w, off_hist, off_arr, off_order;
     int total;
 };
+
+// Programmatic dependent launch: a kernel launched with the programmatic-serialization
+// attribute may be scheduled while its predecessor in the stream still runs; it must not
+// touch anything the predecessor produces before griddep_wait() returns (which is when the
+// predecessor has completed and its writes are visible).  griddep_launch() tells the
+// scheduler that the next kernel in the stream may start being placed.  Both are no-ops for
+// a kernel launched the ordinary way.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // Barrier among a subset of the CTA's warps (id 1..15), `nthreads` a multiple of 32.
 __device__ __forceinline__ void group_sync(int id, int nthreads) {

@@ -11,7 +11,6 @@
 //   combine_kernel<K>                 gather + fp32 weighted sum + one bf16 rounding
 //   layout_kernel                     counts only (ubep_get_dispatch_layout)
 #include <cuda_fp8.h>
-#include <cstdlib>
 
 #include "ubep_kernels.h"
 #include "ubep_layout.cuh"
@@ -107,7 +106,7 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
     int* order_sm = reinterpret_cast<int*>(smem + pl.off_order);
     volatile int* abortp = &abort_flag;
     int issued = 0;  // rows whose load thread 0 has started
-    const unsigned epoch = current_epoch(p);
+    griddep_launch();   // the next kernel in the stream may be placed as soon as SMs have room
 
     constexpr int gn = kThreads - 32;  // layout group: warps 1..15
     constexpr int nw = kWarps - 1;
@@ -129,6 +128,8 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
     }
     for (int r = tid; r < p.R; r += kThreads) arr[r] = 0;
     __syncthreads();
+    griddep_wait();     // set-up done; everything below reads what earlier kernels wrote
+    const unsigned epoch = current_epoch(p);
     if (tid == 0) trace(p, c, kTrStart);
 
     const unsigned in_bytes = (unsigned)(p.H * 2 / p.parts);   // this CTA's piece of a bf16 row
@@ -243,8 +244,18 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
                 mbar_arrive(&ready_bar);
                 trace(p, c, kTrReady);
             }
-            if (part == 0) local_meta_dedup(p, t0, t1, ids_sm, pos_raw, row_sm, gtid, gn);
-            for (int r = c; r < p.R; r += p.grid) local_rank_duty(p, r, ids_sm, rm, hist, gw, nw, lane, gtid, gn, 1);
+            if (part == 0) {
+                float* w_own = reinterpret_cast<float*>(key);   // the ordering keys are no longer needed
+                for (int i = gtid; i < ntok * p.k; i += gn) w_own[i] = __ldg(p.topk_w + (size_t)t0 * p.k + i);
+            }
+            group_sync(1, gn);
+            if (part == 0) local_meta_dedup(p, t0, t1, ids_sm, pos_raw, row_sm, reinterpret_cast<float*>(key), gtid, gn);
+            {
+                // expert-level outputs of rank r: shared by Q CTAs so that no CTA trails the others
+                const int Q = p.grid / p.R > 1 ? p.grid / p.R : 1;
+                for (int u = c; u < p.R * Q; u += p.grid)
+                    local_rank_duty(p, u / Q, u % Q, Q, ids_sm, rm, hist, gw, nw, lane, gtid, gn, 1);
+            }
         } else if (kMode == kModeLocal) {
             // every CTA: bitmaps over the whole routing table -> totals, the rows before its
             // own tokens, and (CTAs with a source-rank duty) that rank's counts
@@ -520,6 +531,7 @@ __global__ void __launch_bounds__(256) combine_kernel(const uint16_t* __restrict
     const int nvec = H / 8;
     const int64_t total = (int64_t)T * nvec;
     const int kk = K > 0 ? K : k;
+    griddep_launch();   // lets a dispatch that follows in the stream be placed while this kernel drains
     for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < total;
          u += (int64_t)gridDim.x * blockDim.x) {
         const int t = (int)(u / nvec), v = (int)(u - (int64_t)t * nvec);
@@ -656,6 +668,11 @@ int plan_dispatch(const Params& p, int mode, int max_smem, SmemPlan* out) {
     if (fixed + 4 * (int64_t)pl.stage_bytes > max_smem) return -1;
     pl.stages = (int)((max_smem - fixed) / pl.stage_bytes);
     if (pl.stages > kMaxStages) pl.stages = kMaxStages;
+    // no more stages than rows this CTA will ever hold at once
+    {
+        const int want = chunk_tokens + 3 < 4 ? 4 : chunk_tokens + 3;
+        if (pl.stages > want) pl.stages = want;
+    }
     int at = pl.stages * pl.stage_bytes;
     pl.off_out = at; at += kOutStages * pl.out_stage_bytes;
     pl.off_ids = at; at += (int)ids_ints * 4;
@@ -673,13 +690,30 @@ int plan_dispatch(const Params& p, int mode, int max_smem, SmemPlan* out) {
     return 0;
 }
 
+// Launch that lets the kernel be placed while its predecessor in the stream drains (the
+// kernels above call griddep_wait() before they read anything).
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_overlapped(void (*kern)(KArgs...), int grid, int block, size_t smem, cudaStream_t st,
+                                     Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, args...);
+}
+
 template <int kMode, bool kFp8>
 static cudaError_t launch_dispatch_t(const Params& p, const SmemPlan& pl, cudaStream_t st) {
     auto kern = dispatch_kernel<kMode, kFp8>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.total);
     if (e != cudaSuccess) return e;
-    kern<<<p.grid, kThreads, pl.total, st>>>(p, pl);
-    return cudaGetLastError();
+    return launch_overlapped(kern, p.grid, kThreads, (size_t)pl.total, st, p, pl);
 }
 
 cudaError_t launch_dispatch(const Params& p, int mode, const SmemPlan& pl, cudaStream_t st, int* launches) {
@@ -709,20 +743,17 @@ cudaError_t launch_combine(const uint16_t* y, const int32_t* slot_pos, const flo
                            uint16_t* out, int num_sms, cudaStream_t st) {
     const int64_t total = (int64_t)T * (H / 8);
     int64_t blocks = (total + 255) / 256;
-    static int knob_carve = getenv("UBEP_X_CARVE") ? atoi(getenv("UBEP_X_CARVE")) : -1;
-    static int knob_wave = getenv("UBEP_X_WAVE") ? atoi(getenv("UBEP_X_WAVE")) : 8;
-    if (knob_carve >= 0) {
-        cudaFuncSetAttribute(combine_kernel<8>, cudaFuncAttributePreferredSharedMemoryCarveout, knob_carve);
-    }
-    const int64_t cap = knob_wave > 0 ? (int64_t)num_sms * knob_wave : blocks;
+    const int64_t cap = (int64_t)num_sms * 8;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
+    const int g = (int)blocks;
+    // ordinary launches: combine CTAs parked beside a running dispatch were measured to slow it down
     switch (k) {
-        case 1: combine_kernel<1><<<(int)blocks, 256, 0, st>>>(y, slot_pos, topk_w, T, H, k, out); break;
-        case 2: combine_kernel<2><<<(int)blocks, 256, 0, st>>>(y, slot_pos, topk_w, T, H, k, out); break;
-        case 4: combine_kernel<4><<<(int)blocks, 256, 0, st>>>(y, slot_pos, topk_w, T, H, k, out); break;
-        case 8: combine_kernel<8><<<(int)blocks, 256, 0, st>>>(y, slot_pos, topk_w, T, H, k, out); break;
-        default: combine_kernel<0><<<(int)blocks, 256, 0, st>>>(y, slot_pos, topk_w, T, H, k, out); break;
+        case 1: combine_kernel<1><<<g, 256, 0, st>>>(y, slot_pos, topk_w, T, H, k, out); break;
+        case 2: combine_kernel<2><<<g, 256, 0, st>>>(y, slot_pos, topk_w, T, H, k, out); break;
+        case 4: combine_kernel<4><<<g, 256, 0, st>>>(y, slot_pos, topk_w, T, H, k, out); break;
+        case 8: combine_kernel<8><<<g, 256, 0, st>>>(y, slot_pos, topk_w, T, H, k, out); break;
+        default: combine_kernel<0><<<g, 256, 0, st>>>(y, slot_pos, topk_w, T, H, k, out); break;
     }
     return cudaGetLastError();
 }

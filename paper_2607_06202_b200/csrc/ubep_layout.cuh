@@ -422,7 +422,7 @@ __device__ void local_rows_dedup(const Params& p, int t0, int t1, const int* ids
 
 // Metadata of this CTA's own tokens (after the movers were released).
 __device__ void local_meta_dedup(const Params& p, int t0, int t1, const int* ids_all, const int* pos_raw,
-                                 const int* row_sm, int gtid, int gn) {
+                                 const int* row_sm, const float* w_own, int gtid, int gn) {
     const int k = p.k, L = p.L;
     const int nslots = (t1 - t0) * k;
     for (int li = gtid; li < nslots; li += gn) {
@@ -440,7 +440,7 @@ __device__ void local_meta_dedup(const Params& p, int t0, int t1, const int* ids
                 const int v2 = ids_all[(size_t)t * k + jj];
                 const bool here = v2 >= 0 && slot_rank(v2) == r;
                 p.recv_topk_idx[(size_t)where * k + jj] = here ? slot_expert(v2) - r * L : -1;
-                p.recv_topk_w[(size_t)where * k + jj] = here ? __ldg(p.topk_w + (size_t)t * k + jj) : 0.0f;
+                p.recv_topk_w[(size_t)where * k + jj] = here ? w_own[tl * k + jj] : 0.0f;
             }
         }
     }
@@ -449,8 +449,10 @@ __device__ void local_meta_dedup(const Params& p, int t0, int t1, const int* ids
 // Everything about rank r that nobody inside the kernel waits for: expert totals and
 // offsets, tokens per rank, counts and offsets per source rank, the per-expert row lists.
 // Needs L < 32.  `sm` holds 2 * 32 ints.  Run by the whole layout group (barrier bar_id).
-__device__ void local_rank_duty(const Params& p, int r, const int* ids_all, const RankMaps& rm, int* sm, int gw,
-                                int nw, int lane, int gtid, int gn, int bar_id) {
+// The rank's share is cut into Q parts handled by Q different CTAs: part q writes every
+// Q-th entry of the per-source tables and of the row lists; part 0 also writes the totals.
+__device__ void local_rank_duty(const Params& p, int r, int q, int Q, const int* ids_all, const RankMaps& rm,
+                                int* sm, int gw, int nw, int lane, int gtid, int gn, int bar_id) {
     const int k = p.k, L = p.L, T = p.T, S = p.S, E = p.E;
     for (int g = gw; g < rm.groups; g += nw) {
         const int t = g * 32 + lane;
@@ -481,24 +483,26 @@ __device__ void local_rank_duty(const Params& p, int r, const int* ids_all, cons
     group_sync(bar_id, gn);
     if (gtid <= L) {
         int o = 0;
-        for (int q = 0; q < gtid; ++q) o += tot[q];
+        for (int i = 0; i < gtid; ++i) o += tot[i];
         eo[gtid] = o;
-        if (gtid < L) {
-            p.expert_offset[r * L + gtid] = o;
-            p.num_tokens_per_expert[r * L + gtid] = tot[gtid];
-        } else {
-            p.num_tokens_per_rank[r] = tot[L];
-            p.num_rows_per_rank[r] = tot[L];
+        if (q == 0) {
+            if (gtid < L) {
+                p.expert_offset[r * L + gtid] = o;
+                p.num_tokens_per_expert[r * L + gtid] = tot[gtid];
+            } else {
+                p.num_tokens_per_rank[r] = tot[L];
+                p.num_rows_per_rank[r] = tot[L];
+            }
         }
     }
     group_sync(bar_id, gn);
-    for (int i = gtid; i < S * L; i += gn) {
+    for (int i = q + Q * gtid; i < S * L; i += Q * gn) {
         const int s = i / L, l = i - s * L;
         const int b0 = src_begin(s, T, S), b1 = src_begin(s + 1, T, S);
         p.cnt[(size_t)s * E + r * L + l] = bits(l, b0, b1);
         p.src_offset[(size_t)s * E + r * L + l] = eo[l] + bits(l, 0, b0);
     }
-    for (int i = gtid; i < T * k; i += gn) {
+    for (int i = q + Q * gtid; i < T * k; i += Q * gn) {
         const int v = ids_all[i];
         if (v < 0 || slot_rank(v) != r) continue;
         const int t = i / k, l = slot_expert(v) - r * L;
