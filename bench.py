@@ -348,8 +348,10 @@ def run_ours(args, cfg, rank: int, world: int, local_rank: int):
     achieved = dom_bytes / (dom_us * 1e-6) / 1e9
     traffic = None
     try:
-        prof = json.load(open(os.path.join(ROOT, "profiles", "traffic.json")))
-        traffic = prof.get(cfg.name, {}).get(dom)
+        for ln in open(os.path.join(ROOT, "profiles", "traffic.txt")):
+            f = ln.split()
+            if len(f) == 3 and f[0] == cfg.name and f[1] == dom:
+                traffic = int(f[2])
     except Exception:
         pass
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
