@@ -151,6 +151,35 @@ int ubep_get_dispatch_layout(ubep_buffer_t *buf, const int32_t *topk_idx /*[dev]
                              uint8_t *is_token_in_rank /*[dev]*/, void *cuda_stream);
 
 /*
+ * Counts without any caller-provided scratch (the paper has no counterpart; this entry
+ * point exists for callers that may not allocate).  Same results as
+ * ubep_get_dispatch_layout, but it needs no buffer handle and no arena: a caller that
+ * runs inside somebody else's memory plan -- a plugin handed fixed input and output
+ * tensors, code running while allocation is forbidden -- cannot reserve an arena, so the
+ * chunk histograms live in a fixed array of UBEP_STATIC_MAX_BINS x 64 32-bit words
+ * (about 257 KB) inside the library's device image.  Every GPU that loads the library holds
+ * that array until the process exits.
+ *
+ * Limits: num_experts + num_ranks <= UBEP_STATIC_MAX_BINS, topk <= 32, num_experts %
+ * num_ranks == 0; anything larger returns UBEP_ERR_ARG and launches nothing.  No replica
+ * table; expert ids outside [-1, num_experts) are skipped.  topk_idx [dev] int32 [T, topk],
+ * 16-byte aligned; outputs [dev] as for ubep_get_dispatch_layout (any may be NULL).
+ *
+ * The first call on each device looks up the array's device address (with that device
+ * current) and keeps it; make that first call before any stream capture begins.  The call
+ * itself calls no cudaMalloc, cudaFree or other allocating routine.  All calls on a device
+ * share the one array: calls whose kernels may overlap on the GPU (different streams) race
+ * on it -- keep them on one stream or otherwise ordered.  The array keeps the previous
+ * call's contents; the kernel overwrites what it reads and re-arms its own counter.
+ */
+#define UBEP_STATIC_MAX_BINS 1024
+int ubep_get_dispatch_layout_static(const int32_t *topk_idx /*[dev]*/, int32_t T, int32_t topk,
+                                    int32_t num_experts, int32_t num_ranks,
+                                    int32_t *num_tokens_per_rank /*[dev]*/,
+                                    int32_t *num_tokens_per_expert /*[dev]*/,
+                                    uint8_t *is_token_in_rank /*[dev]*/, void *cuda_stream);
+
+/*
  * Dispatch (Sec. 2.3 phases 1-5 fused as in Sec. 3.2): counts, prefix-sum offsets, row
  * assignment, optional FP8 quantisation, and the copy of every token row into the receive
  * regions of the ranks that host its experts.  x [dev] bf16 [T, H]; topk_idx [dev] int32

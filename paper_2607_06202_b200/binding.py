@@ -32,7 +32,7 @@ _VIEW_DTYPES = [torch.uint8, torch.float32, torch.int32, torch.float32, torch.in
 
 # every symbol include/ubep.h declares
 EXPORTS = ["ubep_buffer_bytes", "ubep_buffer_create", "ubep_buffer_destroy", "ubep_set_replicas",
-           "ubep_set_dest_order", "ubep_get_dispatch_layout", "ubep_dispatch", "ubep_combine", "ubep_view",
+           "ubep_set_dest_order", "ubep_get_dispatch_layout", "ubep_get_dispatch_layout_static", "ubep_dispatch", "ubep_combine", "ubep_view",
            "ubep_status", "ubep_epoch", "ubep_launch_count", "ubep_debug_withhold_flag", "ubep_debug_trace",
            "ubep_last_cuda_error", "ubep_strerror"]
 
@@ -64,6 +64,8 @@ def load() -> ctypes.CDLL:
     lib.ubep_set_dest_order.restype, lib.ubep_set_dest_order.argtypes = ctypes.c_int, [vp, vp]
     lib.ubep_get_dispatch_layout.restype = ctypes.c_int
     lib.ubep_get_dispatch_layout.argtypes = [vp, vp, i32, vp, vp, vp, vp]
+    lib.ubep_get_dispatch_layout_static.restype = ctypes.c_int
+    lib.ubep_get_dispatch_layout_static.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp]
     lib.ubep_dispatch.restype, lib.ubep_dispatch.argtypes = ctypes.c_int, [vp, vp, vp, vp, i32, vp]
     lib.ubep_combine.restype, lib.ubep_combine.argtypes = ctypes.c_int, [vp, vp, vp, i32, vp, vp]
     lib.ubep_view.restype = ctypes.c_int
@@ -148,6 +150,16 @@ def ubep_get_dispatch_layout(buf, topk_idx: torch.Tensor, T: int, num_tokens_per
     _check(load().ubep_get_dispatch_layout(buf, _ptr(topk_idx), T, _ptr(num_tokens_per_rank),
                                            _ptr(num_tokens_per_expert), _ptr(is_token_in_rank), _stream(stream)),
            "ubep_get_dispatch_layout", buf)
+
+
+def ubep_get_dispatch_layout_static(topk_idx: torch.Tensor, T: int, topk: int, num_experts: int, num_ranks: int,
+                                    num_tokens_per_rank, num_tokens_per_expert, is_token_in_rank, stream=None) -> None:
+    """Counts through the entry point that needs no arena (see include/ubep.h): the caller passes only the
+    routing table and the output tensors; scratch lives in a fixed array inside the library."""
+    _check(load().ubep_get_dispatch_layout_static(_ptr(topk_idx), T, topk, num_experts, num_ranks,
+                                                  _ptr(num_tokens_per_rank), _ptr(num_tokens_per_expert),
+                                                  _ptr(is_token_in_rank), _stream(stream)),
+           "ubep_get_dispatch_layout_static")
 
 
 def ubep_dispatch(buf, x: torch.Tensor, topk_idx: torch.Tensor, topk_w: torch.Tensor, T: int, stream=None) -> None:
