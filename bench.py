@@ -88,6 +88,23 @@ class ClockSampler(threading.Thread):
                 "samples": len(self.samples)}
 
 
+def max_over_ranks(value: float, world: int, device=None) -> float:
+    """Max of a per-rank number over all ranks (replicas run independently; the job is as slow
+    as its slowest rank).  Works on any initialised process group (nccl on GPUs, gloo on CPU)."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(bytes_per_step_per_rank: float, ms_per_step_max: float, world: int) -> float:
+    """Whole-job GB/s of `world` independent replicas given the slowest rank's time per step."""
+    return world * bytes_per_step_per_rank / (ms_per_step_max * 1e-3) / 1e9
+
+
 def physical_gpu_index(local_index: int) -> int:
     vis = os.environ.get("CUDA_VISIBLE_DEVICES")
     if vis:
@@ -250,12 +267,9 @@ def run_ours(args, cfg, rank: int, world: int, local_rank: int):
     if args.pipeline == B.UBEP_PIPELINE_PHASED:
         launches = 4 * args.steps
     _ = n0
-    if world > 1:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, world, dev)
     ms_per_step = total_ms / args.steps
-    value = world * (disp_b + comb_b) / (ms_per_step * 1e-3) / 1e9
+    value = whole_job_value(disp_b + comb_b, ms_per_step, world)
 
     if args.profile:
         if rank == 0:
@@ -324,13 +338,10 @@ def run_ours(args, cfg, rank: int, world: int, local_rank: int):
         ee1.record(stream)
     barrier()
     e2e_ms = ee0.elapsed_time(ee1) / n_e
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(e2e_ms, world, dev)
     h2d = hx.numel() * 2 + hidx.numel() * 4 + hw.numel() * 4
     d2h = hout.numel() * 2
-    e2e = {"value": world * (disp_b + comb_b) / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s",
+    e2e = {"value": whole_job_value(disp_b + comb_b, e2e_ms, world), "unit": "GB/s",
            "us_per_layer": e2e_ms * 1e3, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
            "experts": "synthetic y" if cfg.payload else "identity (y = receive regions)"}
 
