@@ -506,8 +506,7 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
     }
     // pieces of this CTA's rows have landed: add them to the per-region arrival counters
     // (unit: eighths of a row, so that the total does not depend on the column split)
-    __threadfence();
-    fence_proxy_async();
+    fence_proxy_async();   // rows written through the async proxy, counters through the generic one
     for (int r = tid; r < p.R; r += kThreads)
         if (arr[r]) red_release_add(p.arrival + (epoch & 1) * p.R + r, (unsigned)(arr[r] * (8 / p.parts)));
     // the arrival counters of the next call live in the other half; clear them now

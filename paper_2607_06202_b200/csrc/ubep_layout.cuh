@@ -349,6 +349,7 @@ __device__ __forceinline__ int fast_div(int v, unsigned magic) { return (int)__u
 // Stage all T*k slots (packed id | rank << 16) and build the rank bitmaps; lane = token.
 __device__ void local_stage_and_rank_maps(const Params& p, int* ids, const RankMaps& rm, int gw, int nw, int lane) {
     const int k = p.k, T = p.T;
+    const bool vec = (k & 3) == 0;   // a token's ids are whole 16-byte words (topk_idx is 16-byte aligned)
     for (int g = gw; g < rm.groups; g += nw) {
         const int t = g * 32 + lane;
         unsigned m[kRankWords];
@@ -358,8 +359,15 @@ __device__ void local_stage_and_rank_maps(const Params& p, int* ids, const RankM
             const int32_t* src = p.topk_idx + (size_t)t * k;
             for (int j0 = 0; j0 < k; j0 += 8) {       // up to eight ids in flight
                 int raw[8];
+                if (vec) {
+                    const int4 a = __ldg(reinterpret_cast<const int4*>(src + j0));
+                    const int4 b = j0 + 4 < k ? __ldg(reinterpret_cast<const int4*>(src + j0 + 4)) : make_int4(-1, -1, -1, -1);
+                    raw[0] = a.x; raw[1] = a.y; raw[2] = a.z; raw[3] = a.w;
+                    raw[4] = b.x; raw[5] = b.y; raw[6] = b.z; raw[7] = b.w;
+                } else {
 #pragma unroll
-                for (int u = 0; u < 8; ++u) raw[u] = j0 + u < k ? __ldg(src + j0 + u) : -1;
+                    for (int u = 0; u < 8; ++u) raw[u] = j0 + u < k ? __ldg(src + j0 + u) : -1;
+                }
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
                     if (j0 + u >= k) break;
@@ -368,8 +376,12 @@ __device__ void local_stage_and_rank_maps(const Params& p, int* ids, const RankM
                     if (e >= 0) {
                         const int r = fast_div(e, p.L_magic);
                         packed = e | (r << 16);
+                        if (rm.wr == 1) {
+                            m[0] |= 1u << r;
+                        } else {
 #pragma unroll
-                        for (int w = 0; w < kRankWords; ++w) m[w] |= (w == (r >> 5)) ? 1u << (r & 31) : 0u;
+                            for (int w = 0; w < kRankWords; ++w) m[w] |= (w == (r >> 5)) ? 1u << (r & 31) : 0u;
+                        }
                     }
                     ids[t * k + j0 + u] = packed;
                 }
@@ -391,6 +403,8 @@ __device__ __forceinline__ int rank_rows_before(const RankMaps& rm, int r, int t
 }
 
 // Destinations of this CTA's tokens [t0, t1): pos_raw (slot order), dst_rank, row_sm, arr.
+// (Ordering the destinations with warp shuffles right here instead of in a separate pass
+// was measured slower on the decode shape and is not done.)
 __device__ void local_rows_dedup(const Params& p, int t0, int t1, const int* ids_all, const RankMaps& rm,
                                  int* pos_raw, int* dst_rank, int* row_sm, int* arr, int gtid, int gn) {
     const int k = p.k;
