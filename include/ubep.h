@@ -200,6 +200,21 @@ int ubep_dispatch(ubep_buffer_t *buf, const void *x /*[dev]*/, const int32_t *to
 int ubep_combine(ubep_buffer_t *buf, const void *y /*[dev]*/, const float *topk_w /*[dev]*/,
                  int32_t T, void *out /*[dev]*/, void *cuda_stream);
 
+/*
+ * Token-level load partition with the prefix-sum search of Algorithm 1 (Sec. 3.3): the send
+ * sequence is the experts in the order `order` ([dev] int32 [n], ids in [0, num_experts)),
+ * expert e contributing counts[e] tokens ([dev] int32 [num_experts]).  It is cut into
+ * n_workers contiguous slices whose sizes differ by at most one token; worker w starts at
+ * global token floor(w * total / n_workers).  Outputs ([dev], caller-owned, n_workers + 1
+ * entries each; entry n_workers closes the last slice): start_pos[w] = position in `order`
+ * of the expert whose cumulative range covers that token (n if the worker has no work),
+ * start_off[w] = offset inside that expert (int64), iters[w] = search iterations (may be
+ * NULL).  One launch of one CTA on `cuda_stream`; ids of `order` out of range count as empty.
+ */
+int ubep_map_workers(const int32_t *order /*[dev]*/, const int32_t *counts /*[dev]*/, int32_t n,
+                     int32_t num_experts, int32_t n_workers, int32_t *start_pos /*[dev]*/,
+                     int64_t *start_off /*[dev]*/, int32_t *iters /*[dev]*/, void *cuda_stream);
+
 /* Device address and shape (unused dims = 1) of one arena array; valid until destroy. */
 int ubep_view(ubep_buffer_t *buf, int which, void **dev_ptr /*[host]*/, int64_t shape[4] /*[host]*/);
 

@@ -56,6 +56,7 @@ def _load():
     for name in ("orc_resolve_ids", "orc_layout", "orc_fp8_quantize_row", "orc_dispatch",
                  "orc_combine", "orc_quaternary_search"):
         getattr(lib, name).restype = ctypes.c_int
+    lib.orc_hop_distribution.restype = None
     lib.orc_stride_remap.restype = None
     lib.orc_equal_slices.restype = None
     _ = c_i32p
@@ -250,3 +251,13 @@ def equal_slices(total: int, workers: int) -> np.ndarray:
     begin = np.empty(workers + 1, np.int64)
     _load().orc_equal_slices(ctypes.c_int64(total), workers, _p(begin))
     return begin
+
+
+def hop_distribution(order: np.ndarray, counts: np.ndarray, hop_of: np.ndarray, workers: int, n_hops: int) -> np.ndarray:
+    """v[w][h]: tokens of hop class h in worker w's slice of the send sequence."""
+    order = np.ascontiguousarray(order, np.int32)
+    counts = np.ascontiguousarray(counts, np.int32)
+    hop_of = np.ascontiguousarray(hop_of, np.int32)
+    v = np.empty((workers, n_hops), np.int64)
+    _load().orc_hop_distribution(_p(order), _p(counts), _p(hop_of), len(order), workers, n_hops, _p(v))
+    return v

@@ -457,3 +457,26 @@ void orc_equal_slices(int64_t total, int workers, int64_t *begin)
 {
     for (int w = 0; w <= workers; ++w) begin[w] = (int64_t)w * total / workers;
 }
+
+/*
+ * Hop-count distribution of the workers (Sec. 3.3, latency homogenisation): worker w sends
+ * the tokens of its slice of the send sequence; v[w][h] = how many of them go to an expert
+ * of hop class h (hop_of[e] in [0, n_hops)).  The heuristic aims at v[w][h] <= ceil(V_h / n)
+ * with V_h the total number of h-hop tokens.  Literal walk over the slices.
+ */
+void orc_hop_distribution(const int32_t *order, const int32_t *counts, const int32_t *hop_of, int n,
+                          int workers, int n_hops, int64_t *v)
+{
+    int64_t total = cum_before(order, counts, n);
+    memset(v, 0, sizeof(int64_t) * (size_t)workers * n_hops);
+    for (int w = 0; w < workers; ++w) {
+        int64_t lo = (int64_t)w * total / workers, hi = (int64_t)(w + 1) * total / workers;
+        int64_t at = 0;                       /* tokens before expert position i */
+        for (int i = 0; i < n; ++i) {
+            int64_t c = counts[order[i]];
+            int64_t a = at > lo ? at : lo, b = at + c < hi ? at + c : hi;
+            if (b > a) v[(size_t)w * n_hops + hop_of[order[i]]] += b - a;
+            at += c;
+        }
+    }
+}

@@ -34,7 +34,7 @@ _VIEW_DTYPES = [torch.uint8, torch.float32, torch.int32, torch.float32, torch.in
 EXPORTS = ["ubep_buffer_bytes", "ubep_buffer_create", "ubep_buffer_destroy", "ubep_set_replicas",
            "ubep_set_dest_order", "ubep_get_dispatch_layout", "ubep_get_dispatch_layout_static", "ubep_dispatch", "ubep_combine", "ubep_view",
            "ubep_status", "ubep_epoch", "ubep_launch_count", "ubep_debug_withhold_flag", "ubep_debug_trace",
-           "ubep_last_cuda_error", "ubep_strerror"]
+           "ubep_last_cuda_error", "ubep_strerror", "ubep_map_workers"]
 
 
 class ubep_config_t(ctypes.Structure):
@@ -77,6 +77,8 @@ def load() -> ctypes.CDLL:
     lib.ubep_debug_trace.restype, lib.ubep_debug_trace.argtypes = ctypes.c_int, [vp, i32]
     lib.ubep_last_cuda_error.restype, lib.ubep_last_cuda_error.argtypes = ctypes.c_char_p, [vp]
     lib.ubep_strerror.restype, lib.ubep_strerror.argtypes = ctypes.c_char_p, [ctypes.c_int]
+    lib.ubep_map_workers.restype = ctypes.c_int
+    lib.ubep_map_workers.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp]
     _lib = lib
     return lib
 
@@ -169,6 +171,15 @@ def ubep_dispatch(buf, x: torch.Tensor, topk_idx: torch.Tensor, topk_w: torch.Te
 
 def ubep_combine(buf, y: torch.Tensor, topk_w: torch.Tensor, T: int, out: torch.Tensor, stream=None) -> None:
     _check(load().ubep_combine(buf, _ptr(y), _ptr(topk_w), T, _ptr(out), _stream(stream)), "ubep_combine", buf)
+
+
+def ubep_map_workers(order: torch.Tensor, counts: torch.Tensor, n_workers: int, start_pos: torch.Tensor,
+                     start_off: torch.Tensor, iters: Optional[torch.Tensor] = None, stream=None) -> None:
+    assert order.dtype == torch.int32 and counts.dtype == torch.int32
+    assert start_pos.dtype == torch.int32 and start_off.dtype == torch.int64
+    _check(load().ubep_map_workers(_ptr(order), _ptr(counts), order.numel(), counts.numel(), n_workers,
+                                   _ptr(start_pos), _ptr(start_off), _ptr(iters), _stream(stream)),
+           "ubep_map_workers")
 
 
 def ubep_view(buf, which: int):

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libubep.so")
-SOURCES = ["ubep_kernels.cu", "ubep_host.cu", "ubep_static.cu"]
+SOURCES = ["ubep_kernels.cu", "ubep_host.cu", "ubep_static.cu", "ubep_mapper.cu"]
 DEPENDS = SOURCES + ["ubep_common.cuh", "ubep_layout.cuh", "ubep_kernels.h", "../../include/ubep.h"]
 
 

@@ -62,8 +62,7 @@ struct Params {
     int32_t* num_tokens_per_expert;
     int32_t* num_rows_per_rank;
     int32_t* num_tokens_per_rank;
-    int32_t* slot_row;   // [T, k] region-local row (chunk-local count until finalised)
-    int32_t* slot_aux;   // [T, k] dedup: chunk-local index into the expert's row list
+    int32_t* slot_row;   // [T, k] region-local row of each slot, -1 if none
     int32_t* slot_pos;   // [T, k] global row (rank * cap + row) of each slot, -1 if none
     // scratch
     int32_t* chunk_hist;  // [nchunks, B]
@@ -218,7 +217,7 @@ __device__ __forceinline__ void fence_proxy_async_smem() {
 struct SmemPlan {
     int stages, stage_bytes;          // input row ring
     int out_stage_bytes;              // FP8: kOutStages quantised rows
-    int map_groups, map_wb, map_wbs, map_bp;  // bin bitmaps: 32-token groups, words, stride, padded bins
+    int map_groups, map_wb, map_bp;   // bin bitmaps: 32-token groups, words of bins, padded bins
     int off_out, off_ids, off_mask, off_bm, off_pos, off_key, off_ord, off_w, off_hist, off_arr, off_order;
     int total;
 };

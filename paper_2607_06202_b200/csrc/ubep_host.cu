@@ -22,7 +22,7 @@ inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 
 struct ArenaLayout {
     size_t off[UBEP_VIEW_COUNT_];
-    size_t slot_aux, slot_pos, chunk_hist, partial, chunk_base, trace;
+    size_t slot_pos, chunk_hist, partial, chunk_base, trace;
     size_t flags_begin, hist_flag, scan_flag, status, ticket, epoch_ctr, done_ticket, order_pos, flags_end;
     size_t total;
     int er_cap, nchunks, S, rowB, G, B;
@@ -72,7 +72,6 @@ ArenaLayout make_layout(const ubep_config_t& c, int nchunks) {
     a.off[UBEP_VIEW_NUM_ROWS_PER_RANK] = take(R * 4);
     a.off[UBEP_VIEW_NUM_TOKENS_PER_RANK] = take(R * 4);
     a.off[UBEP_VIEW_SLOT_ROW] = take(Tk * 4);
-    a.slot_aux = take(Tk * 4);
     a.slot_pos = take(Tk * 4);
     a.chunk_hist = take(n * B * 4);
     a.partial = take(S * B * 4);
@@ -151,7 +150,6 @@ Params make_params(ubep_buffer* b, int T) {
     p.num_rows_per_rank = at<int32_t>(b, a.off[UBEP_VIEW_NUM_ROWS_PER_RANK]);
     p.num_tokens_per_rank = at<int32_t>(b, a.off[UBEP_VIEW_NUM_TOKENS_PER_RANK]);
     p.slot_row = at<int32_t>(b, a.off[UBEP_VIEW_SLOT_ROW]);
-    p.slot_aux = at<int32_t>(b, a.slot_aux);
     p.slot_pos = at<int32_t>(b, a.slot_pos);
     p.chunk_hist = at<int32_t>(b, a.chunk_hist);
     p.partial = at<int32_t>(b, a.partial);

@@ -24,9 +24,9 @@ __global__ void __launch_bounds__(256) count_kernel(const Params p, const SmemPl
     extern __shared__ __align__(16) uint8_t sm_c[];
     const int c = blockIdx.x, tid = threadIdx.x;
     const int t0 = (int)chunk_begin(c, p.T, p.nchunks), t1 = (int)chunk_begin(c + 1, p.T, p.nchunks);
-    int* ids = reinterpret_cast<int*>(sm_c + (pl.off_ids - pl.off_ids));
+    int* ids = reinterpret_cast<int*>(sm_c);
     BinMaps bmaps{reinterpret_cast<unsigned*>(sm_c + (pl.off_mask - pl.off_ids)),
-                  reinterpret_cast<unsigned*>(sm_c + (pl.off_bm - pl.off_ids)), pl.map_wb, pl.map_wbs, pl.map_bp,
+                  reinterpret_cast<unsigned*>(sm_c + (pl.off_bm - pl.off_ids)), pl.map_wb, pl.map_bp,
                   pl.map_groups};
     stage_ids(p, t0, t1, ids, tid, 256);
     __syncthreads();
@@ -99,7 +99,7 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
     int* key = reinterpret_cast<int*>(smem + pl.off_key);
     float* w_sm = reinterpret_cast<float*>(smem + pl.off_w);
     const BinMaps bmaps{reinterpret_cast<unsigned*>(smem + pl.off_mask),
-                        reinterpret_cast<unsigned*>(smem + pl.off_bm), pl.map_wb, pl.map_wbs, pl.map_bp,
+                        reinterpret_cast<unsigned*>(smem + pl.off_bm), pl.map_wb, pl.map_bp,
                         pl.map_groups};
     int* hist = reinterpret_cast<int*>(smem + pl.off_hist);
     int* arr = reinterpret_cast<int*>(smem + pl.off_arr);
@@ -656,7 +656,6 @@ int plan_dispatch(const Params& p, int mode, int max_smem, SmemPlan* out) {
     if (hist_ints < 64) hist_ints = 64;   // the per-rank duty of the flag-free kernel keeps 2 x 32 ints here
     pl.map_groups = (map_tokens + 31) / 32;
     pl.map_wb = (p.B + 31) / 32;
-    pl.map_wbs = pl.map_wb | 1;
     pl.map_bp = pl.map_wb * 32;
     pl.stage_bytes = round_up_i(p.H * 2 / p.parts, 128);
     pl.out_stage_bytes = p.payload ? round_up_i(p.rowB / p.parts + (p.G / p.parts) * 4, 128) : 0;

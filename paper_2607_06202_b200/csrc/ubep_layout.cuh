@@ -105,7 +105,6 @@ struct BinMaps {
     unsigned* mask_t;  // [groups * 32] scratch words (duty bitmaps of the flag-free kernel)
     unsigned* bm;      // [groups, bp] bit (token & 31) of word [token >> 5][bin]
     int wb;            // words per token row that carry bins: ceil(B / 32)
-    int wbs;           // row stride in words (odd, keeps the rows bank-conflict free)
     int bp;            // bins padded to a multiple of 32
     int groups;        // 32-token groups of the range
 };

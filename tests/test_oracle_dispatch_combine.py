@@ -222,3 +222,32 @@ def test_equal_slices_and_stride_remap(orc):
         m[:n] = np.arange(n)
         ref = m.reshape(rows, cols).T.ravel()
         assert np.array_equal(order, ref[ref >= 0])
+
+
+def test_hop_distribution_and_the_effect_of_the_remap(orc):
+    """Per-worker hop mix: brute force over the expanded token sequence pins the walk; a stride
+    remap whose rows are the four distance groups of the experts (Sec. 3.3; the paper does not
+    give the matrix shape) brings every worker close to the per-hop bound ceil(V_h / n)."""
+    rng = np.random.default_rng(13)
+    n, workers = 64, 16                      # 64 experts in 4 boards of 16; board 0 is one hop away
+    counts = rng.integers(20, 60, n).astype(np.int32)
+    hop_of = (np.arange(n) // 16 >= 1).astype(np.int32)           # 0 = one hop, 1 = two hops
+    natural_order = np.arange(n, dtype=np.int32)
+    remap_order = orc.stride_remap(n, 4)                          # 0, 16, 32, 48, 1, 17, ...
+    for order in (natural_order, remap_order):
+        v = orc.hop_distribution(order, counts, hop_of, workers, 2)
+        seq = np.repeat(hop_of[order], counts[order])            # hop class of every token sent, in order
+        begin = orc.equal_slices(len(seq), workers)
+        brute = np.array([[int((seq[begin[w]:begin[w + 1]] == h).sum()) for h in range(2)] for w in range(workers)])
+        assert np.array_equal(v, brute)
+        assert np.array_equal(v.sum(1), np.diff(begin))          # every token of the slice is counted once
+    V = np.array([counts[hop_of == h].sum() for h in range(2)])
+    bound = -(-V // workers)
+    natural = orc.hop_distribution(natural_order, counts, hop_of, workers, 2)
+    remapped = orc.hop_distribution(remap_order, counts, hop_of, workers, 2)
+    # natural order: four workers send one-hop tokens only, twelve send two-hop tokens only
+    assert natural[:, 0].max() > 3 * bound[0] and (natural[:, 0] == 0).sum() >= 10
+    # remapped: every worker has the global mix, within the size of one expert's token count
+    assert np.all(remapped[:, 0] > 0) and np.all(remapped[:, 1] > 0)
+    assert np.all(remapped <= bound[None, :] + counts.max())
+    assert remapped.var(axis=0).sum() < 0.05 * natural.var(axis=0).sum()      # tr(Sigma) shrinks
