@@ -32,10 +32,11 @@ class Config:
     E_logical: int = 0     # > 0: routing picks among E_logical experts, replica table maps to E
     routing: str = "gauss"  # "gauss" | "zipf"
     zipf_s: float = 1.2
+    num_src_ranks: int = 0  # source ranks; 0 = same as R
 
     @property
     def S(self) -> int:
-        return self.R
+        return self.num_src_ranks if self.num_src_ranks else self.R
 
     @property
     def L(self) -> int:

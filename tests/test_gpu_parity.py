@@ -81,6 +81,30 @@ def test_column_split_rows_and_more_source_ranks_than_chunks(payload, dedup):
     Hn.run_case(W.make_workload(cfg), pipeline=LOCAL, num_ctas=4)
 
 
+@pytest.mark.parametrize("pipeline", [PHASED, FUSED, LOCAL])
+@pytest.mark.parametrize("case", [
+    dict(T=300, H=128, E=64, R=1, k=4),                       # a single rank holding every expert
+    dict(T=100, H=128, E=64, R=2, k=32),                      # the largest top-k the library takes
+    dict(T=257, H=8, E=16, R=4, k=2),                         # the smallest row (16 bytes)
+    dict(T=200, H=256, E=1024, R=128, k=8),                   # many bins: 1152 bitmaps per token range
+    dict(T=90, H=128, E=12, R=4, k=3, num_src_ranks=7),       # source ranks unrelated to the rank count
+    dict(T=5, H=128, E=12, R=4, k=2, num_src_ranks=9),        # more source ranks than tokens
+    dict(T=64, H=128, E=12, R=4, k=2, num_src_ranks=1),       # one source rank
+])
+@pytest.mark.parametrize("dedup", [0, 1])
+def test_extreme_shapes(case, dedup, pipeline):
+    cfg = W.Config("edge", seed=case["T"] + case["E"], dedup=dedup, **case)
+    wl = W.with_empty_slots(W.make_workload(cfg), 0.1, seed=3)
+    Hn.run_case(wl, pipeline=pipeline)
+
+
+@pytest.mark.parametrize("payload,dedup", [(0, 0), (1, 1)])
+def test_many_tokens_per_chunk(payload, dedup):
+    """70 000 tokens on 148 CTAs: 473 tokens (15 bitmap groups) per chunk, rows of 256 bytes."""
+    cfg = W.Config("long", T=70000, H=128, E=32, R=8, k=4, payload=payload, dedup=dedup, seed=71)
+    Hn.run_case(W.make_workload(cfg), pipeline=FUSED, threads=oracle.host_cores())
+
+
 def test_destination_order_table_does_not_change_results():
     cfg = small(300, 256, 32, 8, 4, seed=4)
     wl = W.make_workload(cfg)
