@@ -89,23 +89,6 @@ __device__ __forceinline__ int chunk_of(int b, int T, int n) {
 
 __device__ __forceinline__ void report(int32_t* status, int code) { atomicCAS(status, 0, code); }
 
-// Epoch of the running dispatch: one more than the number of completed dispatches.  Flags
-// must hold this value to count as set, so nothing is ever reset between calls, and a
-// captured CUDA graph can be replayed because the value lives on the device.  The word is
-// only advanced by the last CTA of a dispatch to finish, after every CTA has read it.
-__device__ __forceinline__ unsigned current_epoch(const Params& p) {
-    unsigned e = __ldcg(p.epoch_ctr) + 1u;
-    return e == 0u ? 1u : e;
-}
-__device__ __forceinline__ void finish_dispatch(const Params& p, unsigned epoch) {
-    __threadfence();
-    if (atomicAdd(p.done_ticket, 1u) == (unsigned)p.grid - 1u) {
-        *p.done_ticket = 0u;
-        __threadfence();
-        *p.epoch_ctr = epoch;
-    }
-}
-
 __device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
     unsigned v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -117,6 +100,23 @@ __device__ __forceinline__ void st_release(unsigned* p, unsigned v) {
 __device__ __forceinline__ void red_release_add(unsigned* p, unsigned v) {
     asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
+
+// Epoch of the running dispatch: one more than the number of dispatches that ran before.
+// Flags must hold this value to count as set, so nothing is ever reset between calls, and a
+// captured CUDA graph can be replayed because the value lives on the device.  Thread 0 of
+// every CTA reads the counter (acquire, so that nothing below is performed before the read)
+// and then takes a ticket; the CTA that takes the last ticket knows that every CTA of this
+// launch has read the counter and advances it for the next launch.
+__device__ __forceinline__ unsigned read_epoch_and_check_in(const Params& p) {
+    unsigned e = ld_acquire(p.epoch_ctr) + 1u;
+    if (e == 0u) e = 1u;
+    if (atomicAdd(p.done_ticket, 1u) == (unsigned)p.grid - 1u) {
+        *p.done_ticket = 0u;
+        *p.epoch_ctr = e;
+    }
+    return e;
+}
+
 
 __device__ __forceinline__ unsigned long long global_ns() {
     unsigned long long t;

@@ -86,6 +86,7 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
     __shared__ __align__(8) uint64_t out_empty[kOutStages];   // FP8: its stores have read it
     __shared__ __align__(8) uint64_t ready_bar;               // rows assigned, movers may go
     __shared__ int abort_flag;
+    __shared__ unsigned epoch_sm;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int c = blockIdx.x;
@@ -127,9 +128,10 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
         mbar_fence_init();
     }
     for (int r = tid; r < p.R; r += kThreads) arr[r] = 0;
+    griddep_wait();     // shared-memory set-up done; everything below reads what earlier kernels wrote
+    if (tid == 0) epoch_sm = read_epoch_and_check_in(p);
     __syncthreads();
-    griddep_wait();     // set-up done; everything below reads what earlier kernels wrote
-    const unsigned epoch = current_epoch(p);
+    const unsigned epoch = epoch_sm;
     if (tid == 0) trace(p, c, kTrStart);
 
     const unsigned in_bytes = (unsigned)(p.H * 2 / p.parts);   // this CTA's piece of a bf16 row
@@ -256,6 +258,7 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
                 for (int u = c; u < p.R * Q; u += p.grid)
                     local_rank_duty(p, u / Q, u % Q, Q, ids_sm, rm, hist, gw, nw, lane, gtid, gn, 1);
             }
+            if (gtid == 0) trace(p, c, kTrScanned);   // deferred outputs written
         } else if (kMode == kModeLocal) {
             // every CTA: bitmaps over the whole routing table -> totals, the rows before its
             // own tokens, and (CTAs with a source-rank duty) that rank's counts
@@ -500,7 +503,6 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
         if (tid == 0) {
             for (int n = max(0, issued - stages); n < issued; ++n)
                 (void)mbar_wait(&full_bar[n % stages], (n / stages) & 1, nullptr);
-            finish_dispatch(p, epoch);
         }
         return;
     }
@@ -512,11 +514,7 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
     // the arrival counters of the next call live in the other half; clear them now
     if (c == 0)
         for (int r = tid; r < p.R; r += kThreads) p.arrival[((epoch + 1) & 1) * p.R + r] = 0;
-    __syncthreads();
-    if (tid == 0) {
-        trace(p, c, kTrEnd);
-        finish_dispatch(p, epoch);
-    }
+    if (tid == 0) trace(p, c, kTrEnd);
 }
 
 // ---------------------------------------------------------------------------- combine
