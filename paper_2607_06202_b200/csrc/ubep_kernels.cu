@@ -237,10 +237,10 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
             stage_small();
             group_sync(2, kThreads);
             if (gtid == 0) trace(p, c, kTrCounted);
-            local_rows_dedup(p, t0, t1, ids_sm, rm, pos_raw, key, row_sm, arr, gtid, gn);
+            local_rows_dedup(p, t0, t1, ids_sm, rm, c, order_sm, pos_raw, key, row_sm, arr, gtid, gn);
             group_sync(1, gn);
             if (gtid == 0) trace(p, c, kTrFinalized);
-            order_destinations(p, c, order_sm, pos_raw, key, pos, ntok * p.k, gtid, gn);
+            order_destinations(p, pos_raw, key, pos, ntok * p.k, gtid, gn);
             group_sync(1, gn);
             if (gtid == 0) {
                 mbar_arrive(&ready_bar);
@@ -289,10 +289,10 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
             finalize_chunk(p, t0, t1, ids, w_sm,
                            [&](int e, int tl) { return eo[e] + pre[e] + bits_in_range(bmaps, e, t0, t0 + tl); },
                            [&](int r, int tl) { return pre[p.E + r] + bits_in_range(bmaps, p.E + r, t0, t0 + tl); },
-                           part == 0, pos_raw, key, arr, gtid, gn);
+                           part == 0, c, order_sm, pos_raw, key, arr, gtid, gn);
             group_sync(1, gn);
             if (gtid == 0) trace(p, c, kTrFinalized);
-            order_destinations(p, c, order_sm, pos_raw, key, pos, ntok * p.k, gtid, gn);
+            order_destinations(p, pos_raw, key, pos, ntok * p.k, gtid, gn);
             group_sync(1, gn);
             if (gtid == 0) {
                 mbar_arrive(&ready_bar);
@@ -372,19 +372,21 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
             }
             if (ok) {
                 // rows before a token = rows of earlier chunks (+ the expert's offset in its
-                // region), published by the prefix-sum step, + earlier tokens of this chunk
+                // region), published by the prefix-sum step, + earlier tokens of this chunk.
+                // The published part is fetched once per bin into shared memory (one round
+                // trip to L2), the rest is bit counting.
                 const int32_t* cb = p.chunk_base + (size_t)ch * p.B;
+                int* base_sm = hist + p.B;   // second half of the scratch (the first may hold scan totals)
+                for (int b = gtid; b < p.B; b += gn)
+                    base_sm[b] = __ldcg(cb + b) + (b < p.E ? __ldcg(p.expert_offset + b) : 0);
+                group_sync(1, gn);
                 finalize_chunk(p, t0, t1, ids, w_sm,
-                               [&](int e, int tl) {
-                                   return __ldcg(p.expert_offset + e) + __ldcg(cb + e) + bits_in_range(bmaps, e, 0, tl);
-                               },
-                               [&](int r, int tl) {
-                                   return __ldcg(cb + p.E + r) + bits_in_range(bmaps, p.E + r, 0, tl);
-                               },
-                               true, pos_raw, key, arr, gtid, gn);
+                               [&](int e, int tl) { return base_sm[e] + bits_in_range(bmaps, e, 0, tl); },
+                               [&](int r, int tl) { return base_sm[p.E + r] + bits_in_range(bmaps, p.E + r, 0, tl); },
+                               true, c, order_sm, pos_raw, key, arr, gtid, gn);
                 group_sync(1, gn);
                 if (gtid == 0) trace(p, c, kTrFinalized);
-                order_destinations(p, c, order_sm, pos_raw, key, pos, ntok * p.k, gtid, gn);
+                order_destinations(p, pos_raw, key, pos, ntok * p.k, gtid, gn);
                 group_sync(1, gn);
             }
             if (gtid == 0) {
@@ -650,7 +652,7 @@ int plan_dispatch(const Params& p, int mode, int max_smem, SmemPlan* out) {
     const int chunk_slots = chunk_tokens * p.k;
     const int map_tokens = mode == kModeLocal ? p.T : chunk_tokens;   // tokens the bitmaps cover
     const int64_t ids_ints = (int64_t)map_tokens * p.k;
-    int hist_ints = mode == kModeLocal ? 2 * p.B + p.E : p.B;
+    int hist_ints = mode == kModeLocal ? 2 * p.B + p.E : 2 * p.B;
     if (hist_ints < 64) hist_ints = 64;   // the per-rank duty of the flag-free kernel keeps 2 x 32 ints here
     pl.map_groups = (map_tokens + 31) / 32;
     pl.map_wb = (p.B + 31) / 32;

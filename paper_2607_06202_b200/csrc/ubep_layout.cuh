@@ -42,6 +42,12 @@ __device__ __forceinline__ int warp_incl_scan(int v, int lane) {
 __device__ __forceinline__ int slot_expert(int v) { return v & 0xffff; }
 __device__ __forceinline__ int slot_rank(int v) { return v >> 16; }
 
+// Place of a rank in the destination-ordering table rotated by the worker id.
+__device__ __forceinline__ int rotated_key(const int* order_sm, int r, int worker, int R) {
+    int kv = order_sm[r] - worker % R;
+    return kv < 0 ? kv + R : kv;
+}
+
 // Resolved expert ids (with their ranks) of tokens [t0, t1) into shared memory.  The raw ids
 // are gathered eight at a time before any of them is resolved, so that the loads overlap.
 __device__ __forceinline__ void stage_ids(const Params& p, int t0, int t1, int* ids, int tid, int nthreads) {
@@ -262,12 +268,15 @@ __device__ void scan_rank_sources(const Params& p, int r, const int* sm, int gti
 // rows precede local token tl in expert e's segment (offset of the segment included) / in
 // rank r's region.  Writes slot_row / slot_pos and the per-row metadata (only when
 // `write_meta`; with column parts one CTA of the group does it) and leaves in pos[] the
-// global row to copy to (rank * cap + row), or -1, and in dst_rank[] that row's rank.
+// global row to copy to (rank * cap + row), or -1, and in dst_key[] the place of that row's
+// rank in the destination-ordering table rotated by the worker id (R for "no copy").
 // arr[r] counts the rows this CTA sends to rank r.  w_sm: the tokens' gate weights, staged.
 template <typename RowsE, typename RowsR>
 __device__ void finalize_chunk(const Params& p, int t0, int t1, const int* ids, const float* w_sm, RowsE rows_e,
-                               RowsR rows_r, bool write_meta, int* pos, int* dst_rank, int* arr, int gtid, int gn) {
-    const int k = p.k, L = p.L;
+                               RowsR rows_r, bool write_meta, int worker, const int* order_sm, int* pos,
+                               int* dst_key, int* arr, int gtid, int gn) {
+    const int k = p.k, L = p.L, R = p.R;
+    const int rot = worker % R;
     const int nslots = (t1 - t0) * k;
     for (int li = gtid; li < nslots; li += gn) {
         const int tl = li / k, j = li - tl * k;
@@ -323,7 +332,12 @@ __device__ void finalize_chunk(const Params& p, int t0, int t1, const int* ids, 
             p.slot_pos[i] = gpos;
         }
         pos[li] = where;
-        dst_rank[li] = r;
+        int kv = R;            // empty slots are issued last
+        if (where >= 0) {
+            kv = order_sm[r] - rot;
+            kv += kv < 0 ? R : 0;
+        }
+        dst_key[li] = kv;
     }
 }
 
@@ -405,7 +419,8 @@ __device__ __forceinline__ int rank_rows_before(const RankMaps& rm, int r, int t
 // (Ordering the destinations with warp shuffles right here instead of in a separate pass
 // was measured slower on the decode shape and is not done.)
 __device__ void local_rows_dedup(const Params& p, int t0, int t1, const int* ids_all, const RankMaps& rm,
-                                 int* pos_raw, int* dst_rank, int* row_sm, int* arr, int gtid, int gn) {
+                                 int worker, const int* order_sm, int* pos_raw, int* dst_key, int* row_sm, int* arr,
+                                 int gtid, int gn) {
     const int k = p.k;
     const int nslots = (t1 - t0) * k;
     for (int li = gtid; li < nslots; li += gn) {
@@ -428,7 +443,7 @@ __device__ void local_rows_dedup(const Params& p, int t0, int t1, const int* ids
             }
         }
         pos_raw[li] = where;
-        dst_rank[li] = r;
+        dst_key[li] = where >= 0 ? rotated_key(order_sm, r, worker, p.R) : p.R;
         row_sm[li] = row;
     }
 }
@@ -529,28 +544,20 @@ __device__ void local_rank_duty(const Params& p, int r, int q, int Q, const int*
 // Per token, put the destinations into the order of the destination-ordering table rotated
 // by the worker id (Sec. 3.3: each worker visits a re-mapped destination sequence).  Only
 // the issue order of the copies changes.  One thread per slot: its place is the number of
-// the token's destinations that come earlier in the rotated table (ties keep slot order);
-// empty slots go last.  Reads pos / dst_rank, writes pos_out.
-__device__ void order_destinations(const Params& p, int worker, const int* order_sm, const int* pos,
-                                   const int* dst_rank, int* pos_out, int nslots, int gtid, int gn) {
-    const int k = p.k, R = p.R;
-    const int rot = worker % R;
+// the token's slots with a smaller key (ties keep slot order).  Reads pos / key, writes pos_out.
+__device__ void order_destinations(const Params& p, const int* pos, const int* key, int* pos_out, int nslots,
+                                   int gtid, int gn) {
+    const int k = p.k;
     for (int li = gtid; li < nslots; li += gn) {
         const int tl = li / k, j = li - tl * k;
-        const int* q = pos + tl * k;
-        const int* rk = dst_rank + tl * k;
-        const int mine = q[j];
-        int kv = order_sm[rk[j]] - rot;
-        kv += kv < 0 ? R : 0;
-        if (mine < 0) kv = R;   // after every real destination
+        const int* kk = key + tl * k;
+        const int kv = kk[j];
         int place = 0;
         for (int jj = 0; jj < k; ++jj) {
-            int ko = order_sm[rk[jj]] - rot;
-            ko += ko < 0 ? R : 0;
-            if (q[jj] < 0) ko = R;
+            const int ko = kk[jj];
             place += (ko < kv || (ko == kv && jj < j)) ? 1 : 0;
         }
-        pos_out[tl * k + place] = mine;
+        pos_out[tl * k + place] = pos[li];
     }
 }
 
