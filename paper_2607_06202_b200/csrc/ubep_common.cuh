@@ -18,6 +18,7 @@ constexpr int kMaxTopk = 32;
 constexpr int kMaxChunks = 320;        // scan keeps chunks/32 values per lane in registers
 constexpr int kMaxStages = 16;         // rows in the shared-memory ring
 constexpr int kRankWordsHost = 4;      // the rank-level fast path handles up to 128 ranks
+constexpr int kStealBlock = 2;         // tokens handed out per claim
 constexpr int kOutStages = 4;          // quantised rows waiting for their bulk stores (FP8)
 constexpr int kTraceSlots = 16;        // per-CTA phase time stamps (optional tracing)
 constexpr int kModePhased = 1, kModeFused = 2, kModeLocal = 3;
@@ -71,6 +72,13 @@ struct Params {
     unsigned* hist_flag;  // [nchunks]
     unsigned* scan_flag;  // [R]
     unsigned* arrival;    // [2, R]
+    // token stealing (large T): chunk c's tokens are handed out in blocks through cursor[c],
+    // to its owner and, once pos_flag[c] holds the epoch, to CTAs that ran out of work
+    int steal;            // 1 = on
+    int32_t* copy_pos;    // [T, k] destinations in issue order (-1 = no copy), for thieves
+    unsigned* cursor;     // [nchunks] tokens of the chunk handed out so far
+    unsigned* pos_flag;   // [nchunks] == epoch: copy_pos of the chunk is final
+    unsigned* claimed;    // [2] tokens handed out in this dispatch (half = epoch & 1)
     int32_t* status;
     unsigned long long* trace;  // optional [nchunks, kTraceSlots] globaltimer stamps, or null
 };
@@ -219,6 +227,7 @@ struct SmemPlan {
     int out_stage_bytes;              // FP8: kOutStages quantised rows
     int map_groups, map_wb, map_bp;   // bin bitmaps: 32-token groups, words of bins, padded bins
     int off_out, off_ids, off_mask, off_bm, off_pos, off_key, off_ord, off_w, off_hist, off_arr, off_order;
+    int off_item;                     // per ring stage: where its token comes from, positions of stolen tokens
     int total;
 };
 

@@ -17,13 +17,15 @@ namespace {
 std::atomic<uint64_t> g_launches{0};
 
 constexpr size_t kAlign = 256;
+constexpr int kStealMinTokensPerChunk = 40;  // shorter slices: the hand-out costs more than the tail it removes (measured)
 constexpr int64_t kLocalMaxSlots = 8192;  // AUTO uses the flag-free kernel up to this many (token, slot) pairs
 inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 
 struct ArenaLayout {
     size_t off[UBEP_VIEW_COUNT_];
-    size_t slot_pos, chunk_hist, partial, chunk_base, trace;
-    size_t flags_begin, hist_flag, scan_flag, status, ticket, epoch_ctr, done_ticket, order_pos, flags_end;
+    size_t slot_pos, copy_pos, chunk_hist, partial, chunk_base, trace;
+    size_t flags_begin, hist_flag, scan_flag, status, ticket, epoch_ctr, done_ticket, cursor, pos_flag, claimed,
+        order_pos, flags_end;
     size_t total;
     int er_cap, nchunks, S, rowB, G, B;
 };
@@ -73,6 +75,7 @@ ArenaLayout make_layout(const ubep_config_t& c, int nchunks) {
     a.off[UBEP_VIEW_NUM_TOKENS_PER_RANK] = take(R * 4);
     a.off[UBEP_VIEW_SLOT_ROW] = take(Tk * 4);
     a.slot_pos = take(Tk * 4);
+    a.copy_pos = take(Tk * 4);
     a.chunk_hist = take(n * B * 4);
     a.partial = take(S * B * 4);
     a.chunk_base = take(n * B * 4);
@@ -85,6 +88,9 @@ ArenaLayout make_layout(const ubep_config_t& c, int nchunks) {
     a.ticket = take(4);
     a.off[UBEP_VIEW_EPOCH] = a.epoch_ctr = take(4);
     a.done_ticket = take(4);
+    a.cursor = take(n * 4);
+    a.pos_flag = take(n * 4);
+    a.claimed = take(8);
     a.flags_end = at;
     a.order_pos = take(R * 4);
     a.total = at;
@@ -151,6 +157,11 @@ Params make_params(ubep_buffer* b, int T) {
     p.num_tokens_per_rank = at<int32_t>(b, a.off[UBEP_VIEW_NUM_TOKENS_PER_RANK]);
     p.slot_row = at<int32_t>(b, a.off[UBEP_VIEW_SLOT_ROW]);
     p.slot_pos = at<int32_t>(b, a.slot_pos);
+    p.copy_pos = at<int32_t>(b, a.copy_pos);
+    p.cursor = at<unsigned>(b, a.cursor);
+    p.pos_flag = at<unsigned>(b, a.pos_flag);
+    p.claimed = at<unsigned>(b, a.claimed);
+    p.steal = 0;
     p.chunk_hist = at<int32_t>(b, a.chunk_hist);
     p.partial = at<int32_t>(b, a.partial);
     p.chunk_base = at<int32_t>(b, a.chunk_base);
@@ -335,6 +346,8 @@ int ubep_dispatch(ubep_buffer_t* buf, const void* x, const int32_t* topk_idx, co
             p.grid = n;
         }
     }
+    // slices that are long enough are handed out in blocks so that faster SMs can take over the tail of slower ones
+    if (mode != UBEP_PIPELINE_LOCAL) p.steal = T >= kStealMinTokensPerChunk * p.nchunks ? 1 : 0;
     if (mode != UBEP_PIPELINE_LOCAL && ubep::plan_dispatch(p, mode, buf->max_smem, &pl) != 0) return UBEP_ERR_ARG;
     cudaError_t e = ubep::launch_dispatch(p, mode, pl, st, &launches);
     if (e != cudaSuccess) return cuda_fail(buf, e);

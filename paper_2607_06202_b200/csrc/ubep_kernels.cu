@@ -77,7 +77,7 @@ __device__ __forceinline__ void quantize8(const uint4 in, bool valid, uint2& out
 // Warp roles: warp 0 = mover (one elected thread issues the TMA loads and, for bf16 rows,
 // the TMA stores); warps 1..15 = layout group (count, prefix sums, row assignment); with
 // FP8 rows warp 1 then becomes the store issuer and warps 2..15 quantise.
-template <int kMode, bool kFp8>
+template <int kMode, bool kFp8, bool kSteal>
 __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, const SmemPlan pl) {
     extern __shared__ __align__(128) uint8_t smem[];
     __shared__ __align__(8) uint64_t full_bar[kMaxStages];    // input row landed
@@ -142,21 +142,100 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
     if (warp == 0) {
         // ------------------------------------------------------------------ mover warp
         // Lane 0 issues the TMA loads; for bf16 rows lane j issues the TMA store of slot j,
-        // so the k copies of a row are issued side by side.
+        // so the k copies of a row are issued side by side.  Tokens come from a feeder: the
+        // CTA's own chunk first and, when stealing is on, blocks of other chunks afterwards.
         bool ok = true;
-        auto issue_load = [&](int n) {
-            const int s = n % stages;
-            mbar_arrive_expect_tx(&full_bar[s], in_bytes);
-            bulk_load(smem + (size_t)s * pl.stage_bytes,
-                      reinterpret_cast<const uint8_t*>(p.x) + (size_t)(t0 + n) * p.H * 2 + in_off, in_bytes,
-                      &full_bar[s]);
+        int v = ch, v_t0 = t0, v_ntok = ntok;   // chunk the feeder currently draws from
+        int blk_lo = 0, blk_hi = 0;             // tokens of that chunk this CTA may take now
+        unsigned pend = 0;                      // lane 0: answer of a claim made ahead of time
+        bool pend_valid = false, feeder_done = false;
+        int scanned = 0;                        // victims looked at so far
+        if (!kSteal) blk_hi = ntok;            // no stealing: the whole chunk, no atomics
+        auto pick_victim = [&]() -> int {
+            while (scanned < p.nchunks - 1) {
+                unsigned done = 0;
+                if (lane == 0) done = __ldcg(p.claimed + (epoch & 1));
+                if ((int)__shfl_sync(0xffffffffu, done, 0) >= p.T) return -1;   // every token is handed out
+                const int idx = scanned + lane;
+                int cand = ch + 1 + idx;
+                if (cand >= p.nchunks) cand -= p.nchunks;
+                int rem = 0;
+                if (idx < p.nchunks - 1 && ld_acquire(p.pos_flag + cand) == epoch) {
+                    const int nt = (int)chunk_begin(cand + 1, p.T, p.nchunks) - (int)chunk_begin(cand, p.T, p.nchunks);
+                    rem = nt - (int)__ldcg(p.cursor + cand);
+                }
+                int best = rem > 0 ? (rem << 9) | cand : 0;   // most remaining tokens first (cand < 512)
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, o));
+                if (best > 0) return best & 511;
+                scanned += 32;
+            }
+            return -1;
         };
+        // Next token of the feeder: its index inside chunk v (warp-uniform).  Returns 1 = token,
+        // 0 = nothing left anywhere, 2 = only other chunks have work and the caller does not
+        // want to take it yet (it still has rows of its own queued).
+        bool v_empty = false;   // chunk v has handed out all its tokens
+        auto next_token = [&](int& tl, bool allow_steal) -> int {
+            while (blk_lo >= blk_hi) {
+                if (feeder_done || !kSteal) { feeder_done = true; return 0; }
+                if (v_empty) {
+                    if (!allow_steal) return 2;
+                    v = pick_victim();
+                    if (v < 0) { feeder_done = true; return 0; }
+                    v_t0 = (int)chunk_begin(v, p.T, p.nchunks);
+                    v_ntok = (int)chunk_begin(v + 1, p.T, p.nchunks) - v_t0;
+                    v_empty = false;
+                    pend_valid = false;
+                }
+                if (v != ch && !allow_steal) return 2;
+                if (!pend_valid && lane == 0) pend = atomicAdd(p.cursor + v, (unsigned)kStealBlock);
+                const int old = (int)__shfl_sync(0xffffffffu, pend, 0);
+                pend_valid = false;
+                if (old < v_ntok) {
+                    blk_lo = old;
+                    blk_hi = min(old + kStealBlock, v_ntok);
+                    if (lane == 0) {
+                        atomicAdd(p.claimed + (epoch & 1), (unsigned)(blk_hi - blk_lo));
+                        pend = atomicAdd(p.cursor + v, (unsigned)kStealBlock);   // answer needed a block later
+                    }
+                    pend_valid = true;
+                } else {
+                    v_empty = true;
+                }
+            }
+            tl = blk_lo++;
+            return 1;
+        };
+        int* item_src = reinterpret_cast<int*>(smem + pl.off_item);           // [stages] (chunk << 16 | index), -1 = end
+        int* item_pos = item_src + kMaxStages + kOutStages;                   // [stages, k] destinations of stolen tokens
+        int head = 0, tail = 0;   // rows whose load was issued / whose copies were issued
+        // load of the feeder's next token into ring stage head % stages
+        auto issue_item = [&](int tl) {
+            const int s = head % stages;
+            if (lane == 0) {
+                if (kSteal) item_src[s] = (v << 16) | tl;
+                mbar_arrive_expect_tx(&full_bar[s], in_bytes);
+                bulk_load(smem + (size_t)s * pl.stage_bytes,
+                          reinterpret_cast<const uint8_t*>(p.x) + (size_t)(v_t0 + tl) * p.H * 2 + in_off, in_bytes,
+                          &full_bar[s]);
+            }
+            if (v != ch)   // a stolen token: its destinations come from the owner's published list
+                for (int j = lane; j < p.k; j += 32)
+                    item_pos[s * p.k + j] = __ldcg(p.copy_pos + (size_t)(v_t0 + tl) * p.k + j);
+            if (kSteal) __syncwarp();
+            ++head;
+        };
+        if (kSteal && lane == 0) p.cursor[ch] = 0;   // before anybody can claim from this chunk
         if (!kFp8) {
             // loads run (stages - 3) rows ahead; up to 3 rows' stores stay in flight
-            const int pf = min(stages - 3, ntok);
-            if (lane == 0)
-                for (int n = 0; n < pf; ++n) issue_load(n);
-            issued = pf;
+            int tl = 0;
+            if (kSteal) {
+                while (head < stages - 3 && next_token(tl, false) == 1) issue_item(tl);
+            } else {
+                while (head < min(stages - 3, ntok)) issue_item(head);
+            }
+            issued = head;
             if (fast_local) {
                 // lend a hand with the routing table, then wait for the layout group
                 const RankMaps rm{bmaps.bm, bmaps.mask_t, (p.R + 31) / 32, ((p.R + 31) / 32) * 32, (p.T + 31) / 32};
@@ -164,46 +243,119 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
                 group_sync(2, kThreads);
             }
             ok = mbar_wait(&ready_bar, 0, abortp) && !*abortp;  // no rows without a layout
-            for (int n = 0; ok && n < ntok; ++n) {
-                const int s = n % stages;
-                ok = mbar_wait(&full_bar[s], (n / stages) & 1, abortp);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!kSteal) {
+                // the CTA's own rows, in order: row n sits in stage n % stages
+                for (int n = 0; ok && n < ntok; ++n) {
+                    const int s = n % stages;
+                    ok = mbar_wait(&full_bar[s], (n / stages) & 1, abortp);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    if (n == 0 && lane == 0) trace(p, c, kTrFirstRow);
+                    const uint8_t* src = smem + (size_t)s * pl.stage_bytes;
+                    for (int j = lane; j < p.k; j += 32) {
+                        const int where = pos[n * p.k + j];
+                        if (where >= 0) bulk_store(p.recv_x + (size_t)where * p.rowB + out_off, src, out_bytes);
+                    }
+                    bulk_commit();
+                    if (head < ntok) {
+                        bulk_wait_read<3>();     // every lane: its copies of the row 3 back have read the stage
+                        __syncwarp();
+                        issue_item(head);        // without stealing a row's index in the chunk is its sequence number
+                        issued = head;
+                    }
+                }
+            }
+            while (kSteal && ok) {
+                if (tail == head) {
+                    // nothing queued: take over rows of another chunk, or finish
+                    if (feeder_done || next_token(tl, true) != 1) break;
+                    issue_item(tl);
+                    issued = head;
+                }
+                const int s = tail % stages;
+                ok = mbar_wait(&full_bar[s], (tail / stages) & 1, abortp);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                if (n == 0 && lane == 0) trace(p, c, kTrFirstRow);
+                if (tail == 0 && lane == 0) trace(p, c, kTrFirstRow);
                 const uint8_t* src = smem + (size_t)s * pl.stage_bytes;
+                const int from = kSteal ? item_src[s] : ((ch << 16) | tail);   // without stealing: own rows in order
+                const bool own = (from >> 16) == ch;
                 for (int j = lane; j < p.k; j += 32) {
-                    const int where = pos[n * p.k + j];
-                    if (where >= 0) bulk_store(p.recv_x + (size_t)where * p.rowB + out_off, src, out_bytes);
+                    const int where = own ? pos[(from & 0xffff) * p.k + j] : item_pos[s * p.k + j];
+                    if (where >= 0) {
+                        bulk_store(p.recv_x + (size_t)where * p.rowB + out_off, src, out_bytes);
+                        if (kSteal) atomicAdd(&arr[where / p.cap], 1);   // rows per rank: counted by whoever copies
+                    }
                 }
                 bulk_commit();
-                if (issued < ntok) {
+                ++tail;
+                if (!feeder_done && head - tail < stages - 3) {
                     bulk_wait_read<3>();     // every lane: its copies of the row 3 back have read the stage
                     __syncwarp();
-                    if (lane == 0) issue_load(issued);
-                    ++issued;
+                    // own rows first, then rows of other chunks, all loaded as far ahead as the ring allows
+                    if (next_token(tl, true) == 1) issue_item(tl);
+                    issued = head;
                 }
             }
         } else {
             if (fast_local) {
                 const RankMaps rm{bmaps.bm, bmaps.mask_t, (p.R + 31) / 32, ((p.R + 31) / 32) * 32, (p.T + 31) / 32};
-                if (lane == 0)
-                    for (; issued < min(stages, ntok); ++issued) issue_load(issued);
-                issued = __shfl_sync(0xffffffffu, issued, 0);
+                int tl = 0;
+                while (head < stages && next_token(tl, false) == 1) issue_item(tl);
+                issued = head;
                 local_stage_and_rank_maps(p, ids_sm, rm, 0, kWarps, lane);
                 group_sync(2, kThreads);
             }
-            // loader only (lane 0); the quantising warps free the stages
-            if (lane == 0) {
-                for (int n = issued; ok && n < ntok; ++n) {
-                    const int s = n % stages;
-                    if (n >= stages) ok = mbar_wait(&empty_bar[s], ((n / stages) - 1) & 1, abortp);
-                    if (!ok) break;
-                    issue_load(n);
-                    issued = n + 1;
+            // loader only; the quantising warps free the stages.  A closing item with no row
+            // tells them (and through them the store issuer) that nothing follows.
+            int tl = 0;
+            if (!kSteal) {
+                // the CTA's own rows only: one thread, as far ahead as the ring allows
+                while (ok && head < ntok) {
+                    if (head >= stages) {
+                        if (lane == 0) ok = mbar_wait(&empty_bar[head % stages], ((head / stages) - 1) & 1, abortp);
+                        ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+                        if (!ok) break;
+                    }
+                    tl = head;
+                    issue_item(tl);
+                    issued = head;
                 }
             }
-            issued = __shfl_sync(0xffffffffu, issued, 0);
-            ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+            while (kSteal && ok) {
+                // rows of other chunks are taken only once all but two queued rows are consumed
+                bool drained = head < 3;
+                if (!drained) {
+                    const int hs = head - 3;
+                    drained = mbar_test_wait(&empty_bar[hs % stages], (hs / stages) & 1);
+                    drained = __all_sync(0xffffffffu, drained);
+                }
+                const int got = feeder_done ? 0 : next_token(tl, drained);
+                if (got == 2) {
+                    const int hs = head - 3;   // wait for the queue to drain, then ask again
+                    ok = mbar_wait(&empty_bar[hs % stages], (hs / stages) & 1, abortp);
+                    ok = __all_sync(0xffffffffu, ok);
+                    continue;
+                }
+                const int s = head % stages;
+                if (got == 0 && !kSteal) break;
+                if (head >= stages) {
+                    ok = mbar_wait(&empty_bar[s], ((head / stages) - 1) & 1, abortp);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                }
+                if (got == 1) {
+                    issue_item(tl);
+                    issued = head;
+                } else {
+                    if (kSteal && lane == 0) {   // without stealing the consumers know the row count
+                        item_src[s] = -1;
+                        mbar_arrive(&full_bar[s]);
+                    }
+                    break;
+                }
+            }
         }
         if (!ok && lane == 0) {
             report(p.status, kErrTimeout);  // a wait gave up: record it and let everybody leave
@@ -383,7 +535,7 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
                 finalize_chunk(p, t0, t1, ids, w_sm,
                                [&](int e, int tl) { return base_sm[e] + bits_in_range(bmaps, e, 0, tl); },
                                [&](int r, int tl) { return base_sm[p.E + r] + bits_in_range(bmaps, p.E + r, 0, tl); },
-                               true, c, order_sm, pos_raw, key, arr, gtid, gn);
+                               true, c, order_sm, pos_raw, key, kSteal ? nullptr : arr, gtid, gn);
                 group_sync(1, gn);
                 if (gtid == 0) trace(p, c, kTrFinalized);
                 order_destinations(p, pos_raw, key, pos, ntok * p.k, gtid, gn);
@@ -393,6 +545,15 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
                 mbar_arrive(&ready_bar);
                 trace(p, c, kTrReady);
             }
+            if (ok && kSteal) {
+                // this chunk's destinations, for CTAs that run out of work and take over some of its tokens
+                for (int i = gtid; i < ntok * p.k; i += gn) p.copy_pos[(size_t)t0 * p.k + i] = pos[i];
+                group_sync(1, gn);
+                if (gtid == 0) {
+                    __threadfence();
+                    st_release(p.pos_flag + ch, epoch);
+                }
+            }
             if (ok && deferred >= 0) scan_rank_sources(p, deferred, hist, gtid, gn);
         }
         if (kFp8 && ok) {
@@ -400,28 +561,34 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
             const int g0 = part * (p.G / p.parts);                      // first scale group of this CTA's piece
             const unsigned scale_bytes = (unsigned)(p.G / p.parts) * 4u;  // its scales travel with the payload
             const bool scale_bulk = (scale_bytes & 15u) == 0;             // when a bulk copy can carry them
+            const int* item_src = reinterpret_cast<const int*>(smem + pl.off_item);
+            const int* item_pos = item_src + kMaxStages + kOutStages;
+            int* out_src = reinterpret_cast<int*>(smem + pl.off_item) + kMaxStages;   // [kOutStages] 0 = row, -1 = end
+            int* out_pos = out_src + kOutStages + kMaxStages * p.k;                    // [kOutStages, k]
             if (warp == 1) {
                 // ------------------------------ store issuer: lane j issues the copy of slot j
                 bool sok = true;
                 unsigned long long w_full = 0, w_read = 0, tq = 0;
-                for (int n = 0; n < ntok; ++n) {
+                for (int n = 0; kSteal || n < ntok; ++n) {
                     const int os = n % kOutStages;
                     if (p.trace) tq = global_ns();
                     sok = mbar_wait(&out_full[os], (n / kOutStages) & 1, abortp);
                     if (p.trace) w_full += global_ns() - tq;
                     sok = __all_sync(0xffffffffu, sok);
-                    if (!sok) break;
+                    if (!sok || (kSteal && out_src[os] < 0)) break;
                     if (n == 0 && lane == 0) trace(p, c, kTrFirstRow);
                     const uint8_t* src = out_ring + (size_t)os * pl.out_stage_bytes;
                     // lanes 0..k-1: payload of slot j; lanes k..2k-1: its scales (when bulk-storable)
                     for (int j = lane; j < (scale_bulk ? 2 * p.k : p.k); j += 32) {
                         const int jj = j < p.k ? j : j - p.k;
-                        const int where = pos[n * p.k + jj];
+                        const int where = kSteal ? out_pos[os * p.k + jj] : pos[n * p.k + jj];
                         if (where < 0) continue;
-                        if (j < p.k)
+                        if (j < p.k) {
                             bulk_store(p.recv_x + (size_t)where * p.rowB + out_off, src, out_bytes);
-                        else
+                            if (kSteal) atomicAdd(&arr[where / p.cap], 1);
+                        } else {
                             bulk_store(p.recv_scale + (size_t)where * p.G + g0, src + out_bytes, scale_bytes);
+                        }
                     }
                     bulk_commit();
                     if (n + 1 >= kOutStages) {
@@ -446,13 +613,27 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
                 const int qw = warp - 2;
                 const int nvec = (int)in_bytes / 16;          // 8-channel vectors in this CTA's piece
                 unsigned long long w_in = 0, w_out = 0, t_cmp = 0, tq = 0;
-                for (int n = 0; n < ntok; ++n) {
+                for (int n = 0; kSteal || n < ntok; ++n) {
                     const int s = n % stages, os = n % kOutStages;
                     if (p.trace) tq = global_ns();
                     if (!mbar_wait(&full_bar[s], (n / stages) & 1, abortp)) break;
                     if (p.trace) { unsigned long long t2 = global_ns(); w_in += t2 - tq; tq = t2; }
                     if (n >= kOutStages && !mbar_wait(&out_empty[os], ((n / kOutStages) - 1) & 1, abortp)) break;
                     if (p.trace) { unsigned long long t2 = global_ns(); w_out += t2 - tq; tq = t2; }
+                    const int from = kSteal ? item_src[s] : ((ch << 16) | n);
+                    if (from < 0) {
+                        // the loader's closing item: pass it on to the store issuer and leave
+                        if (qw == 0 && lane == 0) out_src[os] = -1;
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&out_full[os]);
+                        break;
+                    }
+                    const bool own = (from >> 16) == ch;
+                    const int* wpos = own ? pos + (from & 0xffff) * p.k : item_pos + s * p.k;   // this row's destinations
+                    if (kSteal && qw == 0) {
+                        for (int j = lane; j < p.k; j += 32) out_pos[os * p.k + j] = wpos[j];
+                        if (lane == 0) out_src[os] = 0;
+                    }
                     const uint8_t* src = smem + (size_t)s * pl.stage_bytes;
                     uint8_t* dst = out_ring + (size_t)os * pl.out_stage_bytes;
                     float* dst_scale = reinterpret_cast<float*>(dst + out_bytes);
@@ -475,7 +656,7 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
                                 if (ok1) dst_scale[v1 >> 4] = sc1;
                             } else {
                                 for (int j = 0; j < p.k; ++j) {
-                                    const int where = pos[n * p.k + j];
+                                    const int where = wpos[j];
                                     if (where < 0) continue;
                                     if (ok0) p.recv_scale[(size_t)where * p.G + g0 + (v0 >> 4)] = sc0;
                                     if (ok1) p.recv_scale[(size_t)where * p.G + g0 + (v1 >> 4)] = sc1;
@@ -514,8 +695,10 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
     for (int r = tid; r < p.R; r += kThreads)
         if (arr[r]) red_release_add(p.arrival + (epoch & 1) * p.R + r, (unsigned)(arr[r] * (8 / p.parts)));
     // the arrival counters of the next call live in the other half; clear them now
-    if (c == 0)
+    if (c == 0) {
         for (int r = tid; r < p.R; r += kThreads) p.arrival[((epoch + 1) & 1) * p.R + r] = 0;
+        if (tid == 0) p.claimed[(epoch + 1) & 1] = 0;   // same for the count of tokens handed out
+    }
     if (tid == 0) trace(p, c, kTrEnd);
 }
 
@@ -661,7 +844,8 @@ int plan_dispatch(const Params& p, int mode, int max_smem, SmemPlan* out) {
     pl.out_stage_bytes = p.payload ? round_up_i(p.rowB / p.parts + (p.G / p.parts) * 4, 128) : 0;
     const int64_t mask_ints = (int64_t)pl.map_groups * 32;
     const int64_t bm_ints = (int64_t)pl.map_groups * pl.map_bp;
-    const int64_t ints = ids_ints + mask_ints + bm_ints + 4 * (int64_t)chunk_slots + hist_ints + 2 * p.R;
+    const int item_ints = (kMaxStages + kOutStages) * (p.k + 1);
+    const int64_t ints = ids_ints + mask_ints + bm_ints + 4 * (int64_t)chunk_slots + hist_ints + 2 * p.R + item_ints;
     const int64_t fixed = (int64_t)kOutStages * pl.out_stage_bytes + ints * 4 + 128 + 1024;  // 1 KB: static smem
     if (fixed + 4 * (int64_t)pl.stage_bytes > max_smem) return -1;
     pl.stages = (int)((max_smem - fixed) / pl.stage_bytes);
@@ -683,6 +867,7 @@ int plan_dispatch(const Params& p, int mode, int max_smem, SmemPlan* out) {
     pl.off_hist = at; at += hist_ints * 4;
     pl.off_arr = at; at += p.R * 4;
     pl.off_order = at; at += p.R * 4;
+    pl.off_item = at; at += item_ints * 4;
     pl.total = round_up_i(at, 128);
     *out = pl;
     return 0;
@@ -706,12 +891,18 @@ static cudaError_t launch_overlapped(void (*kern)(KArgs...), int grid, int block
     return cudaLaunchKernelEx(&cfg, kern, args...);
 }
 
-template <int kMode, bool kFp8>
-static cudaError_t launch_dispatch_t(const Params& p, const SmemPlan& pl, cudaStream_t st) {
-    auto kern = dispatch_kernel<kMode, kFp8>;
+template <int kMode, bool kFp8, bool kSteal>
+static cudaError_t launch_dispatch_s(const Params& p, const SmemPlan& pl, cudaStream_t st) {
+    auto kern = dispatch_kernel<kMode, kFp8, kSteal>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.total);
     if (e != cudaSuccess) return e;
     return launch_overlapped(kern, p.grid, kThreads, (size_t)pl.total, st, p, pl);
+}
+
+template <int kMode, bool kFp8>
+static cudaError_t launch_dispatch_t(const Params& p, const SmemPlan& pl, cudaStream_t st) {
+    if (kMode != kModeLocal && p.steal) return launch_dispatch_s<kMode, kFp8, true>(p, pl, st);
+    return launch_dispatch_s<kMode, kFp8, false>(p, pl, st);
 }
 
 cudaError_t launch_dispatch(const Params& p, int mode, const SmemPlan& pl, cudaStream_t st, int* launches) {

@@ -270,7 +270,7 @@ __device__ void scan_rank_sources(const Params& p, int r, const int* sm, int gti
 // `write_meta`; with column parts one CTA of the group does it) and leaves in pos[] the
 // global row to copy to (rank * cap + row), or -1, and in dst_key[] the place of that row's
 // rank in the destination-ordering table rotated by the worker id (R for "no copy").
-// arr[r] counts the rows this CTA sends to rank r.  w_sm: the tokens' gate weights, staged.
+// w_sm: the tokens' gate weights, staged.  (Rows per rank are counted by whoever copies them.)
 template <typename RowsE, typename RowsR>
 __device__ void finalize_chunk(const Params& p, int t0, int t1, const int* ids, const float* w_sm, RowsE rows_e,
                                RowsR rows_r, bool write_meta, int worker, const int* order_sm, int* pos,
@@ -308,7 +308,7 @@ __device__ void finalize_chunk(const Params& p, int t0, int t1, const int* ids, 
                 gpos = r * p.cap + row;
                 if (first) {
                     where = gpos;
-                    atomicAdd(&arr[r], 1);
+                    if (arr) atomicAdd(&arr[r], 1);   // rows this CTA will copy to rank r (null: counted at copy time)
                     if (write_meta) {
                         p.recv_src_idx[where] = t;
                         if (!p.dedup) {
