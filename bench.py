@@ -201,6 +201,8 @@ def run_ours(args, cfg, rank: int, world: int, local_rank: int):
         w = torch.from_numpy(wl.topk_w).to(dev)
         if wl.phys is not None:
             buf.set_replicas(torch.from_numpy(wl.phys).to(dev), torch.from_numpy(wl.ncopies).to(dev))
+        if args.quant_warps:
+            B.ubep_debug_set_quant_warps(buf.handle, args.quant_warps)
         y = torch.from_numpy(y_bits).view(torch.bfloat16).to(dev)
         out = torch.empty((cfg.T, cfg.H), dtype=torch.bfloat16, device=dev)
         return dict(buf=buf, x=x, idx=idx, w=w, y=y, out=out)
@@ -419,6 +421,7 @@ def main():
     ap.add_argument("--workload", default="decode")
     ap.add_argument("--pipeline", type=int, default=0)
     ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--quant-warps", type=int, default=0, help="FP8 dispatch: warps that quantise (role-split sweep)")
     ap.add_argument("--profile", action="store_true",
                     help="plain launches of the timed steps only (for ncu): no graph, no e2e, no CPU leg")
     args = ap.parse_args()

@@ -249,6 +249,14 @@ int ubep_debug_withhold_flag(ubep_buffer_t *buf, int32_t chunk);
  */
 int ubep_debug_trace(ubep_buffer_t *buf, int32_t enable);
 
+/*
+ * Warp-role split of the FP8 dispatch kernel (the paper's core-allocation question, Sec. 3.2
+ * and App. A / C: how many cores count and how many send): n of the CTA's 16 warps quantise
+ * rows (1 <= n <= 14, default 14); one warp loads, one issues the stores, the rest idle once
+ * the layout is done.  Results never depend on it.
+ */
+int ubep_debug_set_quant_warps(ubep_buffer_t *buf, int32_t n);
+
 /* Text of the last CUDA runtime error seen by this buffer's calls ("" if none). */
 const char *ubep_last_cuda_error(const ubep_buffer_t *buf);
 

@@ -75,6 +75,7 @@ struct Params {
     // token stealing (large T): chunk c's tokens are handed out in blocks through cursor[c],
     // to its owner and, once pos_flag[c] holds the epoch, to CTAs that ran out of work
     int steal;            // 1 = on
+    int quant_warps;      // FP8: warps that quantise (2 .. kWarps - 2); the others idle after the layout
     int32_t* copy_pos;    // [T, k] destinations in issue order (-1 = no copy), for thieves
     unsigned* cursor;     // [nchunks] tokens of the chunk handed out so far
     unsigned* pos_flag;   // [nchunks] == epoch: copy_pos of the chunk is final

@@ -108,6 +108,7 @@ struct ubep_buffer {
     uint32_t epoch;
     int32_t withhold;
     int32_t tracing;
+    int32_t quant_warps;
     cudaStream_t last_stream;
     const int32_t* phys;
     const int32_t* ncopies;
@@ -162,6 +163,7 @@ Params make_params(ubep_buffer* b, int T) {
     p.pos_flag = at<unsigned>(b, a.pos_flag);
     p.claimed = at<unsigned>(b, a.claimed);
     p.steal = 0;
+    p.quant_warps = b->quant_warps;
     p.chunk_hist = at<int32_t>(b, a.chunk_hist);
     p.partial = at<int32_t>(b, a.partial);
     p.chunk_base = at<int32_t>(b, a.chunk_base);
@@ -221,6 +223,7 @@ int ubep_buffer_create(const ubep_config_t* cfg, void* dev_arena, size_t bytes, 
     b->epoch = 0;
     b->withhold = -1;
     b->tracing = 0;
+    b->quant_warps = ubep::kWarps - 2;
     b->last_stream = nullptr;
     b->phys = nullptr;
     b->ncopies = nullptr;
@@ -439,6 +442,12 @@ int ubep_debug_withhold_flag(ubep_buffer_t* buf, int32_t chunk) {
 int ubep_debug_trace(ubep_buffer_t* buf, int32_t enable) {
     if (!buf) return UBEP_ERR_ARG;
     buf->tracing = enable != 0;
+    return UBEP_OK;
+}
+
+int ubep_debug_set_quant_warps(ubep_buffer_t* buf, int32_t n) {
+    if (!buf || n < 1 || n > ubep::kWarps - 2) return UBEP_ERR_ARG;
+    buf->quant_warps = n;
     return UBEP_OK;
 }
 

@@ -111,7 +111,7 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
 
     constexpr int gn = kThreads - 32;  // layout group: warps 1..15
     constexpr int nw = kWarps - 1;
-    constexpr int nq = kWarps - 2;     // FP8: quantising warps 2..15
+    const int nq = kFp8 ? p.quant_warps : kWarps - 2;   // FP8: warps 2 .. nq + 1 quantise
     const int gtid = tid - 32, gw = warp - 1;
 
     if (tid == 0) {
@@ -608,8 +608,8 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
                     p.trace[(size_t)c * kTraceSlots + 14] = w_full;
                     p.trace[(size_t)c * kTraceSlots + 15] = w_read;
                 }
-            } else {
-                // ------------------------------------------------- quantising warps 2..15
+            } else if (warp - 2 < nq) {
+                // ------------------------------------------------- quantising warps 2 .. nq + 1
                 const int qw = warp - 2;
                 const int nvec = (int)in_bytes / 16;          // 8-channel vectors in this CTA's piece
                 unsigned long long w_in = 0, w_out = 0, t_cmp = 0, tq = 0;

@@ -265,6 +265,20 @@ def test_fp8_special_values_match_the_oracle():
     Hn.run_case(wl, pipeline=FUSED)
 
 
+@pytest.mark.parametrize("n", [1, 3, 8])
+def test_warp_role_split_does_not_change_results(n):
+    cfg = small(600, 1024, 32, 8, 4, payload=1, seed=33)
+    wl = W.make_workload(cfg)
+    ids, lay, cap, recv = Hn.oracle_reference(wl)
+    buf = Hn.make_buffer(cfg, cap, pipeline=FUSED)
+    B.ubep_debug_set_quant_warps(buf.handle, n)
+    x, idx, w, _, _ = Hn.device_inputs(wl)
+    buf.dispatch(x, idx, w)
+    Hn.check_dispatch(buf, wl, lay, cap, recv)
+    with pytest.raises(B.UbepError):
+        B.ubep_debug_set_quant_warps(buf.handle, 15)
+
+
 def test_bounded_wait_reports_timeout_and_the_context_survives():
     """A readiness flag that nobody publishes: the waits run out, the kernel returns, the
     status word says so, and the next dispatch on the same buffer is correct again."""
