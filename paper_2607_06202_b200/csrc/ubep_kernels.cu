@@ -73,10 +73,619 @@ __device__ __forceinline__ void quantize8(const uint4 in, bool valid, uint2& out
     out.y = q[2] | (q[3] << 16);
 }
 
+
+// Everything the roles of one dispatch CTA share.
+struct Cta {
+    const Params& p;
+    const SmemPlan& pl;
+    uint8_t* smem;
+    uint64_t *full_bar, *empty_bar, *out_full, *out_empty, *ready_bar;
+    int* abort_flag;
+    int tid, lane, warp, c, part, ch, t0, t1, ntok, stages, nq;
+    int *ids_sm, *pos, *pos_raw, *key;
+    float* w_sm;
+    BinMaps bmaps;
+    int *hist, *arr, *order_sm;
+    unsigned epoch, in_bytes, out_bytes;
+    size_t in_off, out_off;
+    bool fast_local;
+    int issued;   // rows whose load the mover has started (thread 0's copy is used when leaving early)
+};
+
+// The role functions below keep the names the kernel uses for these.
+#define UBEP_CTA_LOCALS(x)                                                                                   \
+    [[maybe_unused]] const Params& p = (x).p;                                                                \
+    [[maybe_unused]] const SmemPlan& pl = (x).pl;                                                            \
+    [[maybe_unused]] uint8_t* const smem = (x).smem;                                                         \
+    [[maybe_unused]] uint64_t* const full_bar = (x).full_bar;                                                \
+    [[maybe_unused]] uint64_t* const empty_bar = (x).empty_bar;                                              \
+    [[maybe_unused]] uint64_t* const out_full = (x).out_full;                                                \
+    [[maybe_unused]] uint64_t* const out_empty = (x).out_empty;                                              \
+    [[maybe_unused]] uint64_t& ready_bar = *(x).ready_bar;                                                   \
+    [[maybe_unused]] int& abort_flag = *(x).abort_flag;                                                      \
+    [[maybe_unused]] volatile int* const abortp = (x).abort_flag;                                            \
+    [[maybe_unused]] const int tid = (x).tid, lane = (x).lane, warp = (x).warp, c = (x).c;                   \
+    [[maybe_unused]] const int part = (x).part, ch = (x).ch, t0 = (x).t0, t1 = (x).t1, ntok = (x).ntok;     \
+    [[maybe_unused]] const int stages = (x).stages, nq = (x).nq;                                             \
+    [[maybe_unused]] int* const ids_sm = (x).ids_sm;                                                         \
+    [[maybe_unused]] int* const pos = (x).pos;                                                               \
+    [[maybe_unused]] int* const pos_raw = (x).pos_raw;                                                       \
+    [[maybe_unused]] int* const key = (x).key;                                                               \
+    [[maybe_unused]] float* const w_sm = (x).w_sm;                                                           \
+    [[maybe_unused]] const BinMaps& bmaps = (x).bmaps;                                                       \
+    [[maybe_unused]] int* const hist = (x).hist;                                                             \
+    [[maybe_unused]] int* const arr = (x).arr;                                                               \
+    [[maybe_unused]] int* const order_sm = (x).order_sm;                                                     \
+    [[maybe_unused]] const unsigned epoch = (x).epoch, in_bytes = (x).in_bytes, out_bytes = (x).out_bytes;   \
+    [[maybe_unused]] const size_t in_off = (x).in_off, out_off = (x).out_off;                                \
+    [[maybe_unused]] const bool fast_local = (x).fast_local;                                                 \
+    [[maybe_unused]] int& issued = (x).issued;                                                               \
+    [[maybe_unused]] constexpr int gn = kThreads - 32; /* layout group: warps 1..15 */                       \
+    [[maybe_unused]] constexpr int nw = kWarps - 1;                                                          \
+    [[maybe_unused]] const int gtid = (x).tid - 32, gw = (x).warp - 1
+
+// ------------------------------------------------------------------------ mover warp
+// Warp 0.  Lane 0 issues the TMA loads; for bf16 rows lane j issues the TMA store of slot j,
+// so the k copies of a row are issued side by side; for FP8 rows the warp only loads.
+template <int kMode, bool kFp8, bool kSteal>
+__device__ __forceinline__ void mover_warp(Cta& x) {
+    UBEP_CTA_LOCALS(x);
+    // Lane 0 issues the TMA loads; for bf16 rows lane j issues the TMA store of slot j,
+    // so the k copies of a row are issued side by side.  Tokens come from a feeder: the
+    // CTA's own chunk first and, when stealing is on, blocks of other chunks afterwards.
+    bool ok = true;
+    int v = ch, v_t0 = t0, v_ntok = ntok;   // chunk the feeder currently draws from
+    int blk_lo = 0, blk_hi = 0;             // tokens of that chunk this CTA may take now
+    unsigned pend = 0;                      // lane 0: answer of a claim made ahead of time
+    bool pend_valid = false, feeder_done = false;
+    int scanned = 0;                        // victims looked at so far
+    if (!kSteal) blk_hi = ntok;            // no stealing: the whole chunk, no atomics
+    auto pick_victim = [&]() -> int {
+        while (scanned < p.nchunks - 1) {
+            unsigned done = 0;
+            if (lane == 0) done = __ldcg(p.claimed + (epoch & 1));
+            if ((int)__shfl_sync(0xffffffffu, done, 0) >= p.T) return -1;   // every token is handed out
+            const int idx = scanned + lane;
+            int cand = ch + 1 + idx;
+            if (cand >= p.nchunks) cand -= p.nchunks;
+            int rem = 0;
+            if (idx < p.nchunks - 1 && ld_acquire(p.pos_flag + cand) == epoch) {
+                const int nt = (int)chunk_begin(cand + 1, p.T, p.nchunks) - (int)chunk_begin(cand, p.T, p.nchunks);
+                rem = nt - (int)__ldcg(p.cursor + cand);
+            }
+            int best = rem > 0 ? (rem << 9) | cand : 0;   // most remaining tokens first (cand < 512)
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, o));
+            if (best > 0) return best & 511;
+            scanned += 32;
+        }
+        return -1;
+    };
+    // Next token of the feeder: its index inside chunk v (warp-uniform).  Returns 1 = token,
+    // 0 = nothing left anywhere, 2 = only other chunks have work and the caller does not
+    // want to take it yet (it still has rows of its own queued).
+    bool v_empty = false;   // chunk v has handed out all its tokens
+    auto next_token = [&](int& tl, bool allow_steal) -> int {
+        while (blk_lo >= blk_hi) {
+            if (feeder_done || !kSteal) { feeder_done = true; return 0; }
+            if (v_empty) {
+                if (!allow_steal) return 2;
+                v = pick_victim();
+                if (v < 0) { feeder_done = true; return 0; }
+                v_t0 = (int)chunk_begin(v, p.T, p.nchunks);
+                v_ntok = (int)chunk_begin(v + 1, p.T, p.nchunks) - v_t0;
+                v_empty = false;
+                pend_valid = false;
+            }
+            if (v != ch && !allow_steal) return 2;
+            if (!pend_valid && lane == 0) pend = atomicAdd(p.cursor + v, (unsigned)kStealBlock);
+            const int old = (int)__shfl_sync(0xffffffffu, pend, 0);
+            pend_valid = false;
+            if (old < v_ntok) {
+                blk_lo = old;
+                blk_hi = min(old + kStealBlock, v_ntok);
+                if (lane == 0) {
+                    atomicAdd(p.claimed + (epoch & 1), (unsigned)(blk_hi - blk_lo));
+                    pend = atomicAdd(p.cursor + v, (unsigned)kStealBlock);   // answer needed a block later
+                }
+                pend_valid = true;
+            } else {
+                v_empty = true;
+            }
+        }
+        tl = blk_lo++;
+        return 1;
+    };
+    int* item_src = reinterpret_cast<int*>(smem + pl.off_item);           // [stages] (chunk << 16 | index), -1 = end
+    int* item_pos = item_src + kMaxStages + kOutStages;                   // [stages, k] destinations of stolen tokens
+    int head = 0, tail = 0;   // rows whose load was issued / whose copies were issued
+    // load of the feeder's next token into ring stage head % stages
+    auto issue_item = [&](int tl) {
+        const int s = head % stages;
+        if (lane == 0) {
+            if (kSteal) item_src[s] = (v << 16) | tl;
+            mbar_arrive_expect_tx(&full_bar[s], in_bytes);
+            bulk_load(smem + (size_t)s * pl.stage_bytes,
+                      reinterpret_cast<const uint8_t*>(p.x) + (size_t)(v_t0 + tl) * p.H * 2 + in_off, in_bytes,
+                      &full_bar[s]);
+        }
+        if (v != ch)   // a stolen token: its destinations come from the owner's published list
+            for (int j = lane; j < p.k; j += 32)
+                item_pos[s * p.k + j] = __ldcg(p.copy_pos + (size_t)(v_t0 + tl) * p.k + j);
+        if (kSteal) __syncwarp();
+        ++head;
+    };
+    if (kSteal && lane == 0) p.cursor[ch] = 0;   // before anybody can claim from this chunk
+    if (!kFp8) {
+        // loads run (stages - 3) rows ahead; up to 3 rows' stores stay in flight
+        int tl = 0;
+        if (kSteal) {
+            while (head < stages - 3 && next_token(tl, false) == 1) issue_item(tl);
+        } else {
+            while (head < min(stages - 3, ntok)) issue_item(head);
+        }
+        issued = head;
+        if (fast_local) {
+            // lend a hand with the routing table, then wait for the layout group
+            const RankMaps rm{bmaps.bm, bmaps.mask_t, (p.R + 31) / 32, ((p.R + 31) / 32) * 32, (p.T + 31) / 32};
+            local_stage_and_rank_maps(p, ids_sm, rm, 0, kWarps, lane);
+            group_sync(2, kThreads);
+        }
+        ok = mbar_wait(&ready_bar, 0, abortp) && !*abortp;  // no rows without a layout
+        ok = __all_sync(0xffffffffu, ok);
+        if (!kSteal) {
+            // the CTA's own rows, in order: row n sits in stage n % stages
+            for (int n = 0; ok && n < ntok; ++n) {
+                const int s = n % stages;
+                ok = mbar_wait(&full_bar[s], (n / stages) & 1, abortp);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                if (n == 0 && lane == 0) trace(p, c, kTrFirstRow);
+                const uint8_t* src = smem + (size_t)s * pl.stage_bytes;
+                for (int j = lane; j < p.k; j += 32) {
+                    const int where = pos[n * p.k + j];
+                    if (where >= 0) bulk_store(p.recv_x + (size_t)where * p.rowB + out_off, src, out_bytes);
+                }
+                bulk_commit();
+                if (head < ntok) {
+                    bulk_wait_read<3>();     // every lane: its copies of the row 3 back have read the stage
+                    __syncwarp();
+                    issue_item(head);        // without stealing a row's index in the chunk is its sequence number
+                    issued = head;
+                }
+            }
+        }
+        while (kSteal && ok) {
+            if (tail == head) {
+                // nothing queued: take over rows of another chunk, or finish
+                if (feeder_done || next_token(tl, true) != 1) break;
+                issue_item(tl);
+                issued = head;
+            }
+            const int s = tail % stages;
+            ok = mbar_wait(&full_bar[s], (tail / stages) & 1, abortp);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            if (tail == 0 && lane == 0) trace(p, c, kTrFirstRow);
+            const uint8_t* src = smem + (size_t)s * pl.stage_bytes;
+            const int from = kSteal ? item_src[s] : ((ch << 16) | tail);   // without stealing: own rows in order
+            const bool own = (from >> 16) == ch;
+            for (int j = lane; j < p.k; j += 32) {
+                const int where = own ? pos[(from & 0xffff) * p.k + j] : item_pos[s * p.k + j];
+                if (where >= 0) {
+                    bulk_store(p.recv_x + (size_t)where * p.rowB + out_off, src, out_bytes);
+                    if (kSteal) atomicAdd(&arr[where / p.cap], 1);   // rows per rank: counted by whoever copies
+                }
+            }
+            bulk_commit();
+            ++tail;
+            if (!feeder_done && head - tail < stages - 3) {
+                bulk_wait_read<3>();     // every lane: its copies of the row 3 back have read the stage
+                __syncwarp();
+                // own rows first, then rows of other chunks, all loaded as far ahead as the ring allows
+                if (next_token(tl, true) == 1) issue_item(tl);
+                issued = head;
+            }
+        }
+    } else {
+        if (fast_local) {
+            const RankMaps rm{bmaps.bm, bmaps.mask_t, (p.R + 31) / 32, ((p.R + 31) / 32) * 32, (p.T + 31) / 32};
+            int tl = 0;
+            while (head < stages && next_token(tl, false) == 1) issue_item(tl);
+            issued = head;
+            local_stage_and_rank_maps(p, ids_sm, rm, 0, kWarps, lane);
+            group_sync(2, kThreads);
+        }
+        // loader only; the quantising warps free the stages.  A closing item with no row
+        // tells them (and through them the store issuer) that nothing follows.
+        int tl = 0;
+        if (!kSteal) {
+            // the CTA's own rows only: one thread, as far ahead as the ring allows
+            while (ok && head < ntok) {
+                if (head >= stages) {
+                    if (lane == 0) ok = mbar_wait(&empty_bar[head % stages], ((head / stages) - 1) & 1, abortp);
+                    ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+                    if (!ok) break;
+                }
+                tl = head;
+                issue_item(tl);
+                issued = head;
+            }
+        }
+        while (kSteal && ok) {
+            // rows of other chunks are taken only once all but two queued rows are consumed
+            bool drained = head < 3;
+            if (!drained) {
+                const int hs = head - 3;
+                drained = mbar_test_wait(&empty_bar[hs % stages], (hs / stages) & 1);
+                drained = __all_sync(0xffffffffu, drained);
+            }
+            const int got = feeder_done ? 0 : next_token(tl, drained);
+            if (got == 2) {
+                const int hs = head - 3;   // wait for the queue to drain, then ask again
+                ok = mbar_wait(&empty_bar[hs % stages], (hs / stages) & 1, abortp);
+                ok = __all_sync(0xffffffffu, ok);
+                continue;
+            }
+            const int s = head % stages;
+            if (got == 0 && !kSteal) break;
+            if (head >= stages) {
+                ok = mbar_wait(&empty_bar[s], ((head / stages) - 1) & 1, abortp);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+            }
+            if (got == 1) {
+                issue_item(tl);
+                issued = head;
+            } else {
+                if (kSteal && lane == 0) {   // without stealing the consumers know the row count
+                    item_src[s] = -1;
+                    mbar_arrive(&full_bar[s]);
+                }
+                break;
+            }
+        }
+    }
+    if (!ok && lane == 0) {
+        report(p.status, kErrTimeout);  // a wait gave up: record it and let everybody leave
+        abort_flag = 1;
+    }
+    if (lane == 0) trace(p, c, kTrIssued);
+    bulk_wait_all<0>();
+    if (lane == 0) trace(p, c, kTrStored);
+}
+
+// ---------------------------------------------------------------------- layout group
+// Warps 1..15: TokenCnt, CalCumSum (by exchange or alone), slot -> row assignment; releases
+// the movers and then writes what nobody inside the kernel waits for.  Returns false if a
+// wait ran out.
+template <int kMode, bool kFp8, bool kSteal>
+__device__ __forceinline__ bool layout_group(Cta& x) {
+    UBEP_CTA_LOCALS(x);
+    bool ok = true;
+    const int* ids = ids_sm;  // staged slots of this CTA's tokens
+    // Small global reads whose values are needed only after the first barriers: issue the
+    // loads now (first trip of each loop), store to shared memory after the ids are staged.
+    const int order_r = gtid < p.R ? __ldg(p.order_pos + gtid) : 0;
+    const bool stage_w = !(kMode == kModeLocal && p.local_fast);
+    const float w_first = (stage_w && gtid < ntok * p.k) ? __ldg(p.topk_w + (size_t)t0 * p.k + gtid) : 0.0f;
+    auto stage_small = [&]() {
+        if (gtid < p.R) order_sm[gtid] = order_r;
+        for (int r = gtid + gn; r < p.R; r += gn) order_sm[r] = __ldg(p.order_pos + r);
+        if (stage_w) {
+            if (gtid < ntok * p.k) w_sm[gtid] = w_first;
+            for (int i = gtid + gn; i < ntok * p.k; i += gn) w_sm[i] = __ldg(p.topk_w + (size_t)t0 * p.k + i);
+        }
+    };
+    if (kMode == kModeLocal && p.local_fast) {
+        // rank-level rows first, movers released, expert-level outputs afterwards
+        const RankMaps rm{bmaps.bm, bmaps.mask_t, (p.R + 31) / 32, ((p.R + 31) / 32) * 32, (p.T + 31) / 32};
+        int* row_sm = reinterpret_cast<int*>(w_sm);
+        local_stage_and_rank_maps(p, ids_sm, rm, warp, kWarps, lane);   // with the mover warp
+        stage_small();
+        group_sync(2, kThreads);
+        if (gtid == 0) trace(p, c, kTrCounted);
+        local_rows_dedup(p, t0, t1, ids_sm, rm, c, order_sm, pos_raw, key, row_sm, arr, gtid, gn);
+        group_sync(1, gn);
+        if (gtid == 0) trace(p, c, kTrFinalized);
+        order_destinations(p, pos_raw, key, pos, ntok * p.k, gtid, gn);
+        group_sync(1, gn);
+        if (gtid == 0) {
+            mbar_arrive(&ready_bar);
+            trace(p, c, kTrReady);
+        }
+        if (part == 0) {
+            float* w_own = reinterpret_cast<float*>(key);   // the ordering keys are no longer needed
+            for (int i = gtid; i < ntok * p.k; i += gn) w_own[i] = __ldg(p.topk_w + (size_t)t0 * p.k + i);
+        }
+        group_sync(1, gn);
+        if (part == 0) local_meta_dedup(p, t0, t1, ids_sm, pos_raw, row_sm, reinterpret_cast<float*>(key), gtid, gn);
+        {
+            // expert-level outputs of rank r: shared by Q CTAs so that no CTA trails the others
+            const int Q = p.grid / p.R > 1 ? p.grid / p.R : 1;
+            for (int u = c; u < p.R * Q; u += p.grid)
+                local_rank_duty(p, u / Q, u % Q, Q, ids_sm, rm, hist, gw, nw, lane, gtid, gn, 1);
+        }
+        if (gtid == 0) trace(p, c, kTrScanned);   // deferred outputs written
+    } else if (kMode == kModeLocal) {
+        // every CTA: bitmaps over the whole routing table -> totals, the rows before its
+        // own tokens, and (CTAs with a source-rank duty) that rank's counts
+        int* tot = hist;
+        int* pre = hist + p.B;
+        int* eo = hist + 2 * p.B;
+        stage_ids(p, 0, p.T, ids_sm, gtid, gn);
+        stage_small();
+        group_sync(1, gn);
+        if (gtid == 0) trace(p, c, kTrCounted);
+        build_bin_maps(p, ids_sm, p.T, bmaps, gw, nw, lane);
+        group_sync(1, gn);
+        if (gtid == 0) trace(p, c, kTrHistSeen);
+        for (int b = gtid; b < p.B; b += gn) {
+            const int before = bits_in_range(bmaps, b, 0, t0);
+            pre[b] = before;
+            tot[b] = before + bits_in_range(bmaps, b, t0, p.T);
+        }
+        group_sync(1, gn);
+        for (int e = gtid; e < p.E; e += gn) {
+            int o = 0;
+            for (int q = (e / p.L) * p.L; q < e; ++q) o += tot[q];
+            eo[e] = o;
+        }
+        group_sync(1, gn);
+        if (gtid == 0) trace(p, c, kTrScanSeen);
+        ids = ids_sm + (size_t)t0 * p.k;
+        finalize_chunk(p, t0, t1, ids, w_sm,
+                       [&](int e, int tl) { return eo[e] + pre[e] + bits_in_range(bmaps, e, t0, t0 + tl); },
+                       [&](int r, int tl) { return pre[p.E + r] + bits_in_range(bmaps, p.E + r, t0, t0 + tl); },
+                       part == 0, c, order_sm, pos_raw, key, arr, gtid, gn);
+        group_sync(1, gn);
+        if (gtid == 0) trace(p, c, kTrFinalized);
+        order_destinations(p, pos_raw, key, pos, ntok * p.k, gtid, gn);
+        group_sync(1, gn);
+        if (gtid == 0) {
+            mbar_arrive(&ready_bar);
+            trace(p, c, kTrReady);
+        }
+        // outputs nobody inside this kernel waits for
+        if (c == 0) {
+            for (int e = gtid; e < p.E; e += gn) {
+                p.expert_offset[e] = eo[e];
+                p.num_tokens_per_expert[e] = tot[e];
+            }
+            for (int r = gtid; r < p.R; r += gn) {
+                p.num_tokens_per_rank[r] = tot[p.E + r];
+                int rows = tot[p.E + r];
+                if (!p.dedup) {
+                    rows = 0;
+                    for (int q = r * p.L; q < (r + 1) * p.L; ++q) rows += tot[q];
+                }
+                p.num_rows_per_rank[r] = rows;
+            }
+        }
+        if (part == 0)
+            for (int s = ch; s < p.S; s += p.nchunks) {   // source ranks this CTA reports
+                const int b0 = src_begin(s, p.T, p.S), b1 = src_begin(s + 1, p.T, p.S);
+                for (int e = gtid; e < p.E; e += gn) {
+                    p.cnt[(size_t)s * p.E + e] = bits_in_range(bmaps, e, b0, b1);
+                    p.src_offset[(size_t)s * p.E + e] = eo[e] + bits_in_range(bmaps, e, 0, b0);
+                }
+            }
+    } else {
+        stage_ids(p, t0, t1, ids_sm, gtid, gn);
+        stage_small();
+        group_sync(1, gn);
+        build_bin_maps(p, ids_sm, ntok, bmaps, gw, nw, lane);
+        group_sync(1, gn);
+        int deferred = -1;
+        if (kMode == kModeFused) {
+            publish_chunk_counts(p, ch, t0, t1, bmaps, gtid, gn);
+            group_sync(1, gn);
+            if (gtid == 0) {
+                if (ch != p.withhold) {
+                    __threadfence();
+                    st_release(p.hist_flag + ch, epoch);
+                }
+                trace(p, c, kTrCounted);
+            }
+            // CalCumSum duty: this CTA serves rank ch (and ch + nchunks, ...)
+            bool lost = false;  // a wait of this thread ran out
+            for (int r = ch; r < p.R; r += p.nchunks) {
+                for (int cc = gtid; cc < p.nchunks; cc += gn)
+                    if (!wait_flag(p.hist_flag + cc, epoch, abortp)) lost = true;
+                if (group_or(1, gn, lost || *abortp)) { lost = true; break; }  // same answer for all
+                if (gtid == 0) trace(p, c, kTrHistSeen);
+                scan_rank_publish(p, r, hist, gw, nw, lane, 1);
+                if (gtid == 0) {
+                    __threadfence();
+                    st_release(p.scan_flag + r, epoch);
+                    trace(p, c, kTrScanned);
+                }
+                if (r + p.nchunks < p.R) {
+                    scan_rank_sources(p, r, hist, gtid, gn);
+                    group_sync(1, gn);
+                } else {
+                    deferred = r;   // cnt / src_offset: after our own movers are released
+                }
+            }
+            // every slot of this chunk may need any rank's bases
+            if (!lost)
+                for (int r = gtid; r < p.R; r += gn)
+                    if (!wait_flag(p.scan_flag + r, epoch, abortp)) lost = true;
+            ok = !group_or(1, gn, lost || *abortp);
+            if (gtid == 0) trace(p, c, kTrScanSeen);
+            if (!ok && gtid == 0) {
+                report(p.status, kErrTimeout);
+                abort_flag = 1;
+            }
+        }
+        if (ok) {
+            // rows before a token = rows of earlier chunks (+ the expert's offset in its
+            // region), published by the prefix-sum step, + earlier tokens of this chunk.
+            // The published part is fetched once per bin into shared memory (one round
+            // trip to L2), the rest is bit counting.
+            const int32_t* cb = p.chunk_base + (size_t)ch * p.B;
+            int* base_sm = hist + p.B;   // second half of the scratch (the first may hold scan totals)
+            for (int b = gtid; b < p.B; b += gn)
+                base_sm[b] = __ldcg(cb + b) + (b < p.E ? __ldcg(p.expert_offset + b) : 0);
+            group_sync(1, gn);
+            finalize_chunk(p, t0, t1, ids, w_sm,
+                           [&](int e, int tl) { return base_sm[e] + bits_in_range(bmaps, e, 0, tl); },
+                           [&](int r, int tl) { return base_sm[p.E + r] + bits_in_range(bmaps, p.E + r, 0, tl); },
+                           true, c, order_sm, pos_raw, key, kSteal ? nullptr : arr, gtid, gn);
+            group_sync(1, gn);
+            if (gtid == 0) trace(p, c, kTrFinalized);
+            order_destinations(p, pos_raw, key, pos, ntok * p.k, gtid, gn);
+            group_sync(1, gn);
+        }
+        if (gtid == 0) {
+            mbar_arrive(&ready_bar);
+            trace(p, c, kTrReady);
+        }
+        if (ok && kSteal) {
+            // this chunk's destinations, for CTAs that run out of work and take over some of its tokens
+            for (int i = gtid; i < ntok * p.k; i += gn) p.copy_pos[(size_t)t0 * p.k + i] = pos[i];
+            group_sync(1, gn);
+            if (gtid == 0) {
+                __threadfence();
+                st_release(p.pos_flag + ch, epoch);
+            }
+        }
+        if (ok && deferred >= 0) scan_rank_sources(p, deferred, hist, gtid, gn);
+    }
+    return ok;
+}
+
+// ------------------------------------------------------------ FP8: quantise and store
+// After the layout: warp 1 issues the stores, warps 2 .. nq + 1 quantise.
+template <bool kSteal>
+__device__ __forceinline__ void fp8_consumers(Cta& x) {
+    UBEP_CTA_LOCALS(x);
+    uint8_t* out_ring = smem + pl.off_out;
+    const int g0 = part * (p.G / p.parts);                      // first scale group of this CTA's piece
+    const unsigned scale_bytes = (unsigned)(p.G / p.parts) * 4u;  // its scales travel with the payload
+    const bool scale_bulk = (scale_bytes & 15u) == 0;             // when a bulk copy can carry them
+    const int* item_src = reinterpret_cast<const int*>(smem + pl.off_item);
+    const int* item_pos = item_src + kMaxStages + kOutStages;
+    int* out_src = reinterpret_cast<int*>(smem + pl.off_item) + kMaxStages;   // [kOutStages] 0 = row, -1 = end
+    int* out_pos = out_src + kOutStages + kMaxStages * p.k;                    // [kOutStages, k]
+    if (warp == 1) {
+        // ------------------------------ store issuer: lane j issues the copy of slot j
+        bool sok = true;
+        unsigned long long w_full = 0, w_read = 0, tq = 0;
+        for (int n = 0; kSteal || n < ntok; ++n) {
+            const int os = n % kOutStages;
+            if (p.trace) tq = global_ns();
+            sok = mbar_wait(&out_full[os], (n / kOutStages) & 1, abortp);
+            if (p.trace) w_full += global_ns() - tq;
+            sok = __all_sync(0xffffffffu, sok);
+            if (!sok || (kSteal && out_src[os] < 0)) break;
+            if (n == 0 && lane == 0) trace(p, c, kTrFirstRow);
+            const uint8_t* src = out_ring + (size_t)os * pl.out_stage_bytes;
+            // lanes 0..k-1: payload of slot j; lanes k..2k-1: its scales (when bulk-storable)
+            for (int j = lane; j < (scale_bulk ? 2 * p.k : p.k); j += 32) {
+                const int jj = j < p.k ? j : j - p.k;
+                const int where = kSteal ? out_pos[os * p.k + jj] : pos[n * p.k + jj];
+                if (where < 0) continue;
+                if (j < p.k) {
+                    bulk_store(p.recv_x + (size_t)where * p.rowB + out_off, src, out_bytes);
+                    if (kSteal) atomicAdd(&arr[where / p.cap], 1);
+                } else {
+                    bulk_store(p.recv_scale + (size_t)where * p.G + g0, src + out_bytes, scale_bytes);
+                }
+            }
+            bulk_commit();
+            if (n + 1 >= kOutStages) {
+                if (p.trace) tq = global_ns();
+                bulk_wait_read<kOutStages - 1>();   // every lane: the oldest row's copies have read it
+                if (p.trace) w_read += global_ns() - tq;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&out_empty[(n + 1) % kOutStages]);
+            }
+        }
+        if (!sok && lane == 0) {
+            report(p.status, kErrTimeout);
+            abort_flag = 1;
+        }
+        bulk_wait_all<0>();
+        if (p.trace && lane == 0) {
+            p.trace[(size_t)c * kTraceSlots + 14] = w_full;
+            p.trace[(size_t)c * kTraceSlots + 15] = w_read;
+        }
+    } else if (warp - 2 < nq) {
+        // ------------------------------------------------- quantising warps 2 .. nq + 1
+        const int qw = warp - 2;
+        const int nvec = (int)in_bytes / 16;          // 8-channel vectors in this CTA's piece
+        unsigned long long w_in = 0, w_out = 0, t_cmp = 0, tq = 0;
+        for (int n = 0; kSteal || n < ntok; ++n) {
+            const int s = n % stages, os = n % kOutStages;
+            if (p.trace) tq = global_ns();
+            if (!mbar_wait(&full_bar[s], (n / stages) & 1, abortp)) break;
+            if (p.trace) { unsigned long long t2 = global_ns(); w_in += t2 - tq; tq = t2; }
+            if (n >= kOutStages && !mbar_wait(&out_empty[os], ((n / kOutStages) - 1) & 1, abortp)) break;
+            if (p.trace) { unsigned long long t2 = global_ns(); w_out += t2 - tq; tq = t2; }
+            const int from = kSteal ? item_src[s] : ((ch << 16) | n);
+            if (from < 0) {
+                // the loader's closing item: pass it on to the store issuer and leave
+                if (qw == 0 && lane == 0) out_src[os] = -1;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&out_full[os]);
+                break;
+            }
+            const bool own = (from >> 16) == ch;
+            const int* wpos = own ? pos + (from & 0xffff) * p.k : item_pos + s * p.k;   // this row's destinations
+            if (kSteal && qw == 0) {
+                for (int j = lane; j < p.k; j += 32) out_pos[os * p.k + j] = wpos[j];
+                if (lane == 0) out_src[os] = 0;
+            }
+            const uint8_t* src = smem + (size_t)s * pl.stage_bytes;
+            uint8_t* dst = out_ring + (size_t)os * pl.out_stage_bytes;
+            float* dst_scale = reinterpret_cast<float*>(dst + out_bytes);
+            // two vectors per thread and trip, independent of each other
+            for (int vb = qw * 32; vb < nvec; vb += 2 * nq * 32) {
+                const int v0 = vb + lane, v1 = v0 + nq * 32;
+                const bool ok0 = v0 < nvec, ok1 = v1 < nvec;
+                uint4 in0 = make_uint4(0, 0, 0, 0), in1 = make_uint4(0, 0, 0, 0);
+                if (ok0) in0 = *reinterpret_cast<const uint4*>(src + (size_t)v0 * 16);
+                if (ok1) in1 = *reinterpret_cast<const uint4*>(src + (size_t)v1 * 16);
+                uint2 q0, q1;
+                float sc0, sc1;
+                quantize8(in0, ok0, q0, sc0);
+                quantize8(in1, ok1, q1, sc1);
+                if (ok0) *reinterpret_cast<uint2*>(dst + (size_t)v0 * 8) = q0;
+                if (ok1) *reinterpret_cast<uint2*>(dst + (size_t)v1 * 8) = q1;
+                if ((lane & 15) == 0) {
+                    if (scale_bulk) {
+                        if (ok0) dst_scale[v0 >> 4] = sc0;
+                        if (ok1) dst_scale[v1 >> 4] = sc1;
+                    } else {
+                        for (int j = 0; j < p.k; ++j) {
+                            const int where = wpos[j];
+                            if (where < 0) continue;
+                            if (ok0) p.recv_scale[(size_t)where * p.G + g0 + (v0 >> 4)] = sc0;
+                            if (ok1) p.recv_scale[(size_t)where * p.G + g0 + (v1 >> 4)] = sc1;
+                        }
+                    }
+                }
+            }
+            fence_proxy_async_smem();   // the bulk stores read what we just wrote
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(&out_full[os]);
+                mbar_arrive(&empty_bar[s]);
+            }
+            if (p.trace) t_cmp += global_ns() - tq;
+        }
+        if (p.trace && warp == 2 && lane == 0) {
+            p.trace[(size_t)c * kTraceSlots + 11] = w_in;
+            p.trace[(size_t)c * kTraceSlots + 12] = w_out;
+            p.trace[(size_t)c * kTraceSlots + 13] = t_cmp;
+        }
+    }
+}
+
 // --------------------------------------------------------------------- dispatch kernel
-// Warp roles: warp 0 = mover (one elected thread issues the TMA loads and, for bf16 rows,
-// the TMA stores); warps 1..15 = layout group (count, prefix sums, row assignment); with
-// FP8 rows warp 1 then becomes the store issuer and warps 2..15 quantise.
+// Warp roles: warp 0 = mover; warps 1..15 = layout group (count, prefix sums, row
+// assignment); with FP8 rows warp 1 then becomes the store issuer and warps 2..15 quantise.
 template <int kMode, bool kFp8, bool kSteal>
 __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, const SmemPlan pl) {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -88,31 +697,14 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
     __shared__ int abort_flag;
     __shared__ unsigned epoch_sm;
 
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x;
     const int c = blockIdx.x;
     const int part = c % p.parts, ch = c / p.parts;
     const int t0 = (int)chunk_begin(ch, p.T, p.nchunks), t1 = (int)chunk_begin(ch + 1, p.T, p.nchunks);
-    const int ntok = t1 - t0;
     const int stages = pl.stages;
-    int* ids_sm = reinterpret_cast<int*>(smem + pl.off_ids);
-    int* pos = reinterpret_cast<int*>(smem + pl.off_ord);     // destinations in issue order
-    int* pos_raw = reinterpret_cast<int*>(smem + pl.off_pos);  // destinations in slot order
-    int* key = reinterpret_cast<int*>(smem + pl.off_key);
-    float* w_sm = reinterpret_cast<float*>(smem + pl.off_w);
-    const BinMaps bmaps{reinterpret_cast<unsigned*>(smem + pl.off_mask),
-                        reinterpret_cast<unsigned*>(smem + pl.off_bm), pl.map_wb, pl.map_bp,
-                        pl.map_groups};
-    int* hist = reinterpret_cast<int*>(smem + pl.off_hist);
-    int* arr = reinterpret_cast<int*>(smem + pl.off_arr);
-    int* order_sm = reinterpret_cast<int*>(smem + pl.off_order);
-    volatile int* abortp = &abort_flag;
-    int issued = 0;  // rows whose load thread 0 has started
-    griddep_launch();   // the next kernel in the stream may be placed as soon as SMs have room
-
-    constexpr int gn = kThreads - 32;  // layout group: warps 1..15
-    constexpr int nw = kWarps - 1;
     const int nq = kFp8 ? p.quant_warps : kWarps - 2;   // FP8: warps 2 .. nq + 1 quantise
-    const int gtid = tid - 32, gw = warp - 1;
+    int* arr = reinterpret_cast<int*>(smem + pl.off_arr);
+    griddep_launch();   // the next kernel in the stream may be placed as soon as SMs have room
 
     if (tid == 0) {
         for (int s = 0; s < stages; ++s) {
@@ -136,555 +728,30 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
 
     const unsigned in_bytes = (unsigned)(p.H * 2 / p.parts);   // this CTA's piece of a bf16 row
     const unsigned out_bytes = (unsigned)(p.rowB / p.parts);   // and of a payload row
-    const size_t in_off = (size_t)part * in_bytes, out_off = (size_t)part * out_bytes;
+    Cta x{p, pl, smem, full_bar, empty_bar, out_full, out_empty, &ready_bar, &abort_flag,
+          tid, tid & 31, tid >> 5, c, part, ch, t0, t1, t1 - t0, stages, nq,
+          reinterpret_cast<int*>(smem + pl.off_ids),
+          reinterpret_cast<int*>(smem + pl.off_ord),    // destinations in issue order
+          reinterpret_cast<int*>(smem + pl.off_pos),    // destinations in slot order
+          reinterpret_cast<int*>(smem + pl.off_key),
+          reinterpret_cast<float*>(smem + pl.off_w),
+          BinMaps{reinterpret_cast<unsigned*>(smem + pl.off_mask), reinterpret_cast<unsigned*>(smem + pl.off_bm),
+                  pl.map_wb, pl.map_bp, pl.map_groups},
+          reinterpret_cast<int*>(smem + pl.off_hist), arr, reinterpret_cast<int*>(smem + pl.off_order),
+          epoch, in_bytes, out_bytes, (size_t)part * in_bytes, (size_t)part * out_bytes,
+          kMode == kModeLocal && p.local_fast != 0, 0};
 
-    const bool fast_local = kMode == kModeLocal && p.local_fast;
-    if (warp == 0) {
-        // ------------------------------------------------------------------ mover warp
-        // Lane 0 issues the TMA loads; for bf16 rows lane j issues the TMA store of slot j,
-        // so the k copies of a row are issued side by side.  Tokens come from a feeder: the
-        // CTA's own chunk first and, when stealing is on, blocks of other chunks afterwards.
-        bool ok = true;
-        int v = ch, v_t0 = t0, v_ntok = ntok;   // chunk the feeder currently draws from
-        int blk_lo = 0, blk_hi = 0;             // tokens of that chunk this CTA may take now
-        unsigned pend = 0;                      // lane 0: answer of a claim made ahead of time
-        bool pend_valid = false, feeder_done = false;
-        int scanned = 0;                        // victims looked at so far
-        if (!kSteal) blk_hi = ntok;            // no stealing: the whole chunk, no atomics
-        auto pick_victim = [&]() -> int {
-            while (scanned < p.nchunks - 1) {
-                unsigned done = 0;
-                if (lane == 0) done = __ldcg(p.claimed + (epoch & 1));
-                if ((int)__shfl_sync(0xffffffffu, done, 0) >= p.T) return -1;   // every token is handed out
-                const int idx = scanned + lane;
-                int cand = ch + 1 + idx;
-                if (cand >= p.nchunks) cand -= p.nchunks;
-                int rem = 0;
-                if (idx < p.nchunks - 1 && ld_acquire(p.pos_flag + cand) == epoch) {
-                    const int nt = (int)chunk_begin(cand + 1, p.T, p.nchunks) - (int)chunk_begin(cand, p.T, p.nchunks);
-                    rem = nt - (int)__ldcg(p.cursor + cand);
-                }
-                int best = rem > 0 ? (rem << 9) | cand : 0;   // most remaining tokens first (cand < 512)
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, o));
-                if (best > 0) return best & 511;
-                scanned += 32;
-            }
-            return -1;
-        };
-        // Next token of the feeder: its index inside chunk v (warp-uniform).  Returns 1 = token,
-        // 0 = nothing left anywhere, 2 = only other chunks have work and the caller does not
-        // want to take it yet (it still has rows of its own queued).
-        bool v_empty = false;   // chunk v has handed out all its tokens
-        auto next_token = [&](int& tl, bool allow_steal) -> int {
-            while (blk_lo >= blk_hi) {
-                if (feeder_done || !kSteal) { feeder_done = true; return 0; }
-                if (v_empty) {
-                    if (!allow_steal) return 2;
-                    v = pick_victim();
-                    if (v < 0) { feeder_done = true; return 0; }
-                    v_t0 = (int)chunk_begin(v, p.T, p.nchunks);
-                    v_ntok = (int)chunk_begin(v + 1, p.T, p.nchunks) - v_t0;
-                    v_empty = false;
-                    pend_valid = false;
-                }
-                if (v != ch && !allow_steal) return 2;
-                if (!pend_valid && lane == 0) pend = atomicAdd(p.cursor + v, (unsigned)kStealBlock);
-                const int old = (int)__shfl_sync(0xffffffffu, pend, 0);
-                pend_valid = false;
-                if (old < v_ntok) {
-                    blk_lo = old;
-                    blk_hi = min(old + kStealBlock, v_ntok);
-                    if (lane == 0) {
-                        atomicAdd(p.claimed + (epoch & 1), (unsigned)(blk_hi - blk_lo));
-                        pend = atomicAdd(p.cursor + v, (unsigned)kStealBlock);   // answer needed a block later
-                    }
-                    pend_valid = true;
-                } else {
-                    v_empty = true;
-                }
-            }
-            tl = blk_lo++;
-            return 1;
-        };
-        int* item_src = reinterpret_cast<int*>(smem + pl.off_item);           // [stages] (chunk << 16 | index), -1 = end
-        int* item_pos = item_src + kMaxStages + kOutStages;                   // [stages, k] destinations of stolen tokens
-        int head = 0, tail = 0;   // rows whose load was issued / whose copies were issued
-        // load of the feeder's next token into ring stage head % stages
-        auto issue_item = [&](int tl) {
-            const int s = head % stages;
-            if (lane == 0) {
-                if (kSteal) item_src[s] = (v << 16) | tl;
-                mbar_arrive_expect_tx(&full_bar[s], in_bytes);
-                bulk_load(smem + (size_t)s * pl.stage_bytes,
-                          reinterpret_cast<const uint8_t*>(p.x) + (size_t)(v_t0 + tl) * p.H * 2 + in_off, in_bytes,
-                          &full_bar[s]);
-            }
-            if (v != ch)   // a stolen token: its destinations come from the owner's published list
-                for (int j = lane; j < p.k; j += 32)
-                    item_pos[s * p.k + j] = __ldcg(p.copy_pos + (size_t)(v_t0 + tl) * p.k + j);
-            if (kSteal) __syncwarp();
-            ++head;
-        };
-        if (kSteal && lane == 0) p.cursor[ch] = 0;   // before anybody can claim from this chunk
-        if (!kFp8) {
-            // loads run (stages - 3) rows ahead; up to 3 rows' stores stay in flight
-            int tl = 0;
-            if (kSteal) {
-                while (head < stages - 3 && next_token(tl, false) == 1) issue_item(tl);
-            } else {
-                while (head < min(stages - 3, ntok)) issue_item(head);
-            }
-            issued = head;
-            if (fast_local) {
-                // lend a hand with the routing table, then wait for the layout group
-                const RankMaps rm{bmaps.bm, bmaps.mask_t, (p.R + 31) / 32, ((p.R + 31) / 32) * 32, (p.T + 31) / 32};
-                local_stage_and_rank_maps(p, ids_sm, rm, 0, kWarps, lane);
-                group_sync(2, kThreads);
-            }
-            ok = mbar_wait(&ready_bar, 0, abortp) && !*abortp;  // no rows without a layout
-            ok = __all_sync(0xffffffffu, ok);
-            if (!kSteal) {
-                // the CTA's own rows, in order: row n sits in stage n % stages
-                for (int n = 0; ok && n < ntok; ++n) {
-                    const int s = n % stages;
-                    ok = mbar_wait(&full_bar[s], (n / stages) & 1, abortp);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                    if (n == 0 && lane == 0) trace(p, c, kTrFirstRow);
-                    const uint8_t* src = smem + (size_t)s * pl.stage_bytes;
-                    for (int j = lane; j < p.k; j += 32) {
-                        const int where = pos[n * p.k + j];
-                        if (where >= 0) bulk_store(p.recv_x + (size_t)where * p.rowB + out_off, src, out_bytes);
-                    }
-                    bulk_commit();
-                    if (head < ntok) {
-                        bulk_wait_read<3>();     // every lane: its copies of the row 3 back have read the stage
-                        __syncwarp();
-                        issue_item(head);        // without stealing a row's index in the chunk is its sequence number
-                        issued = head;
-                    }
-                }
-            }
-            while (kSteal && ok) {
-                if (tail == head) {
-                    // nothing queued: take over rows of another chunk, or finish
-                    if (feeder_done || next_token(tl, true) != 1) break;
-                    issue_item(tl);
-                    issued = head;
-                }
-                const int s = tail % stages;
-                ok = mbar_wait(&full_bar[s], (tail / stages) & 1, abortp);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                if (tail == 0 && lane == 0) trace(p, c, kTrFirstRow);
-                const uint8_t* src = smem + (size_t)s * pl.stage_bytes;
-                const int from = kSteal ? item_src[s] : ((ch << 16) | tail);   // without stealing: own rows in order
-                const bool own = (from >> 16) == ch;
-                for (int j = lane; j < p.k; j += 32) {
-                    const int where = own ? pos[(from & 0xffff) * p.k + j] : item_pos[s * p.k + j];
-                    if (where >= 0) {
-                        bulk_store(p.recv_x + (size_t)where * p.rowB + out_off, src, out_bytes);
-                        if (kSteal) atomicAdd(&arr[where / p.cap], 1);   // rows per rank: counted by whoever copies
-                    }
-                }
-                bulk_commit();
-                ++tail;
-                if (!feeder_done && head - tail < stages - 3) {
-                    bulk_wait_read<3>();     // every lane: its copies of the row 3 back have read the stage
-                    __syncwarp();
-                    // own rows first, then rows of other chunks, all loaded as far ahead as the ring allows
-                    if (next_token(tl, true) == 1) issue_item(tl);
-                    issued = head;
-                }
-            }
-        } else {
-            if (fast_local) {
-                const RankMaps rm{bmaps.bm, bmaps.mask_t, (p.R + 31) / 32, ((p.R + 31) / 32) * 32, (p.T + 31) / 32};
-                int tl = 0;
-                while (head < stages && next_token(tl, false) == 1) issue_item(tl);
-                issued = head;
-                local_stage_and_rank_maps(p, ids_sm, rm, 0, kWarps, lane);
-                group_sync(2, kThreads);
-            }
-            // loader only; the quantising warps free the stages.  A closing item with no row
-            // tells them (and through them the store issuer) that nothing follows.
-            int tl = 0;
-            if (!kSteal) {
-                // the CTA's own rows only: one thread, as far ahead as the ring allows
-                while (ok && head < ntok) {
-                    if (head >= stages) {
-                        if (lane == 0) ok = mbar_wait(&empty_bar[head % stages], ((head / stages) - 1) & 1, abortp);
-                        ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-                        if (!ok) break;
-                    }
-                    tl = head;
-                    issue_item(tl);
-                    issued = head;
-                }
-            }
-            while (kSteal && ok) {
-                // rows of other chunks are taken only once all but two queued rows are consumed
-                bool drained = head < 3;
-                if (!drained) {
-                    const int hs = head - 3;
-                    drained = mbar_test_wait(&empty_bar[hs % stages], (hs / stages) & 1);
-                    drained = __all_sync(0xffffffffu, drained);
-                }
-                const int got = feeder_done ? 0 : next_token(tl, drained);
-                if (got == 2) {
-                    const int hs = head - 3;   // wait for the queue to drain, then ask again
-                    ok = mbar_wait(&empty_bar[hs % stages], (hs / stages) & 1, abortp);
-                    ok = __all_sync(0xffffffffu, ok);
-                    continue;
-                }
-                const int s = head % stages;
-                if (got == 0 && !kSteal) break;
-                if (head >= stages) {
-                    ok = mbar_wait(&empty_bar[s], ((head / stages) - 1) & 1, abortp);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                }
-                if (got == 1) {
-                    issue_item(tl);
-                    issued = head;
-                } else {
-                    if (kSteal && lane == 0) {   // without stealing the consumers know the row count
-                        item_src[s] = -1;
-                        mbar_arrive(&full_bar[s]);
-                    }
-                    break;
-                }
-            }
-        }
-        if (!ok && lane == 0) {
-            report(p.status, kErrTimeout);  // a wait gave up: record it and let everybody leave
-            abort_flag = 1;
-        }
-        if (lane == 0) trace(p, c, kTrIssued);
-        bulk_wait_all<0>();
-        if (lane == 0) trace(p, c, kTrStored);
+    if (x.warp == 0) {
+        mover_warp<kMode, kFp8, kSteal>(x);
     } else {
-        // ------------------------------------------------------------- layout group
-        bool ok = true;
-        const int* ids = ids_sm;  // staged slots of this CTA's tokens
-        // Small global reads whose values are needed only after the first barriers: issue the
-        // loads now (first trip of each loop), store to shared memory after the ids are staged.
-        const int order_r = gtid < p.R ? __ldg(p.order_pos + gtid) : 0;
-        const bool stage_w = !(kMode == kModeLocal && p.local_fast);
-        const float w_first = (stage_w && gtid < ntok * p.k) ? __ldg(p.topk_w + (size_t)t0 * p.k + gtid) : 0.0f;
-        auto stage_small = [&]() {
-            if (gtid < p.R) order_sm[gtid] = order_r;
-            for (int r = gtid + gn; r < p.R; r += gn) order_sm[r] = __ldg(p.order_pos + r);
-            if (stage_w) {
-                if (gtid < ntok * p.k) w_sm[gtid] = w_first;
-                for (int i = gtid + gn; i < ntok * p.k; i += gn) w_sm[i] = __ldg(p.topk_w + (size_t)t0 * p.k + i);
-            }
-        };
-        if (kMode == kModeLocal && p.local_fast) {
-            // rank-level rows first, movers released, expert-level outputs afterwards
-            const RankMaps rm{bmaps.bm, bmaps.mask_t, (p.R + 31) / 32, ((p.R + 31) / 32) * 32, (p.T + 31) / 32};
-            int* row_sm = reinterpret_cast<int*>(w_sm);
-            local_stage_and_rank_maps(p, ids_sm, rm, warp, kWarps, lane);   // with the mover warp
-            stage_small();
-            group_sync(2, kThreads);
-            if (gtid == 0) trace(p, c, kTrCounted);
-            local_rows_dedup(p, t0, t1, ids_sm, rm, c, order_sm, pos_raw, key, row_sm, arr, gtid, gn);
-            group_sync(1, gn);
-            if (gtid == 0) trace(p, c, kTrFinalized);
-            order_destinations(p, pos_raw, key, pos, ntok * p.k, gtid, gn);
-            group_sync(1, gn);
-            if (gtid == 0) {
-                mbar_arrive(&ready_bar);
-                trace(p, c, kTrReady);
-            }
-            if (part == 0) {
-                float* w_own = reinterpret_cast<float*>(key);   // the ordering keys are no longer needed
-                for (int i = gtid; i < ntok * p.k; i += gn) w_own[i] = __ldg(p.topk_w + (size_t)t0 * p.k + i);
-            }
-            group_sync(1, gn);
-            if (part == 0) local_meta_dedup(p, t0, t1, ids_sm, pos_raw, row_sm, reinterpret_cast<float*>(key), gtid, gn);
-            {
-                // expert-level outputs of rank r: shared by Q CTAs so that no CTA trails the others
-                const int Q = p.grid / p.R > 1 ? p.grid / p.R : 1;
-                for (int u = c; u < p.R * Q; u += p.grid)
-                    local_rank_duty(p, u / Q, u % Q, Q, ids_sm, rm, hist, gw, nw, lane, gtid, gn, 1);
-            }
-            if (gtid == 0) trace(p, c, kTrScanned);   // deferred outputs written
-        } else if (kMode == kModeLocal) {
-            // every CTA: bitmaps over the whole routing table -> totals, the rows before its
-            // own tokens, and (CTAs with a source-rank duty) that rank's counts
-            int* tot = hist;
-            int* pre = hist + p.B;
-            int* eo = hist + 2 * p.B;
-            stage_ids(p, 0, p.T, ids_sm, gtid, gn);
-            stage_small();
-            group_sync(1, gn);
-            if (gtid == 0) trace(p, c, kTrCounted);
-            build_bin_maps(p, ids_sm, p.T, bmaps, gw, nw, lane);
-            group_sync(1, gn);
-            if (gtid == 0) trace(p, c, kTrHistSeen);
-            for (int b = gtid; b < p.B; b += gn) {
-                const int before = bits_in_range(bmaps, b, 0, t0);
-                pre[b] = before;
-                tot[b] = before + bits_in_range(bmaps, b, t0, p.T);
-            }
-            group_sync(1, gn);
-            for (int e = gtid; e < p.E; e += gn) {
-                int o = 0;
-                for (int q = (e / p.L) * p.L; q < e; ++q) o += tot[q];
-                eo[e] = o;
-            }
-            group_sync(1, gn);
-            if (gtid == 0) trace(p, c, kTrScanSeen);
-            ids = ids_sm + (size_t)t0 * p.k;
-            finalize_chunk(p, t0, t1, ids, w_sm,
-                           [&](int e, int tl) { return eo[e] + pre[e] + bits_in_range(bmaps, e, t0, t0 + tl); },
-                           [&](int r, int tl) { return pre[p.E + r] + bits_in_range(bmaps, p.E + r, t0, t0 + tl); },
-                           part == 0, c, order_sm, pos_raw, key, arr, gtid, gn);
-            group_sync(1, gn);
-            if (gtid == 0) trace(p, c, kTrFinalized);
-            order_destinations(p, pos_raw, key, pos, ntok * p.k, gtid, gn);
-            group_sync(1, gn);
-            if (gtid == 0) {
-                mbar_arrive(&ready_bar);
-                trace(p, c, kTrReady);
-            }
-            // outputs nobody inside this kernel waits for
-            if (c == 0) {
-                for (int e = gtid; e < p.E; e += gn) {
-                    p.expert_offset[e] = eo[e];
-                    p.num_tokens_per_expert[e] = tot[e];
-                }
-                for (int r = gtid; r < p.R; r += gn) {
-                    p.num_tokens_per_rank[r] = tot[p.E + r];
-                    int rows = tot[p.E + r];
-                    if (!p.dedup) {
-                        rows = 0;
-                        for (int q = r * p.L; q < (r + 1) * p.L; ++q) rows += tot[q];
-                    }
-                    p.num_rows_per_rank[r] = rows;
-                }
-            }
-            if (part == 0)
-                for (int s = ch; s < p.S; s += p.nchunks) {   // source ranks this CTA reports
-                    const int b0 = src_begin(s, p.T, p.S), b1 = src_begin(s + 1, p.T, p.S);
-                    for (int e = gtid; e < p.E; e += gn) {
-                        p.cnt[(size_t)s * p.E + e] = bits_in_range(bmaps, e, b0, b1);
-                        p.src_offset[(size_t)s * p.E + e] = eo[e] + bits_in_range(bmaps, e, 0, b0);
-                    }
-                }
-        } else {
-            stage_ids(p, t0, t1, ids_sm, gtid, gn);
-            stage_small();
-            group_sync(1, gn);
-            build_bin_maps(p, ids_sm, ntok, bmaps, gw, nw, lane);
-            group_sync(1, gn);
-            int deferred = -1;
-            if (kMode == kModeFused) {
-                publish_chunk_counts(p, ch, t0, t1, bmaps, gtid, gn);
-                group_sync(1, gn);
-                if (gtid == 0) {
-                    if (ch != p.withhold) {
-                        __threadfence();
-                        st_release(p.hist_flag + ch, epoch);
-                    }
-                    trace(p, c, kTrCounted);
-                }
-                // CalCumSum duty: this CTA serves rank ch (and ch + nchunks, ...)
-                bool lost = false;  // a wait of this thread ran out
-                for (int r = ch; r < p.R; r += p.nchunks) {
-                    for (int cc = gtid; cc < p.nchunks; cc += gn)
-                        if (!wait_flag(p.hist_flag + cc, epoch, abortp)) lost = true;
-                    if (group_or(1, gn, lost || *abortp)) { lost = true; break; }  // same answer for all
-                    if (gtid == 0) trace(p, c, kTrHistSeen);
-                    scan_rank_publish(p, r, hist, gw, nw, lane, 1);
-                    if (gtid == 0) {
-                        __threadfence();
-                        st_release(p.scan_flag + r, epoch);
-                        trace(p, c, kTrScanned);
-                    }
-                    if (r + p.nchunks < p.R) {
-                        scan_rank_sources(p, r, hist, gtid, gn);
-                        group_sync(1, gn);
-                    } else {
-                        deferred = r;   // cnt / src_offset: after our own movers are released
-                    }
-                }
-                // every slot of this chunk may need any rank's bases
-                if (!lost)
-                    for (int r = gtid; r < p.R; r += gn)
-                        if (!wait_flag(p.scan_flag + r, epoch, abortp)) lost = true;
-                ok = !group_or(1, gn, lost || *abortp);
-                if (gtid == 0) trace(p, c, kTrScanSeen);
-                if (!ok && gtid == 0) {
-                    report(p.status, kErrTimeout);
-                    abort_flag = 1;
-                }
-            }
-            if (ok) {
-                // rows before a token = rows of earlier chunks (+ the expert's offset in its
-                // region), published by the prefix-sum step, + earlier tokens of this chunk.
-                // The published part is fetched once per bin into shared memory (one round
-                // trip to L2), the rest is bit counting.
-                const int32_t* cb = p.chunk_base + (size_t)ch * p.B;
-                int* base_sm = hist + p.B;   // second half of the scratch (the first may hold scan totals)
-                for (int b = gtid; b < p.B; b += gn)
-                    base_sm[b] = __ldcg(cb + b) + (b < p.E ? __ldcg(p.expert_offset + b) : 0);
-                group_sync(1, gn);
-                finalize_chunk(p, t0, t1, ids, w_sm,
-                               [&](int e, int tl) { return base_sm[e] + bits_in_range(bmaps, e, 0, tl); },
-                               [&](int r, int tl) { return base_sm[p.E + r] + bits_in_range(bmaps, p.E + r, 0, tl); },
-                               true, c, order_sm, pos_raw, key, kSteal ? nullptr : arr, gtid, gn);
-                group_sync(1, gn);
-                if (gtid == 0) trace(p, c, kTrFinalized);
-                order_destinations(p, pos_raw, key, pos, ntok * p.k, gtid, gn);
-                group_sync(1, gn);
-            }
-            if (gtid == 0) {
-                mbar_arrive(&ready_bar);
-                trace(p, c, kTrReady);
-            }
-            if (ok && kSteal) {
-                // this chunk's destinations, for CTAs that run out of work and take over some of its tokens
-                for (int i = gtid; i < ntok * p.k; i += gn) p.copy_pos[(size_t)t0 * p.k + i] = pos[i];
-                group_sync(1, gn);
-                if (gtid == 0) {
-                    __threadfence();
-                    st_release(p.pos_flag + ch, epoch);
-                }
-            }
-            if (ok && deferred >= 0) scan_rank_sources(p, deferred, hist, gtid, gn);
-        }
-        if (kFp8 && ok) {
-            uint8_t* out_ring = smem + pl.off_out;
-            const int g0 = part * (p.G / p.parts);                      // first scale group of this CTA's piece
-            const unsigned scale_bytes = (unsigned)(p.G / p.parts) * 4u;  // its scales travel with the payload
-            const bool scale_bulk = (scale_bytes & 15u) == 0;             // when a bulk copy can carry them
-            const int* item_src = reinterpret_cast<const int*>(smem + pl.off_item);
-            const int* item_pos = item_src + kMaxStages + kOutStages;
-            int* out_src = reinterpret_cast<int*>(smem + pl.off_item) + kMaxStages;   // [kOutStages] 0 = row, -1 = end
-            int* out_pos = out_src + kOutStages + kMaxStages * p.k;                    // [kOutStages, k]
-            if (warp == 1) {
-                // ------------------------------ store issuer: lane j issues the copy of slot j
-                bool sok = true;
-                unsigned long long w_full = 0, w_read = 0, tq = 0;
-                for (int n = 0; kSteal || n < ntok; ++n) {
-                    const int os = n % kOutStages;
-                    if (p.trace) tq = global_ns();
-                    sok = mbar_wait(&out_full[os], (n / kOutStages) & 1, abortp);
-                    if (p.trace) w_full += global_ns() - tq;
-                    sok = __all_sync(0xffffffffu, sok);
-                    if (!sok || (kSteal && out_src[os] < 0)) break;
-                    if (n == 0 && lane == 0) trace(p, c, kTrFirstRow);
-                    const uint8_t* src = out_ring + (size_t)os * pl.out_stage_bytes;
-                    // lanes 0..k-1: payload of slot j; lanes k..2k-1: its scales (when bulk-storable)
-                    for (int j = lane; j < (scale_bulk ? 2 * p.k : p.k); j += 32) {
-                        const int jj = j < p.k ? j : j - p.k;
-                        const int where = kSteal ? out_pos[os * p.k + jj] : pos[n * p.k + jj];
-                        if (where < 0) continue;
-                        if (j < p.k) {
-                            bulk_store(p.recv_x + (size_t)where * p.rowB + out_off, src, out_bytes);
-                            if (kSteal) atomicAdd(&arr[where / p.cap], 1);
-                        } else {
-                            bulk_store(p.recv_scale + (size_t)where * p.G + g0, src + out_bytes, scale_bytes);
-                        }
-                    }
-                    bulk_commit();
-                    if (n + 1 >= kOutStages) {
-                        if (p.trace) tq = global_ns();
-                        bulk_wait_read<kOutStages - 1>();   // every lane: the oldest row's copies have read it
-                        if (p.trace) w_read += global_ns() - tq;
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(&out_empty[(n + 1) % kOutStages]);
-                    }
-                }
-                if (!sok && lane == 0) {
-                    report(p.status, kErrTimeout);
-                    abort_flag = 1;
-                }
-                bulk_wait_all<0>();
-                if (p.trace && lane == 0) {
-                    p.trace[(size_t)c * kTraceSlots + 14] = w_full;
-                    p.trace[(size_t)c * kTraceSlots + 15] = w_read;
-                }
-            } else if (warp - 2 < nq) {
-                // ------------------------------------------------- quantising warps 2 .. nq + 1
-                const int qw = warp - 2;
-                const int nvec = (int)in_bytes / 16;          // 8-channel vectors in this CTA's piece
-                unsigned long long w_in = 0, w_out = 0, t_cmp = 0, tq = 0;
-                for (int n = 0; kSteal || n < ntok; ++n) {
-                    const int s = n % stages, os = n % kOutStages;
-                    if (p.trace) tq = global_ns();
-                    if (!mbar_wait(&full_bar[s], (n / stages) & 1, abortp)) break;
-                    if (p.trace) { unsigned long long t2 = global_ns(); w_in += t2 - tq; tq = t2; }
-                    if (n >= kOutStages && !mbar_wait(&out_empty[os], ((n / kOutStages) - 1) & 1, abortp)) break;
-                    if (p.trace) { unsigned long long t2 = global_ns(); w_out += t2 - tq; tq = t2; }
-                    const int from = kSteal ? item_src[s] : ((ch << 16) | n);
-                    if (from < 0) {
-                        // the loader's closing item: pass it on to the store issuer and leave
-                        if (qw == 0 && lane == 0) out_src[os] = -1;
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(&out_full[os]);
-                        break;
-                    }
-                    const bool own = (from >> 16) == ch;
-                    const int* wpos = own ? pos + (from & 0xffff) * p.k : item_pos + s * p.k;   // this row's destinations
-                    if (kSteal && qw == 0) {
-                        for (int j = lane; j < p.k; j += 32) out_pos[os * p.k + j] = wpos[j];
-                        if (lane == 0) out_src[os] = 0;
-                    }
-                    const uint8_t* src = smem + (size_t)s * pl.stage_bytes;
-                    uint8_t* dst = out_ring + (size_t)os * pl.out_stage_bytes;
-                    float* dst_scale = reinterpret_cast<float*>(dst + out_bytes);
-                    // two vectors per thread and trip, independent of each other
-                    for (int vb = qw * 32; vb < nvec; vb += 2 * nq * 32) {
-                        const int v0 = vb + lane, v1 = v0 + nq * 32;
-                        const bool ok0 = v0 < nvec, ok1 = v1 < nvec;
-                        uint4 in0 = make_uint4(0, 0, 0, 0), in1 = make_uint4(0, 0, 0, 0);
-                        if (ok0) in0 = *reinterpret_cast<const uint4*>(src + (size_t)v0 * 16);
-                        if (ok1) in1 = *reinterpret_cast<const uint4*>(src + (size_t)v1 * 16);
-                        uint2 q0, q1;
-                        float sc0, sc1;
-                        quantize8(in0, ok0, q0, sc0);
-                        quantize8(in1, ok1, q1, sc1);
-                        if (ok0) *reinterpret_cast<uint2*>(dst + (size_t)v0 * 8) = q0;
-                        if (ok1) *reinterpret_cast<uint2*>(dst + (size_t)v1 * 8) = q1;
-                        if ((lane & 15) == 0) {
-                            if (scale_bulk) {
-                                if (ok0) dst_scale[v0 >> 4] = sc0;
-                                if (ok1) dst_scale[v1 >> 4] = sc1;
-                            } else {
-                                for (int j = 0; j < p.k; ++j) {
-                                    const int where = wpos[j];
-                                    if (where < 0) continue;
-                                    if (ok0) p.recv_scale[(size_t)where * p.G + g0 + (v0 >> 4)] = sc0;
-                                    if (ok1) p.recv_scale[(size_t)where * p.G + g0 + (v1 >> 4)] = sc1;
-                                }
-                            }
-                        }
-                    }
-                    fence_proxy_async_smem();   // the bulk stores read what we just wrote
-                    __syncwarp();
-                    if (lane == 0) {
-                        mbar_arrive(&out_full[os]);
-                        mbar_arrive(&empty_bar[s]);
-                    }
-                    if (p.trace) t_cmp += global_ns() - tq;
-                }
-                if (p.trace && warp == 2 && lane == 0) {
-                    p.trace[(size_t)c * kTraceSlots + 11] = w_in;
-                    p.trace[(size_t)c * kTraceSlots + 12] = w_out;
-                    p.trace[(size_t)c * kTraceSlots + 13] = t_cmp;
-                }
-            }
-        }
+        const bool ok = layout_group<kMode, kFp8, kSteal>(x);
+        if (kFp8 && ok) fp8_consumers<kSteal>(x);
     }
     __syncthreads();
     if (abort_flag) {
         // leaving early: the newest load of every ring stage may still be landing
         if (tid == 0) {
-            for (int n = max(0, issued - stages); n < issued; ++n)
+            for (int n = max(0, x.issued - stages); n < x.issued; ++n)
                 (void)mbar_wait(&full_bar[n % stages], (n / stages) & 1, nullptr);
         }
         return;
