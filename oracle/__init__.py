@@ -261,3 +261,58 @@ def hop_distribution(order: np.ndarray, counts: np.ndarray, hop_of: np.ndarray, 
     v = np.empty((workers, n_hops), np.int64)
     _load().orc_hop_distribution(_p(order), _p(counts), _p(hop_of), len(order), workers, n_hops, _p(v))
     return v
+
+
+# ------------------------------------------------- Sec. 3.4: Data-as-Flag encodings
+
+def tff_blocks(row_bytes: int, block_bytes: int, flag_bytes: int) -> int:
+    n = int(_load().orc_tff_blocks(row_bytes, block_bytes, flag_bytes))
+    if n < 0:
+        raise ValueError("orc_tff_blocks: bad arguments")
+    return n
+
+
+def tff_pack(row: np.ndarray, block_bytes: int, flag_bytes: int, flag: int) -> np.ndarray:
+    """DataBlocks (uint8 [blocks, block_bytes]) of one row of bytes."""
+    row = np.ascontiguousarray(row).view(np.uint8).reshape(-1)
+    nb = tff_blocks(row.size, block_bytes, flag_bytes)
+    wire = np.empty((nb, block_bytes), np.uint8)
+    _load().orc_tff_pack(_p(row), row.size, block_bytes, flag_bytes, ctypes.c_uint32(flag), _p(wire))
+    return wire
+
+
+def tff_unpack(wire: np.ndarray, row_bytes: int, block_bytes: int, flag_bytes: int, flag: int,
+               row: Optional[np.ndarray] = None):
+    """Returns (row bytes, number of DataBlocks that have not arrived)."""
+    wire = np.ascontiguousarray(wire).view(np.uint8).reshape(-1)
+    if row is None:
+        row = np.zeros(row_bytes, np.uint8)
+    assert row.dtype == np.uint8 and row.size == row_bytes and row.flags["C_CONTIGUOUS"]
+    missing = int(_load().orc_tff_unpack(_p(wire), row_bytes, block_bytes, flag_bytes,
+                                         ctypes.c_uint32(flag), _p(row)))
+    if missing < 0:
+        raise ValueError("orc_tff_unpack: bad arguments")
+    return row, missing
+
+
+def dc_checksum(rows: np.ndarray, block_bytes: int, marker_bytes: int) -> int:
+    """Accumulated marker sum (mod 2^64) of rows given as a 2-D byte-viewable array."""
+    rows = np.ascontiguousarray(rows)
+    b = rows.view(np.uint8).reshape(rows.shape[0], -1) if rows.shape[0] else np.zeros((0, 8), np.uint8)
+    fn = _load().orc_dc_checksum
+    fn.restype = ctypes.c_uint64
+    return int(fn(_p(b), ctypes.c_int64(b.shape[0]), int(b.shape[1]), ctypes.c_int64(b.shape[1]),
+                  block_bytes, marker_bytes))
+
+
+def sp_pending(data: np.ndarray, block_bytes: int, probe_bytes: int, sentinel: int) -> int:
+    data = np.ascontiguousarray(data).view(np.uint8).reshape(-1)
+    fn = _load().orc_sp_pending
+    fn.restype = ctypes.c_int64
+    return int(fn(_p(data), ctypes.c_int64(data.size), block_bytes, probe_bytes, ctypes.c_uint16(sentinel)))
+
+
+def count_f32_rounding_to_bf16(code: int) -> int:
+    fn = _load().orc_count_f32_rounding_to_bf16
+    fn.restype = ctypes.c_int64
+    return int(fn(ctypes.c_uint16(code)))

@@ -18,6 +18,8 @@
  *     (Sec. 2.3 phase 5, Token-Reordering);
  *   - senders store rows straight into the pre-partitioned destination memory
  *     (Sec. 4, "Global Load/Store for Point-to-Point Synchronization").
+ *   - the Data-as-Flag encodings (Sec. 3.4): Token-Flag Fusion DataBlocks, the
+ *     Data-for-Checksum marker sum and the Sentinel-Polling arrival test.
  * The paper gives no numerics for combine, no FP8 format and no per-rank token
  * de-duplication; those follow the build's stated readings (one fp32 fused
  * multiply-add per slot in slot order and one final round-to-nearest-even to
@@ -28,7 +30,10 @@
  * numpy bincount / cumsum / stable argsort, an exhaustive nearest-code search
  * over all 256 e4m3 codes, torch's CPU float8 cast for in-range values, closed
  * forms (y == 1, identity experts round trip), a float64 error bound, and the
- * post-condition of the prefix-sum search (Algorithm 1) against searchsorted.
+ * post-condition of the prefix-sum search (Algorithm 1) against searchsorted; for the
+ * Sec. 3.4 encodings the paper's own figures (480 payload bytes per 512-byte DataBlock),
+ * a hand-worked fixture, numpy slicing written independently, permutation invariance
+ * of the checksum and an exhaustive walk over all 16-bit probes.
  * Parity unpinned: none of the functions below.
  *
  * Notation: T tokens, H hidden size, E physical experts, R ranks, L = E / R
@@ -479,4 +484,134 @@ void orc_hop_distribution(const int32_t *order, const int32_t *counts, const int
             at += c;
         }
     }
+}
+
+/* --------------------------------------- Sec. 3.4: Data-as-Flag encodings */
+/*
+ * The three readiness schemes of Sec. 3.4 ("Data-as-Flag Synchronization"),
+ * written for a DataBlock of any size so that the same code states the paper's
+ * instance (512-byte blocks, 32-byte flag / marker / probe) and the smaller
+ * blocks a fabric with a smaller atomic store needs (Sec. 7, limitation 1).
+ * Byte order inside a word is little endian.
+ */
+
+/* Token-Flag Fusion: DataBlocks a row of row_bytes turns into, each holding
+ * (block_bytes - flag_bytes) bytes of payload behind a leading flag field. */
+int orc_tff_blocks(int row_bytes, int block_bytes, int flag_bytes)
+{
+    int payload = block_bytes - flag_bytes;
+    if (row_bytes < 0 || payload <= 0 || flag_bytes <= 0 || flag_bytes % 4 != 0) return ORC_ERR_ARG;
+    return (row_bytes + payload - 1) / payload;
+}
+
+/*
+ * Token-Flag Fusion, sender side: block b = flag field (the 32-bit `flag`
+ * repeated over flag_bytes) followed by payload bytes [b*P, (b+1)*P) of the row,
+ * P = block_bytes - flag_bytes; the last block is padded with zeros.
+ */
+int orc_tff_pack(const uint8_t *row, int row_bytes, int block_bytes, int flag_bytes, uint32_t flag,
+                 uint8_t *wire)
+{
+    int nb = orc_tff_blocks(row_bytes, block_bytes, flag_bytes);
+    if (nb < 0) return nb;
+    int P = block_bytes - flag_bytes;
+    for (int b = 0; b < nb; ++b) {
+        uint8_t *blk = wire + (size_t)b * block_bytes;
+        for (int i = 0; i < flag_bytes; ++i) blk[i] = (uint8_t)(flag >> (8 * (i % 4)));
+        for (int i = 0; i < P; ++i) {
+            int at = b * P + i;
+            blk[flag_bytes + i] = at < row_bytes ? row[at] : 0;
+        }
+    }
+    return nb;
+}
+
+/*
+ * Token-Flag Fusion, receiver side: a block has arrived when its whole flag
+ * field holds `flag`; the payload of every arrived block is copied to its place
+ * in the row.  Returns the number of blocks that have NOT arrived (0 = the row
+ * is complete); their part of `row` is left as it was.
+ */
+int orc_tff_unpack(const uint8_t *wire, int row_bytes, int block_bytes, int flag_bytes, uint32_t flag,
+                   uint8_t *row)
+{
+    int nb = orc_tff_blocks(row_bytes, block_bytes, flag_bytes);
+    if (nb < 0) return nb;
+    int P = block_bytes - flag_bytes, missing = 0;
+    for (int b = 0; b < nb; ++b) {
+        const uint8_t *blk = wire + (size_t)b * block_bytes;
+        int here = 1;
+        for (int i = 0; i < flag_bytes; ++i)
+            if (blk[i] != (uint8_t)(flag >> (8 * (i % 4)))) here = 0;
+        if (!here) { ++missing; continue; }
+        for (int i = 0; i < P; ++i) {
+            int at = b * P + i;
+            if (at < row_bytes) row[at] = blk[flag_bytes + i];
+        }
+    }
+    return missing;
+}
+
+/*
+ * Data-for-Checksum: the leading marker_bytes of every DataBlock of every row
+ * are the verification markers; the checksum the sender transmits after the
+ * batch is their accumulated sum.  The paper does not name the sum: here the
+ * markers are read as little-endian 64-bit words and added modulo 2^64.  A
+ * marker cut short by the end of the row contributes the words it has
+ * (row_bytes is a multiple of 8).  rows: n_rows rows, row_stride bytes apart.
+ */
+uint64_t orc_dc_checksum(const uint8_t *rows, int64_t n_rows, int row_bytes, int64_t row_stride,
+                         int block_bytes, int marker_bytes)
+{
+    uint64_t sum = 0;
+    for (int64_t r = 0; r < n_rows; ++r) {
+        const uint8_t *row = rows + r * row_stride;
+        for (int b0 = 0; b0 < row_bytes; b0 += block_bytes)
+            for (int i = 0; i + 8 <= marker_bytes && b0 + i + 8 <= row_bytes && i + 8 <= block_bytes; i += 8) {
+                uint64_t w = 0;
+                for (int j = 0; j < 8; ++j) w |= (uint64_t)row[b0 + i + j] << (8 * j);
+                sum += w;
+            }
+    }
+    return sum;
+}
+
+/*
+ * Sentinel Polling: the receiver fills its buffer with a sentinel and takes a
+ * DataBlock as arrived once its leading probe_bytes differ from it.  Returns
+ * how many DataBlocks of `data` still show the sentinel in all probe bytes
+ * (applied to a receive buffer: blocks not yet arrived; applied to a payload:
+ * blocks whose arrival could never be seen, the deadlock case of Sec. 3.4).
+ * The sentinel is the 16-bit pattern `sentinel` repeated (a bf16 / fp16 code).
+ */
+int64_t orc_sp_pending(const uint8_t *data, int64_t n_bytes, int block_bytes, int probe_bytes, uint16_t sentinel)
+{
+    int64_t pending = 0;
+    for (int64_t b0 = 0; b0 < n_bytes; b0 += block_bytes) {
+        int same = 1;
+        for (int i = 0; i < probe_bytes && i < block_bytes && b0 + i < n_bytes; ++i)
+            if (data[b0 + i] != (uint8_t)(sentinel >> (8 * (i % 2)))) same = 0;
+        pending += same;
+    }
+    return pending;
+}
+
+/*
+ * How many fp32 values that are not NaN round (nearest, ties to even) to the
+ * bf16 code `code`: a literal walk over all 2^32 bit patterns.  Zero for a code
+ * means arithmetic that never yields NaN cannot emit it, which is what Sec. 3.4
+ * asks of the reserved sentinel.
+ */
+int64_t orc_count_f32_rounding_to_bf16(uint16_t code)
+{
+    int64_t n = 0;
+#pragma omp parallel for reduction(+ : n) schedule(static)
+    for (int64_t v = 0; v < (1ll << 32); ++v) {
+        uint32_t u = (uint32_t)v;
+        float f;
+        memcpy(&f, &u, 4);
+        if (f != f) continue;
+        if (f32_to_bf16_rne(f) == code) ++n;
+    }
+    return n;
 }
