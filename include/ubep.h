@@ -36,7 +36,9 @@ enum {
     UBEP_ERR_CAPACITY = -3,  /* device: a region needs more than cap rows; extra rows dropped */
     UBEP_ERR_TIMEOUT = -4,   /* device: a bounded wait on a readiness flag ran out            */
     UBEP_ERR_BAD_INDEX = -5, /* device: an expert id outside [-1, E) was skipped              */
-    UBEP_ERR_ARENA = -6      /* arena too small or not 256-byte aligned                       */
+    UBEP_ERR_ARENA = -6,     /* arena too small or not 256-byte aligned                       */
+    UBEP_ERR_CHECKSUM = -7   /* device: the marker sum a receiver computed differs from the   */
+                             /* checksum its senders announced (ubep_dispatch_sync, DC)       */
 };
 
 enum { UBEP_PAYLOAD_BF16 = 0, UBEP_PAYLOAD_FP8_E4M3 = 1 };
@@ -214,6 +216,100 @@ int ubep_combine(ubep_buffer_t *buf, const void *y /*[dev]*/, const float *topk_
 int ubep_map_workers(const int32_t *order /*[dev]*/, const int32_t *counts /*[dev]*/, int32_t n,
                      int32_t num_experts, int32_t n_workers, int32_t *start_pos /*[dev]*/,
                      int64_t *start_off /*[dev]*/, int32_t *iters /*[dev]*/, void *cuda_stream);
+
+/* ----------------------------------------------------------------------------------------
+ * Readiness protocols (Sec. 3.4, "Data-as-Flag Synchronization").
+ *
+ * ubep_dispatch_sync is a second dispatch path in which the way a receiver learns that its
+ * rows have landed is the protocol under study.  Every CTA of one persistent kernel first
+ * sends the rows of its tokens (sender role) and then, for the receive region it is given,
+ * waits until the protocol says that all expected rows are there (receiver role).  The four
+ * protocols differ only in what the sender adds to the data and in what the receiver looks at:
+ *
+ *   SW   stop-and-wait, the scheme Data-as-Flag replaces: rows are stored into the region,
+ *        then a fence, then one release-add per row on a counter of the region; the receiver
+ *        waits for the counter to reach the region's row count.
+ *   TFF  Token-Flag Fusion: every DataBlock carries a leading flag.  A B200 thread can store
+ *        16 bytes as one access, not 512, so a DataBlock is UBEP_SYNC_BLOCK_BYTES = 16 bytes:
+ *        a 4-byte flag (the sequence number of the call) and 12 bytes of payload, written with
+ *        one 128-bit store into a wire buffer (payload efficiency 12/16 against the paper's
+ *        480/512).  The receiver polls each block's flag, and moves the payload of arrived
+ *        blocks into the region.  No fence and no counter on the sender side.
+ *   DC   Data-for-Checksum: rows are stored into the region unchanged; the leading
+ *        UBEP_SYNC_DC_MARKER_BYTES = 32 bytes of every UBEP_SYNC_DC_BLOCK_BYTES = 512 bytes
+ *        of a row are its markers.  After its last row every sender adds, per region, the sum
+ *        of the markers it sent (little-endian 64-bit words, modulo 2^64 -- the paper does not
+ *        name the sum) to the region's checksum word and announces itself (one fence per
+ *        sender and batch).  The receiver waits for all announcements, sums the markers it
+ *        finds in its region and compares; a difference is reported as UBEP_ERR_CHECKSUM.
+ *   SP   Sentinel Polling: the wire buffer of every region is pre-filled with the sentinel
+ *        (bf16 code 0xFFFF, a NaN pattern no rounding of a number yields, in every element);
+ *        rows are stored into it unchanged with 128-bit stores.  The receiver polls every
+ *        16-byte block until it differs from the sentinel, moves it into the region and puts
+ *        the sentinel back.  A 16-byte block of the input that equals the sentinel is never
+ *        seen to arrive: the wait runs out and UBEP_ERR_TIMEOUT is reported
+ *        (ubep_sync_scan_sentinel counts such blocks beforehand).
+ *
+ * The protocols assume that a naturally aligned 16-byte store of one thread becomes visible
+ * as a whole, which holds on this hardware but is stronger than what the PTX memory model
+ * promises for vector accesses.  All waits are bounded (about 1.5 s); a wait that runs out
+ * records UBEP_ERR_TIMEOUT and the kernel returns.
+ *
+ * Limits: bf16 payload only, T * k <= 8192 (every CTA derives the layout from the whole
+ * routing table, as UBEP_PIPELINE_LOCAL does), one CTA per SM at most.  Everything
+ * ubep_dispatch leaves in the arena is left here too, with identical contents; ubep_combine
+ * may follow.  The arrival counters of ubep_dispatch (UBEP_VIEW_ARRIVAL) are not touched.
+ */
+enum { UBEP_SYNC_SW = 0, UBEP_SYNC_TFF = 1, UBEP_SYNC_DC = 2, UBEP_SYNC_SP = 3 };
+#define UBEP_SYNC_BLOCK_BYTES 16
+#define UBEP_SYNC_FLAG_BYTES 4
+#define UBEP_SYNC_DC_BLOCK_BYTES 512
+#define UBEP_SYNC_DC_MARKER_BYTES 32
+#define UBEP_SYNC_SENTINEL 0xFFFFu
+
+/* Arrays of the wire buffer (ubep_sync_view). */
+enum {
+    UBEP_SYNC_VIEW_TFF_WIRE = 0, /* u8  [R, cap, 16 * ceil(2H / 12)]  DataBlocks of every row     */
+    UBEP_SYNC_VIEW_SP_WIRE = 1,  /* u8  [R, cap, 2H]  all sentinel between calls                  */
+    UBEP_SYNC_VIEW_CHECKSUM = 2, /* u64 [2, R]  DC: marker sums announced (half = call number & 1)*/
+    UBEP_SYNC_VIEW_COUNTERS = 3, /* u32 [4, R]  DC announcements [2, R], then SW row counts [2, R]*/
+    UBEP_SYNC_VIEW_TIMES = 4,    /* u64 [CTAs, 8]  device nanosecond timer of the last call, per CTA:
+                                    0 kernel entry, 1 layout done, 2 last row sent, 3 receiver duty
+                                    confirmed (= 2 for a CTA without one), 4 exit; 5-7 unused      */
+    UBEP_SYNC_VIEW_SEQ = 5,      /* u32 [1]  number of ubep_dispatch_sync kernels that have run   */
+    UBEP_SYNC_VIEW_COUNT_
+};
+
+/* Bytes of the wire buffer for this configuration (0 if it is invalid or not bf16). */
+size_t ubep_sync_wire_bytes(const ubep_config_t *cfg /*[host]*/);
+
+/*
+ * Gives the buffer a wire buffer ([dev], 256-byte aligned, at least ubep_sync_wire_bytes,
+ * caller-owned, must outlive the buffer's last ubep_dispatch_sync) and initialises it on
+ * `cuda_stream`: flags and counters zero, SP wire all sentinel.  Waits for the stream.
+ */
+int ubep_sync_attach(ubep_buffer_t *buf, void *dev_wire /*[dev]*/, size_t bytes, void *cuda_stream);
+
+/*
+ * Dispatch with readiness protocol `protocol` (UBEP_SYNC_*); arguments as ubep_dispatch.
+ * One kernel launch (a memset before it when an earlier call left the SP wire dirty, which
+ * the library learns when ubep_status reports that call's error).  UBEP_ERR_ARG if no wire
+ * buffer is attached, the payload is not bf16 or T * k > 8192.
+ */
+int ubep_dispatch_sync(ubep_buffer_t *buf, int protocol, const void *x /*[dev]*/,
+                       const int32_t *topk_idx /*[dev]*/, const float *topk_w /*[dev]*/, int32_t T,
+                       void *cuda_stream);
+
+/* Device address and shape of one wire-buffer array; valid while the wire buffer is. */
+int ubep_sync_view(ubep_buffer_t *buf, int which, void **dev_ptr /*[host]*/, int64_t shape[4] /*[host]*/);
+
+/*
+ * The check Sec. 3.4 asks for before Sentinel Polling is trusted: counts the 16-byte blocks
+ * of x ([dev] bf16 [T, H]) that equal the sentinel into *count ([host]).  Runs on
+ * `cuda_stream` and waits for it.  Needs an attached wire buffer (its counter word).
+ */
+int ubep_sync_scan_sentinel(ubep_buffer_t *buf, const void *x /*[dev]*/, int32_t T, int64_t *count /*[host]*/,
+                            void *cuda_stream);
 
 /* Device address and shape (unused dims = 1) of one arena array; valid until destroy. */
 int ubep_view(ubep_buffer_t *buf, int which, void **dev_ptr /*[host]*/, int64_t shape[4] /*[host]*/);

@@ -20,6 +20,15 @@ LIB_PATH = os.path.join(_HERE, "libubep.so")
 UBEP_OK = 0
 UBEP_ERR_ARG, UBEP_ERR_CUDA, UBEP_ERR_CAPACITY, UBEP_ERR_TIMEOUT, UBEP_ERR_BAD_INDEX, UBEP_ERR_ARENA = \
     -1, -2, -3, -4, -5, -6
+UBEP_ERR_CHECKSUM = -7
+UBEP_SYNC_SW, UBEP_SYNC_TFF, UBEP_SYNC_DC, UBEP_SYNC_SP = 0, 1, 2, 3
+UBEP_SYNC_BLOCK_BYTES, UBEP_SYNC_FLAG_BYTES = 16, 4
+UBEP_SYNC_DC_BLOCK_BYTES, UBEP_SYNC_DC_MARKER_BYTES = 512, 32
+UBEP_SYNC_SENTINEL = 0xFFFF
+SYNC_NAMES = {"sw": 0, "tff": 1, "dc": 2, "sp": 3}
+SYNC_VIEW_NAMES = ["tff_wire", "sp_wire", "checksum", "counters", "times", "seq"]
+_SYNC_VIEW_DTYPES = [torch.uint8, torch.uint8, torch.int64, torch.int32, torch.int64, torch.int32]
+_SYNC_VIEW_RANK = [3, 3, 2, 2, 2, 1]
 UBEP_PAYLOAD_BF16, UBEP_PAYLOAD_FP8_E4M3 = 0, 1
 UBEP_PIPELINE_AUTO, UBEP_PIPELINE_PHASED, UBEP_PIPELINE_FUSED, UBEP_PIPELINE_LOCAL = 0, 1, 2, 3
 
@@ -35,7 +44,9 @@ EXPORTS = ["ubep_buffer_bytes", "ubep_buffer_create", "ubep_buffer_destroy", "ub
            "ubep_set_dest_order", "ubep_get_dispatch_layout", "ubep_get_dispatch_layout_static", "ubep_dispatch", "ubep_combine", "ubep_view",
            "ubep_status", "ubep_epoch", "ubep_launch_count", "ubep_debug_withhold_flag", "ubep_debug_trace",
            "ubep_debug_set_quant_warps",
-           "ubep_last_cuda_error", "ubep_strerror", "ubep_map_workers"]
+           "ubep_last_cuda_error", "ubep_strerror", "ubep_map_workers",
+           "ubep_sync_wire_bytes", "ubep_sync_attach", "ubep_dispatch_sync", "ubep_sync_view",
+           "ubep_sync_scan_sentinel"]
 
 
 class ubep_config_t(ctypes.Structure):
@@ -81,6 +92,14 @@ def load() -> ctypes.CDLL:
     lib.ubep_strerror.restype, lib.ubep_strerror.argtypes = ctypes.c_char_p, [ctypes.c_int]
     lib.ubep_map_workers.restype = ctypes.c_int
     lib.ubep_map_workers.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp]
+    lib.ubep_sync_wire_bytes.restype, lib.ubep_sync_wire_bytes.argtypes = ctypes.c_size_t, [cfgp]
+    lib.ubep_sync_attach.restype, lib.ubep_sync_attach.argtypes = ctypes.c_int, [vp, vp, ctypes.c_size_t, vp]
+    lib.ubep_dispatch_sync.restype = ctypes.c_int
+    lib.ubep_dispatch_sync.argtypes = [vp, ctypes.c_int, vp, vp, vp, i32, vp]
+    lib.ubep_sync_view.restype = ctypes.c_int
+    lib.ubep_sync_view.argtypes = [vp, ctypes.c_int, ctypes.POINTER(vp), ctypes.POINTER(ctypes.c_int64)]
+    lib.ubep_sync_scan_sentinel.restype = ctypes.c_int
+    lib.ubep_sync_scan_sentinel.argtypes = [vp, vp, i32, ctypes.POINTER(ctypes.c_int64), vp]
     _lib = lib
     return lib
 
@@ -217,6 +236,35 @@ def ubep_debug_withhold_flag(buf, chunk: int) -> None:
     _check(load().ubep_debug_withhold_flag(buf, chunk), "ubep_debug_withhold_flag", buf)
 
 
+def ubep_sync_wire_bytes(cfg: ubep_config_t) -> int:
+    return int(load().ubep_sync_wire_bytes(ctypes.byref(cfg)))
+
+
+def ubep_sync_attach(buf, wire: torch.Tensor, stream=None) -> None:
+    _check(load().ubep_sync_attach(buf, _ptr(wire), wire.numel() * wire.element_size(), _stream(stream)),
+           "ubep_sync_attach", buf)
+
+
+def ubep_dispatch_sync(buf, protocol: int, x: torch.Tensor, topk_idx: torch.Tensor, topk_w: torch.Tensor, T: int,
+                       stream=None) -> None:
+    _check(load().ubep_dispatch_sync(buf, protocol, _ptr(x), _ptr(topk_idx), _ptr(topk_w), T, _stream(stream)),
+           "ubep_dispatch_sync", buf)
+
+
+def ubep_sync_view(buf, which: int):
+    ptr = ctypes.c_void_p()
+    shape = (ctypes.c_int64 * 4)()
+    _check(load().ubep_sync_view(buf, which, ctypes.byref(ptr), shape), "ubep_sync_view", buf)
+    return ptr.value, list(shape)
+
+
+def ubep_sync_scan_sentinel(buf, x: torch.Tensor, T: int, stream=None) -> int:
+    n = ctypes.c_int64(0)
+    _check(load().ubep_sync_scan_sentinel(buf, _ptr(x), T, ctypes.byref(n), _stream(stream)),
+           "ubep_sync_scan_sentinel", buf)
+    return n.value
+
+
 # ------------------------------------------------------------------------ convenience
 
 class Buffer:
@@ -288,6 +336,35 @@ class Buffer:
 
     def status(self) -> int:
         return ubep_status(self.handle)
+
+    def attach_sync(self, fill: Optional[int] = None, stream=None):
+        """Allocates and attaches the wire buffer of the readiness-protocol dispatch."""
+        nbytes = ubep_sync_wire_bytes(self.cfg)
+        if nbytes == 0:
+            raise UbepError(UBEP_ERR_ARG, "ubep_sync_wire_bytes")
+        self.wire = torch.empty(nbytes, dtype=torch.uint8, device=self.arena.device)
+        if fill is not None:
+            self.wire.fill_(fill)
+        ubep_sync_attach(self.handle, self.wire, stream)
+        self.sync_views = {}
+        base = self.wire.data_ptr()
+        for which, (name, dt, rank) in enumerate(zip(SYNC_VIEW_NAMES, _SYNC_VIEW_DTYPES, _SYNC_VIEW_RANK)):
+            ptr, shape = ubep_sync_view(self.handle, which)
+            shape = shape[:rank]
+            n = 1
+            for s in shape:
+                n *= s
+            esz = torch.empty(0, dtype=dt).element_size()
+            self.sync_views[name] = self.wire[ptr - base: ptr - base + n * esz].view(dt).view(shape)
+        return self.sync_views
+
+    def dispatch_sync(self, protocol, x, topk_idx, topk_w, stream=None):
+        if isinstance(protocol, str):
+            protocol = SYNC_NAMES[protocol]
+        ubep_dispatch_sync(self.handle, protocol, x, topk_idx, topk_w, x.shape[0], stream)
+
+    def scan_sentinel(self, x, stream=None) -> int:
+        return ubep_sync_scan_sentinel(self.handle, x, x.shape[0], stream)
 
     def close(self):
         if getattr(self, "handle", None):

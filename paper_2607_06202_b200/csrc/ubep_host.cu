@@ -9,6 +9,7 @@
 
 #include "../../include/ubep.h"
 #include "ubep_kernels.h"
+#include "ubep_sync.h"
 
 using ubep::Params;
 
@@ -97,6 +98,34 @@ ArenaLayout make_layout(const ubep_config_t& c, int nchunks) {
     return a;
 }
 
+// Wire buffer of the readiness-protocol dispatch (byte offsets).
+struct WireLayout {
+    size_t off[UBEP_SYNC_VIEW_COUNT_];
+    size_t flags_begin, seq_ticket, scan_count, flags_end, total;
+    int tff_blocks;
+};
+
+WireLayout make_wire_layout(const ubep_config_t& c, int nchunks) {
+    WireLayout w{};
+    const size_t R = c.num_ranks, cap = c.rows_per_rank_cap, rowB = 2 * (size_t)c.hidden;
+    const int payload = UBEP_SYNC_BLOCK_BYTES - UBEP_SYNC_FLAG_BYTES;
+    w.tff_blocks = (int)((rowB + payload - 1) / payload);
+    size_t at = 0;
+    auto take = [&](size_t bytes) { size_t o = at; at = align_up(at + bytes); return o; };
+    w.off[UBEP_SYNC_VIEW_TFF_WIRE] = take(R * cap * (size_t)w.tff_blocks * UBEP_SYNC_BLOCK_BYTES);
+    w.off[UBEP_SYNC_VIEW_SP_WIRE] = take(R * cap * rowB);
+    w.flags_begin = at;
+    w.off[UBEP_SYNC_VIEW_CHECKSUM] = take(2 * R * 8);
+    w.off[UBEP_SYNC_VIEW_COUNTERS] = take(4 * R * 4);
+    w.off[UBEP_SYNC_VIEW_SEQ] = take(4);
+    w.seq_ticket = take(4);
+    w.scan_count = take(8);
+    w.off[UBEP_SYNC_VIEW_TIMES] = take((size_t)(nchunks > 0 ? nchunks : ubep::kMaxChunks) * ubep::kSyncTimeSlots * 8);
+    w.flags_end = at;
+    w.total = at;
+    return w;
+}
+
 }  // namespace
 
 struct ubep_buffer {
@@ -113,6 +142,9 @@ struct ubep_buffer {
     const int32_t* phys;
     const int32_t* ncopies;
     int32_t E_log, C;
+    uint8_t* wire;      // readiness-protocol wire buffer (caller-owned) or null
+    WireLayout wlay;
+    bool sp_dirty;      // an earlier call may have left non-sentinel blocks in the SP wire
     std::string cuda_error;
 };
 
@@ -229,6 +261,9 @@ int ubep_buffer_create(const ubep_config_t* cfg, void* dev_arena, size_t bytes, 
     b->ncopies = nullptr;
     b->E_log = 0;
     b->C = 0;
+    b->wire = nullptr;
+    b->wlay = WireLayout{};
+    b->sp_dirty = false;
     cudaError_t e = cudaMemset(b->arena + b->lay.flags_begin, 0, b->lay.flags_end - b->lay.flags_begin);
     if (e == cudaSuccess) {
         std::vector<int32_t> ident(cfg->num_ranks);
@@ -375,6 +410,127 @@ int ubep_combine(ubep_buffer_t* buf, const void* y, const float* topk_w, int32_t
     return UBEP_OK;
 }
 
+size_t ubep_sync_wire_bytes(const ubep_config_t* cfg) {
+    if (!cfg || !valid_config(*cfg) || cfg->payload != UBEP_PAYLOAD_BF16) return 0;
+    return make_wire_layout(*cfg, cfg->num_ctas).total;
+}
+
+int ubep_sync_attach(ubep_buffer_t* buf, void* dev_wire, size_t bytes, void* cuda_stream) {
+    if (!buf || !dev_wire || buf->cfg.payload != UBEP_PAYLOAD_BF16) return UBEP_ERR_ARG;
+    if ((reinterpret_cast<uintptr_t>(dev_wire) & (kAlign - 1)) != 0) return UBEP_ERR_ARENA;
+    if (bytes < make_wire_layout(buf->cfg, buf->cfg.num_ctas).total) return UBEP_ERR_ARENA;
+    DeviceGuard guard(buf->cfg.device);
+    if (guard.err != cudaSuccess) return cuda_fail(buf, guard.err);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const WireLayout w = make_wire_layout(buf->cfg, buf->lay.nchunks);
+    uint8_t* base = static_cast<uint8_t*>(dev_wire);
+    // flags of no call (0), sentinel everywhere (0xFF bytes = bf16 code 0xFFFF), counters zero
+    cudaError_t e = cudaMemsetAsync(base + w.off[UBEP_SYNC_VIEW_TFF_WIRE], 0,
+                                    w.off[UBEP_SYNC_VIEW_SP_WIRE] - w.off[UBEP_SYNC_VIEW_TFF_WIRE], st);
+    if (e == cudaSuccess)
+        e = cudaMemsetAsync(base + w.off[UBEP_SYNC_VIEW_SP_WIRE], 0xFF, w.flags_begin - w.off[UBEP_SYNC_VIEW_SP_WIRE], st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(base + w.flags_begin, 0, w.flags_end - w.flags_begin, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(buf, e);
+    buf->wire = base;
+    buf->wlay = w;
+    buf->sp_dirty = false;
+    return UBEP_OK;
+}
+
+int ubep_dispatch_sync(ubep_buffer_t* buf, int protocol, const void* x, const int32_t* topk_idx, const float* topk_w,
+                       int32_t T, void* cuda_stream) {
+    if (!buf || !buf->wire || protocol < UBEP_SYNC_SW || protocol > UBEP_SYNC_SP) return UBEP_ERR_ARG;
+    if (T < 0 || T > buf->cfg.max_tokens || (int64_t)T * buf->cfg.topk > kLocalMaxSlots) return UBEP_ERR_ARG;
+    if (T > 0 && (!x || !topk_idx || !topk_w)) return UBEP_ERR_ARG;
+    if (!aligned16(x) || !aligned16(topk_idx) || !aligned16(topk_w)) return UBEP_ERR_ARG;
+    DeviceGuard guard(buf->cfg.device);
+    if (guard.err != cudaSuccess) return cuda_fail(buf, guard.err);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    buf->last_stream = st;
+    if (T == 0) {
+        const size_t lo = buf->lay.off[UBEP_VIEW_CNT], hi = buf->lay.off[UBEP_VIEW_SLOT_ROW];
+        cudaError_t e0 = cudaMemsetAsync(buf->arena + lo, 0, hi - lo, st);
+        return e0 == cudaSuccess ? UBEP_OK : cuda_fail(buf, e0);
+    }
+    Params p = make_params(buf, T);
+    p.x = static_cast<const uint16_t*>(x);
+    p.topk_idx = topk_idx;
+    p.topk_w = topk_w;
+    p.trace = nullptr;
+    p.parts = 1;
+    p.grid = p.nchunks;
+    ubep::SmemPlan pl{};
+    const int extra = ubep::sync_extra_smem(p);
+    if (ubep::plan_dispatch(p, UBEP_PIPELINE_LOCAL, buf->max_smem - extra, &pl) != 0) return UBEP_ERR_ARG;
+    const WireLayout& w = buf->wlay;
+    ubep::SyncParams sp{};
+    sp.protocol = protocol;
+    sp.tff_blocks = w.tff_blocks;
+    sp.tff_wire = buf->wire + w.off[UBEP_SYNC_VIEW_TFF_WIRE];
+    sp.sp_wire = buf->wire + w.off[UBEP_SYNC_VIEW_SP_WIRE];
+    sp.checksum = reinterpret_cast<unsigned long long*>(buf->wire + w.off[UBEP_SYNC_VIEW_CHECKSUM]);
+    sp.announced = reinterpret_cast<unsigned*>(buf->wire + w.off[UBEP_SYNC_VIEW_COUNTERS]);
+    sp.sw_rows = sp.announced + 2 * (size_t)p.R;
+    sp.seq_ctr = reinterpret_cast<unsigned*>(buf->wire + w.off[UBEP_SYNC_VIEW_SEQ]);
+    sp.seq_ticket = reinterpret_cast<unsigned*>(buf->wire + w.seq_ticket);
+    sp.times = reinterpret_cast<unsigned long long*>(buf->wire + w.off[UBEP_SYNC_VIEW_TIMES]);
+    cudaError_t e = cudaSuccess;
+    if (buf->sp_dirty) {
+        // a call that gave up may have left arrived blocks behind: every block back to the
+        // sentinel, and the counters and the check-in ticket of that call back to zero
+        e = cudaMemsetAsync(sp.sp_wire, 0xFF, w.flags_begin - w.off[UBEP_SYNC_VIEW_SP_WIRE], st);
+        if (e == cudaSuccess)
+            e = cudaMemsetAsync(buf->wire + w.off[UBEP_SYNC_VIEW_CHECKSUM], 0,
+                                w.off[UBEP_SYNC_VIEW_SEQ] - w.off[UBEP_SYNC_VIEW_CHECKSUM], st);
+        if (e != cudaSuccess) return cuda_fail(buf, e);
+        buf->sp_dirty = false;
+    }
+    e = ubep::launch_sync_dispatch(p, pl, sp, st);
+    if (e != cudaSuccess) return cuda_fail(buf, e);
+    g_launches += 1;
+    return UBEP_OK;
+}
+
+int ubep_sync_view(ubep_buffer_t* buf, int which, void** dev_ptr, int64_t shape[4]) {
+    if (!buf || !buf->wire || !dev_ptr || !shape || which < 0 || which >= UBEP_SYNC_VIEW_COUNT_) return UBEP_ERR_ARG;
+    const ubep_config_t& c = buf->cfg;
+    int64_t s[4] = {1, 1, 1, 1};
+    switch (which) {
+        case UBEP_SYNC_VIEW_TFF_WIRE:
+            s[0] = c.num_ranks; s[1] = c.rows_per_rank_cap; s[2] = (int64_t)buf->wlay.tff_blocks * UBEP_SYNC_BLOCK_BYTES;
+            break;
+        case UBEP_SYNC_VIEW_SP_WIRE: s[0] = c.num_ranks; s[1] = c.rows_per_rank_cap; s[2] = 2 * (int64_t)c.hidden; break;
+        case UBEP_SYNC_VIEW_CHECKSUM: s[0] = 2; s[1] = c.num_ranks; break;
+        case UBEP_SYNC_VIEW_COUNTERS: s[0] = 4; s[1] = c.num_ranks; break;
+        case UBEP_SYNC_VIEW_TIMES: s[0] = buf->lay.nchunks; s[1] = ubep::kSyncTimeSlots; break;
+        case UBEP_SYNC_VIEW_SEQ: s[0] = 1; break;
+        default: return UBEP_ERR_ARG;
+    }
+    *dev_ptr = buf->wire + buf->wlay.off[which];
+    for (int i = 0; i < 4; ++i) shape[i] = s[i];
+    return UBEP_OK;
+}
+
+int ubep_sync_scan_sentinel(ubep_buffer_t* buf, const void* x, int32_t T, int64_t* count, void* cuda_stream) {
+    if (!buf || !buf->wire || !count || T < 0 || (T > 0 && !x) || !aligned16(x)) return UBEP_ERR_ARG;
+    DeviceGuard guard(buf->cfg.device);
+    if (guard.err != cudaSuccess) return cuda_fail(buf, guard.err);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    unsigned long long* dev_count = reinterpret_cast<unsigned long long*>(buf->wire + buf->wlay.scan_count);
+    unsigned long long host_count = 0;
+    cudaError_t e = cudaMemsetAsync(dev_count, 0, sizeof(unsigned long long), st);
+    if (e == cudaSuccess && T > 0) {
+        e = ubep::launch_sentinel_scan(x, (long long)T * (buf->cfg.hidden / 8), dev_count, buf->num_sms, st);
+        g_launches += 1;
+    }
+    if (e == cudaSuccess) e = cudaMemcpyAsync(&host_count, dev_count, sizeof(host_count), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(buf, e);
+    *count = (int64_t)host_count;
+    return UBEP_OK;
+}
+
 int ubep_view(ubep_buffer_t* buf, int which, void** dev_ptr, int64_t shape[4]) {
     if (!buf || !dev_ptr || !shape || which < 0 || which >= UBEP_VIEW_COUNT_) return UBEP_ERR_ARG;
     const ubep_config_t& c = buf->cfg;
@@ -425,6 +581,7 @@ int ubep_status(ubep_buffer_t* buf, int32_t* last_async_status) {
         if (e == cudaSuccess) e = cudaStreamSynchronize(buf->last_stream);
     }
     if (e != cudaSuccess) return cuda_fail(buf, e);
+    if (v != 0) buf->sp_dirty = true;   // a call that gave up may not have put every sentinel back
     *last_async_status = v;
     return UBEP_OK;
 }
@@ -462,6 +619,7 @@ const char* ubep_strerror(int code) {
         case UBEP_ERR_TIMEOUT: return "a bounded wait on a readiness flag ran out";
         case UBEP_ERR_BAD_INDEX: return "expert id out of range";
         case UBEP_ERR_ARENA: return "arena too small or misaligned";
+        case UBEP_ERR_CHECKSUM: return "marker sum of a receive region differs from the announced checksum";
         default: return "unknown error";
     }
 }

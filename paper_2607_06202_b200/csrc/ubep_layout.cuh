@@ -9,6 +9,9 @@
 
 namespace ubep {
 
+// (The functions that are not forced inline have internal linkage: more than one source
+// file includes this header.)
+
 // Physical expert of slot (t, j): logical id -> phys[l][t mod ncopies[l]] when a replica
 // table is set.  -1 for an empty slot; ids out of range are reported and treated as empty.
 __device__ __forceinline__ int resolve_expert(const Params& p, int t, int raw) {
@@ -130,7 +133,7 @@ __device__ __forceinline__ unsigned transpose32(unsigned x, int lane) {
 // ids: staged slots of the range (index 0 = first token's slot 0); run by nw warps.  One unit
 // of work = one 32-token group x one 32-bin word: the lane (= token) collects the bins of
 // that word its token selected, the warp transposes the tile and stores it bin-major.
-__device__ void build_bin_maps(const Params& p, const int* ids, int ntok, const BinMaps& bmaps, int gw, int nw,
+static __device__ void build_bin_maps(const Params& p, const int* ids, int ntok, const BinMaps& bmaps, int gw, int nw,
                                int lane) {
     const int k = p.k;
     const int units = bmaps.groups * bmaps.wb;
@@ -166,7 +169,7 @@ __device__ __forceinline__ int bits_in_range(const BinMaps& bmaps, int bin, int 
 
 // Chunk histogram and its running value at the source-rank boundaries inside the chunk
 // (tokens [t0, t1), bitmaps over the chunk), written to chunk_hist[ch] and partial[s].
-__device__ void publish_chunk_counts(const Params& p, int ch, int t0, int t1, const BinMaps& bmaps, int gtid,
+static __device__ void publish_chunk_counts(const Params& p, int ch, int t0, int t1, const BinMaps& bmaps, int gtid,
                                      int gn) {
     const int T = p.T, S = p.S, B = p.B;
     const int s_lo = (int)(((int64_t)t0 * S + T - 1) / T);  // smallest s with src_begin(s) >= t0
@@ -193,7 +196,7 @@ __device__ void publish_chunk_counts(const Params& p, int ch, int t0, int t1, co
 // the region follow from the totals.  `sm` holds L + 1 ints.  Inputs written by other CTAs
 // are read past L1 (__ldcg).  scan_rank_publish must complete before the rank's readiness
 // flag is released; scan_rank_sources only fills cnt / src_offset, which no mover needs.
-__device__ void scan_rank_publish(const Params& p, int r, int* sm, int gw, int nw, int lane, int bar_id) {
+static __device__ void scan_rank_publish(const Params& p, int r, int* sm, int gw, int nw, int lane, int bar_id) {
     const int n = p.nchunks, L = p.L, B = p.B, E = p.E;
     const int nb = L + 1;
     for (int bi = gw; bi < nb; bi += nw) {
@@ -243,7 +246,7 @@ __device__ void scan_rank_publish(const Params& p, int r, int* sm, int gw, int n
     group_sync(bar_id, nw * 32);
 }
 
-__device__ void scan_rank_sources(const Params& p, int r, const int* sm, int gtid, int gn) {
+static __device__ void scan_rank_sources(const Params& p, int r, const int* sm, int gtid, int gn) {
     // tokens before each source boundary = chunk prefix + running histogram at the boundary
     const int n = p.nchunks, L = p.L, B = p.B, T = p.T, S = p.S, E = p.E;
     for (int i = gtid; i < S * L; i += gn) {
@@ -360,7 +363,7 @@ constexpr int kRankWords = 4;
 __device__ __forceinline__ int fast_div(int v, unsigned magic) { return (int)__umulhi((unsigned)v, magic); }
 
 // Stage all T*k slots (packed id | rank << 16) and build the rank bitmaps; lane = token.
-__device__ void local_stage_and_rank_maps(const Params& p, int* ids, const RankMaps& rm, int gw, int nw, int lane) {
+static __device__ void local_stage_and_rank_maps(const Params& p, int* ids, const RankMaps& rm, int gw, int nw, int lane) {
     const int k = p.k, T = p.T;
     const bool vec = (k & 3) == 0;   // a token's ids are whole 16-byte words (topk_idx is 16-byte aligned)
     for (int g = gw; g < rm.groups; g += nw) {
@@ -418,7 +421,7 @@ __device__ __forceinline__ int rank_rows_before(const RankMaps& rm, int r, int t
 // Destinations of this CTA's tokens [t0, t1): pos_raw (slot order), dst_rank, row_sm, arr.
 // (Ordering the destinations with warp shuffles right here instead of in a separate pass
 // was measured slower on the decode shape and is not done.)
-__device__ void local_rows_dedup(const Params& p, int t0, int t1, const int* ids_all, const RankMaps& rm,
+static __device__ void local_rows_dedup(const Params& p, int t0, int t1, const int* ids_all, const RankMaps& rm,
                                  int worker, const int* order_sm, int* pos_raw, int* dst_key, int* row_sm, int* arr,
                                  int gtid, int gn) {
     const int k = p.k;
@@ -449,7 +452,7 @@ __device__ void local_rows_dedup(const Params& p, int t0, int t1, const int* ids
 }
 
 // Metadata of this CTA's own tokens (after the movers were released).
-__device__ void local_meta_dedup(const Params& p, int t0, int t1, const int* ids_all, const int* pos_raw,
+static __device__ void local_meta_dedup(const Params& p, int t0, int t1, const int* ids_all, const int* pos_raw,
                                  const int* row_sm, const float* w_own, int gtid, int gn) {
     const int k = p.k, L = p.L;
     const int nslots = (t1 - t0) * k;
@@ -479,7 +482,7 @@ __device__ void local_meta_dedup(const Params& p, int t0, int t1, const int* ids
 // Needs L < 32.  `sm` holds 2 * 32 ints.  Run by the whole layout group (barrier bar_id).
 // The rank's share is cut into Q parts handled by Q different CTAs: part q writes every
 // Q-th entry of the per-source tables and of the row lists; part 0 also writes the totals.
-__device__ void local_rank_duty(const Params& p, int r, int q, int Q, const int* ids_all, const RankMaps& rm,
+static __device__ void local_rank_duty(const Params& p, int r, int q, int Q, const int* ids_all, const RankMaps& rm,
                                 int* sm, int gw, int nw, int lane, int gtid, int gn, int bar_id) {
     const int k = p.k, L = p.L, T = p.T, S = p.S, E = p.E;
     for (int g = gw; g < rm.groups; g += nw) {
@@ -545,7 +548,7 @@ __device__ void local_rank_duty(const Params& p, int r, int q, int Q, const int*
 // by the worker id (Sec. 3.3: each worker visits a re-mapped destination sequence).  Only
 // the issue order of the copies changes.  One thread per slot: its place is the number of
 // the token's slots with a smaller key (ties keep slot order).  Reads pos / key, writes pos_out.
-__device__ void order_destinations(const Params& p, const int* pos, const int* key, int* pos_out, int nslots,
+static __device__ void order_destinations(const Params& p, const int* pos, const int* key, int* pos_out, int nslots,
                                    int gtid, int gn) {
     const int k = p.k;
     for (int li = gtid; li < nslots; li += gn) {

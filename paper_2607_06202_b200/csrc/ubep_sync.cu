@@ -1,0 +1,374 @@
+// Dispatch with a selectable readiness protocol (Sec. 3.4 of the paper, "Data-as-Flag
+// Synchronization"): stop-and-wait counters, Token-Flag Fusion, Data-for-Checksum and
+// Sentinel Polling.  One persistent kernel; every CTA is first a sender (the rows of its
+// token chunk) and then a receiver (a slice of one receive region), so the waits of the
+// receivers are satisfied by CTAs that never wait themselves.  All CTAs must be resident
+// (grid <= number of SMs, one CTA per SM).
+//
+// The layout (TokenCnt, CalCumSum, slot -> row) is derived by every CTA alone from the
+// whole routing table, with the same device functions and in the same order as the
+// flag-free instance of the main dispatch kernel, so the two paths leave identical
+// metadata in the arena.
+//
+// A DataBlock is the 16 bytes one thread stores with a single 128-bit access.
+#include "ubep_layout.cuh"
+#include "ubep_sync.h"
+
+namespace ubep {
+
+namespace {
+
+constexpr int kSW = 0, kTFF = 1, kDC = 2, kSP = 3;
+constexpr int kDcBlockVecs = 32;    // 512-byte checksum block = 32 vectors of 16 bytes
+constexpr int kDcMarkerVecs = 2;    // its leading 32 bytes are the marker
+
+__device__ __forceinline__ uint4 ld_relaxed_v4(const void* ptr) {
+    uint4 v;
+    asm volatile("ld.relaxed.gpu.global.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(ptr)
+                 : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_relaxed_v4(void* ptr, const uint4 v) {
+    asm volatile("st.relaxed.gpu.global.v4.u32 [%0], {%1, %2, %3, %4};" ::"l"(ptr), "r"(v.x), "r"(v.y), "r"(v.z),
+                 "r"(v.w)
+                 : "memory");
+}
+__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* ptr) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(ptr) : "memory");
+    return v;
+}
+__device__ __forceinline__ bool is_sentinel(const uint4 v) { return (v.x & v.y & v.z & v.w) == 0xffffffffu; }
+__device__ __forceinline__ unsigned long long marker_words(const uint4 v) {
+    return ((unsigned long long)v.x | ((unsigned long long)v.y << 32)) +
+           ((unsigned long long)v.z | ((unsigned long long)v.w << 32));
+}
+
+// Sequence number of the running call, kept on the device like the dispatch epoch: every
+// CTA reads the counter and takes a ticket, the last ticket advances the counter.
+__device__ __forceinline__ unsigned read_seq_and_check_in(const SyncParams& sp, int grid) {
+    unsigned s = ld_acquire(sp.seq_ctr) + 1u;
+    if (s == 0u) s = 1u;   // 0 is what a never-written flag holds
+    if (atomicAdd(sp.seq_ticket, 1u) == (unsigned)grid - 1u) {
+        *sp.seq_ticket = 0u;
+        *sp.seq_ctr = s;
+    }
+    return s;
+}
+
+// Bounded polling: give up after kWaitLimitNs or when another thread of the CTA has.
+struct Waiter {
+    volatile int* abort;
+    unsigned long long t_end;
+    int32_t* status;
+    __device__ __forceinline__ bool keep_waiting(unsigned& spins) {
+        __nanosleep(32);
+        if ((++spins & 127u) != 0) return true;
+        if (*abort) return false;
+        if (global_ns() > t_end) {
+            *abort = 1;
+            report(status, kErrTimeout);
+            return false;
+        }
+        return true;
+    }
+};
+
+__device__ __forceinline__ bool wait_count(const unsigned* ctr, unsigned want, Waiter& wt) {
+    unsigned spins = 0;
+    while (ld_acquire(ctr) != want)
+        if (!wt.keep_waiting(spins)) return false;
+    return true;
+}
+
+template <int kProto>
+__global__ void __launch_bounds__(kThreads, 1) sync_dispatch_kernel(const Params p, const SmemPlan pl,
+                                                                   const SyncParams sp) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    __shared__ unsigned seq_sm;
+    __shared__ int abort_flag;
+    __shared__ unsigned long long tok_sum[2];   // DC: marker sum of the token being sent
+    __shared__ unsigned long long rx_sum;       // DC: marker sum the receiver finds
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, c = blockIdx.x;
+    const int k = p.k, R = p.R;
+    unsigned long long* times = sp.times + (size_t)c * kSyncTimeSlots;
+    if (tid == 0) times[0] = global_ns();
+
+    int* ids_sm = reinterpret_cast<int*>(smem + pl.off_ids);
+    int* pos = reinterpret_cast<int*>(smem + pl.off_pos);
+    int* key = reinterpret_cast<int*>(smem + pl.off_key);
+    float* w_sm = reinterpret_cast<float*>(smem + pl.off_w);
+    int* hist = reinterpret_cast<int*>(smem + pl.off_hist);
+    int* nrows = reinterpret_cast<int*>(smem + pl.off_arr);     // rows every region receives
+    int* order_sm = reinterpret_cast<int*>(smem + pl.off_order);
+    unsigned long long* chk_sm = reinterpret_cast<unsigned long long*>(smem + pl.total);   // DC: [R]
+    const BinMaps bmaps{reinterpret_cast<unsigned*>(smem + pl.off_mask), reinterpret_cast<unsigned*>(smem + pl.off_bm),
+                        pl.map_wb, pl.map_bp, pl.map_groups};
+    const int t0 = (int)chunk_begin(c, p.T, p.nchunks), t1 = (int)chunk_begin(c + 1, p.T, p.nchunks);
+    const int ntok = t1 - t0;
+
+    if (tid == 0) {
+        seq_sm = read_seq_and_check_in(sp, p.grid);
+        abort_flag = 0;
+        tok_sum[0] = tok_sum[1] = 0ull;
+        rx_sum = 0ull;
+    }
+    if (kProto == kDC)
+        for (int r = tid; r < R; r += kThreads) chk_sm[r] = 0ull;
+
+    // ---- layout: bitmaps of every bin over the whole routing table -> totals, the rows
+    // before this CTA's tokens, expert offsets, rows of this CTA's slots
+    int* tot = hist;
+    int* pre = hist + p.B;
+    int* eo = hist + 2 * p.B;
+    stage_ids(p, 0, p.T, ids_sm, tid, kThreads);
+    for (int r = tid; r < R; r += kThreads) order_sm[r] = __ldg(p.order_pos + r);
+    for (int i = tid; i < ntok * k; i += kThreads) w_sm[i] = __ldg(p.topk_w + (size_t)t0 * k + i);
+    __syncthreads();
+    const unsigned seq = seq_sm;
+    const int par = (int)(seq & 1u);
+    build_bin_maps(p, ids_sm, p.T, bmaps, warp, kWarps, lane);
+    __syncthreads();
+    for (int b = tid; b < p.B; b += kThreads) {
+        const int before = bits_in_range(bmaps, b, 0, t0);
+        pre[b] = before;
+        tot[b] = before + bits_in_range(bmaps, b, t0, p.T);
+    }
+    __syncthreads();
+    for (int e = tid; e < p.E; e += kThreads) {
+        int o = 0;
+        for (int q = (e / p.L) * p.L; q < e; ++q) o += tot[q];
+        eo[e] = o;
+    }
+    for (int r = tid; r < R; r += kThreads) {
+        int rows = tot[p.E + r];
+        if (!p.dedup) {
+            rows = 0;
+            for (int q = r * p.L; q < (r + 1) * p.L; ++q) rows += tot[q];
+        }
+        nrows[r] = rows;
+    }
+    __syncthreads();
+    finalize_chunk(p, t0, t1, ids_sm + (size_t)t0 * k, w_sm,
+                   [&](int e, int tl) { return eo[e] + pre[e] + bits_in_range(bmaps, e, t0, t0 + tl); },
+                   [&](int r, int tl) { return pre[p.E + r] + bits_in_range(bmaps, p.E + r, t0, t0 + tl); },
+                   true, c, order_sm, pos, key, nullptr, tid, kThreads);
+    __syncthreads();
+    if (tid == 0) times[1] = global_ns();
+    // counts and offsets nobody inside this kernel waits for
+    if (c == 0) {
+        for (int e = tid; e < p.E; e += kThreads) {
+            p.expert_offset[e] = eo[e];
+            p.num_tokens_per_expert[e] = tot[e];
+        }
+        for (int r = tid; r < R; r += kThreads) {
+            p.num_tokens_per_rank[r] = tot[p.E + r];
+            p.num_rows_per_rank[r] = nrows[r];
+        }
+    }
+    for (int s = c; s < p.S; s += p.grid) {
+        const int b0 = src_begin(s, p.T, p.S), b1 = src_begin(s + 1, p.T, p.S);
+        for (int e = tid; e < p.E; e += kThreads) {
+            p.cnt[(size_t)s * p.E + e] = bits_in_range(bmaps, e, b0, b1);
+            p.src_offset[(size_t)s * p.E + e] = eo[e] + bits_in_range(bmaps, e, 0, b0);
+        }
+    }
+
+    // ---- sender: the rows of tokens [t0, t1), one token at a time, all threads on a row
+    const int nvec = p.rowB / 16;
+    const int nwords = p.rowB / 4;
+    const size_t wire_row = (size_t)sp.tff_blocks * 16;
+    for (int tl = 0; tl < ntok; ++tl) {
+        const int* ps = pos + tl * k;
+        if (kProto == kTFF) {
+            const uint32_t* xw = reinterpret_cast<const uint32_t*>(p.x + (size_t)(t0 + tl) * p.H);
+            for (int g = tid; g < sp.tff_blocks; g += kThreads) {
+                const int w0 = 3 * g;
+                uint4 blk;
+                blk.x = seq;   // the flag leads the block
+                blk.y = w0 < nwords ? __ldg(xw + w0) : 0u;
+                blk.z = w0 + 1 < nwords ? __ldg(xw + w0 + 1) : 0u;
+                blk.w = w0 + 2 < nwords ? __ldg(xw + w0 + 2) : 0u;
+                for (int j = 0; j < k; ++j) {
+                    const int where = ps[j];
+                    if (where >= 0) st_relaxed_v4(sp.tff_wire + (size_t)where * wire_row + (size_t)g * 16, blk);
+                }
+            }
+        } else {
+            const uint4* src = reinterpret_cast<const uint4*>(p.x + (size_t)(t0 + tl) * p.H);
+            uint8_t* dst = kProto == kSP ? sp.sp_wire : p.recv_x;
+            unsigned long long mine = 0ull;
+            for (int v = tid; v < nvec; v += kThreads) {
+                const uint4 d = __ldg(src + v);
+                if (kProto == kDC && (v % kDcBlockVecs) < kDcMarkerVecs) mine += marker_words(d);
+                for (int j = 0; j < k; ++j) {
+                    const int where = ps[j];
+                    if (where < 0) continue;
+                    uint8_t* at = dst + (size_t)where * p.rowB + (size_t)v * 16;
+                    if (kProto == kSP) st_relaxed_v4(at, d);
+                    else *reinterpret_cast<uint4*>(at) = d;
+                }
+            }
+            if (kProto == kDC) {
+                // marker sum of this row, added to the running sum of every region it goes to
+                if (mine) atomicAdd(&tok_sum[tl & 1], mine);
+                __syncthreads();
+                if (tid == 0) tok_sum[(tl + 1) & 1] = 0ull;
+                if (tid < k && ps[tid] >= 0) atomicAdd(&chk_sm[ps[tid] / p.cap], tok_sum[tl & 1]);
+                __syncthreads();
+            }
+            if (kProto == kSW) {
+                // stop-and-wait: the row's stores are fenced before its flag is raised
+                __threadfence();
+                __syncthreads();
+                if (tid < k && ps[tid] >= 0) red_release_add(sp.sw_rows + par * R + ps[tid] / p.cap, 1u);
+            }
+        }
+    }
+    if (kProto == kDC) {
+        // one fence per sender and batch, then the checksum packet of every region
+        __threadfence();
+        __syncthreads();
+        for (int r = tid; r < R; r += kThreads) {
+            if (chk_sm[r]) atomicAdd(sp.checksum + par * R + r, chk_sm[r]);
+            red_release_add(sp.announced + par * R + r, 1u);
+        }
+    }
+    if (tid == 0) times[2] = global_ns();
+
+    // ---- receiver: region u / Q, slice u % Q of its rows
+    Waiter wt{&abort_flag, global_ns() + kWaitLimitNs, p.status};
+    const int Q = p.grid / R > 1 ? p.grid / R : 1;
+    bool duty = false;
+    for (int u = c; u < R * Q; u += p.grid) {
+        const int r = u / Q, q = u % Q;
+        const int n_r = nrows[r] < p.cap ? nrows[r] : p.cap;
+        if (kProto == kTFF || kProto == kSP) {
+            const int lo = (int)((long long)n_r * q / Q), hi = (int)((long long)n_r * (q + 1) / Q);
+            duty = duty || hi > lo;
+            for (int row = lo; row < hi && !abort_flag; ++row) {
+                const size_t grow = (size_t)r * p.cap + row;
+                if (kProto == kTFF) {
+                    const uint8_t* w = sp.tff_wire + grow * wire_row;
+                    uint32_t* out = reinterpret_cast<uint32_t*>(p.recv_x + grow * p.rowB);
+                    for (int g = tid; g < sp.tff_blocks; g += kThreads) {
+                        uint4 blk;
+                        unsigned spins = 0;
+                        bool ok = true;
+                        for (;;) {
+                            blk = ld_relaxed_v4(w + (size_t)g * 16);
+                            if (blk.x == seq) break;
+                            if (!wt.keep_waiting(spins)) { ok = false; break; }
+                        }
+                        if (!ok) break;
+                        const int w0 = 3 * g;
+                        if (w0 < nwords) out[w0] = blk.y;
+                        if (w0 + 1 < nwords) out[w0 + 1] = blk.z;
+                        if (w0 + 2 < nwords) out[w0 + 2] = blk.w;
+                    }
+                } else {
+                    uint8_t* w = sp.sp_wire + grow * p.rowB;
+                    uint4* out = reinterpret_cast<uint4*>(p.recv_x + grow * p.rowB);
+                    const uint4 sentinel = make_uint4(0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu);
+                    for (int v = tid; v < nvec; v += kThreads) {
+                        uint4 d;
+                        unsigned spins = 0;
+                        bool ok = true;
+                        for (;;) {
+                            d = ld_relaxed_v4(w + (size_t)v * 16);
+                            if (!is_sentinel(d)) break;
+                            if (!wt.keep_waiting(spins)) { ok = false; break; }
+                        }
+                        if (!ok) break;
+                        out[v] = d;
+                        st_relaxed_v4(w + (size_t)v * 16, sentinel);   // consumed: ready for the next call
+                    }
+                }
+            }
+        } else if (q == 0) {
+            duty = true;
+            if (kProto == kSW) {
+                if (tid == 0) (void)wait_count(sp.sw_rows + par * R + r, (unsigned)n_r, wt);
+            } else {
+                if (tid == 0) (void)wait_count(sp.announced + par * R + r, (unsigned)p.grid, wt);
+                __syncthreads();
+                if (!abort_flag) {
+                    const int nblk = (nvec + kDcBlockVecs - 1) / kDcBlockVecs;
+                    const int per_row = nblk * kDcMarkerVecs;
+                    unsigned long long mine = 0ull;
+                    for (int i = tid; i < n_r * per_row; i += kThreads) {
+                        const int row = i / per_row, rem = i - row * per_row;
+                        const int v = (rem / kDcMarkerVecs) * kDcBlockVecs + rem % kDcMarkerVecs;
+                        if (v < nvec)
+                            mine += marker_words(__ldcg(
+                                reinterpret_cast<const uint4*>(p.recv_x + ((size_t)r * p.cap + row) * p.rowB) + v));
+                    }
+                    if (mine) atomicAdd(&rx_sum, mine);
+                    __syncthreads();
+                    if (tid == 0) {
+                        if (rx_sum != ld_relaxed_u64(sp.checksum + par * R + r)) report(p.status, kErrChecksum);
+                        rx_sum = 0ull;
+                    }
+                }
+                __syncthreads();
+            }
+        }
+    }
+    __syncthreads();
+    if (tid == 0) times[3] = (duty && !abort_flag) ? global_ns() : times[2];
+    // the counters of the next call live in the other half: clear them now
+    if (c == 0)
+        for (int r = tid; r < R; r += kThreads) {
+            sp.checksum[(par ^ 1) * R + r] = 0ull;
+            sp.announced[(par ^ 1) * R + r] = 0u;
+            sp.sw_rows[(par ^ 1) * R + r] = 0u;
+        }
+    if (tid == 0) times[4] = global_ns();
+}
+
+__global__ void __launch_bounds__(256) sentinel_scan_kernel(const uint4* __restrict__ x, long long n_vec,
+                                                            unsigned long long* count) {
+    unsigned long long mine = 0ull;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec;
+         i += (long long)gridDim.x * blockDim.x)
+        mine += is_sentinel(__ldg(x + i)) ? 1ull : 0ull;
+    for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
+    if ((threadIdx.x & 31) == 0 && mine) atomicAdd(count, mine);
+}
+
+template <int kProto>
+cudaError_t launch_one(const Params& p, const SmemPlan& pl, const SyncParams& sp, cudaStream_t st) {
+    auto kern = sync_dispatch_kernel<kProto>;
+    const int smem = pl.total + sync_extra_smem(p);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    kern<<<p.grid, kThreads, smem, st>>>(p, pl, sp);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+int sync_extra_smem(const Params& p) { return p.R * 8 + 128; }
+
+cudaError_t launch_sync_dispatch(const Params& p, const SmemPlan& pl, const SyncParams& sp, cudaStream_t st) {
+    switch (sp.protocol) {
+        case kSW: return launch_one<kSW>(p, pl, sp, st);
+        case kTFF: return launch_one<kTFF>(p, pl, sp, st);
+        case kDC: return launch_one<kDC>(p, pl, sp, st);
+        case kSP: return launch_one<kSP>(p, pl, sp, st);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+cudaError_t launch_sentinel_scan(const void* x, long long n_vec, unsigned long long* count, int num_sms,
+                                 cudaStream_t st) {
+    long long blocks = (n_vec + 255) / 256;
+    if (blocks > (long long)num_sms * 8) blocks = (long long)num_sms * 8;
+    if (blocks < 1) blocks = 1;
+    sentinel_scan_kernel<<<(int)blocks, 256, 0, st>>>(static_cast<const uint4*>(x), n_vec, count);
+    return cudaGetLastError();
+}
+
+}  // namespace ubep

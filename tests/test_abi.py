@@ -36,7 +36,7 @@ def test_header_is_plain_c():
 def test_strerror_and_codes(lib):
     assert B.ubep_strerror(0) == "ok"
     for code in (B.UBEP_ERR_ARG, B.UBEP_ERR_CUDA, B.UBEP_ERR_CAPACITY, B.UBEP_ERR_TIMEOUT,
-                 B.UBEP_ERR_BAD_INDEX, B.UBEP_ERR_ARENA):
+                 B.UBEP_ERR_BAD_INDEX, B.UBEP_ERR_ARENA, B.UBEP_ERR_CHECKSUM):
         assert B.ubep_strerror(code) not in ("ok", "unknown error")
     assert B.ubep_strerror(-99) == "unknown error"
 
@@ -78,6 +78,26 @@ def test_null_arguments_are_rejected_without_a_gpu(lib):
     assert lib.ubep_status(None, None) == B.UBEP_ERR_ARG
     assert lib.ubep_epoch(None) == 0
     assert lib.ubep_launch_count() == 0
+    assert lib.ubep_sync_attach(None, None, 0, None) == B.UBEP_ERR_ARG
+    assert lib.ubep_dispatch_sync(None, 0, None, None, None, 0, None) == B.UBEP_ERR_ARG
+    assert lib.ubep_sync_view(None, 0, None, None) == B.UBEP_ERR_ARG
+    assert lib.ubep_sync_scan_sentinel(None, None, 0, None, None) == B.UBEP_ERR_ARG
+
+
+def test_wire_bytes_of_the_readiness_protocols(lib):
+    # decode-sized: Token-Flag blocks (16 bytes per 12 of payload) plus the sentinel wire
+    kw = dict(num_ranks=32, num_experts=256, hidden=7168, topk=8, max_tokens=512, rows_per_rank_cap=256, dedup=1)
+    rows = 32 * 256
+    tff_row = 16 * -(-14336 // 12)
+    n = B.ubep_sync_wire_bytes(_cfg(**kw))
+    assert rows * (tff_row + 14336) < n < rows * (tff_row + 14336) * 1.01
+    assert B.ubep_sync_wire_bytes(_cfg(payload=1)) == 0            # bf16 rows only
+    assert B.ubep_sync_wire_bytes(_cfg(num_experts=18)) == 0
+    assert (B.UBEP_SYNC_BLOCK_BYTES - B.UBEP_SYNC_FLAG_BYTES) / B.UBEP_SYNC_BLOCK_BYTES == 0.75
+    header = open(os.path.join(ROOT, "include", "ubep.h")).read()
+    for name in ("UBEP_SYNC_BLOCK_BYTES", "UBEP_SYNC_FLAG_BYTES", "UBEP_SYNC_DC_BLOCK_BYTES",
+                 "UBEP_SYNC_DC_MARKER_BYTES"):
+        assert int(re.search(rf"#define {name} (\d+)", header).group(1)) == getattr(B, name)
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
