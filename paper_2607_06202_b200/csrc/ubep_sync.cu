@@ -46,6 +46,12 @@ __device__ __forceinline__ unsigned long long marker_words(const uint4 v) {
            ((unsigned long long)v.z | ((unsigned long long)v.w << 32));
 }
 
+__device__ __forceinline__ unsigned long long warp_sum64(unsigned long long v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
 // Sequence number of the running call, kept on the device like the dispatch epoch: every
 // CTA reads the counter and takes a ticket, the last ticket advances the counter.
 __device__ __forceinline__ unsigned read_seq_and_check_in(const SyncParams& sp, int grid) {
@@ -89,8 +95,7 @@ __global__ void __launch_bounds__(kThreads, 1) sync_dispatch_kernel(const Params
     extern __shared__ __align__(128) uint8_t smem[];
     __shared__ unsigned seq_sm;
     __shared__ int abort_flag;
-    __shared__ unsigned long long tok_sum[2];   // DC: marker sum of the token being sent
-    __shared__ unsigned long long rx_sum;       // DC: marker sum the receiver finds
+    __shared__ unsigned long long wsum[2][kWarps];   // DC: per-warp marker sums (two tokens in flight)
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, c = blockIdx.x;
     const int k = p.k, R = p.R;
     unsigned long long* times = sp.times + (size_t)c * kSyncTimeSlots;
@@ -112,8 +117,6 @@ __global__ void __launch_bounds__(kThreads, 1) sync_dispatch_kernel(const Params
     if (tid == 0) {
         seq_sm = read_seq_and_check_in(sp, p.grid);
         abort_flag = 0;
-        tok_sum[0] = tok_sum[1] = 0ull;
-        rx_sum = 0ull;
     }
     if (kProto == kDC)
         for (int r = tid; r < R; r += kThreads) chk_sm[r] = 0ull;
@@ -213,11 +216,15 @@ __global__ void __launch_bounds__(kThreads, 1) sync_dispatch_kernel(const Params
             }
             if (kProto == kDC) {
                 // marker sum of this row, added to the running sum of every region it goes to
-                if (mine) atomicAdd(&tok_sum[tl & 1], mine);
+                // (the slot of the token after next is written only after the next barrier)
+                mine = warp_sum64(mine);
+                if (lane == 0) wsum[tl & 1][warp] = mine;
                 __syncthreads();
-                if (tid == 0) tok_sum[(tl + 1) & 1] = 0ull;
-                if (tid < k && ps[tid] >= 0) atomicAdd(&chk_sm[ps[tid] / p.cap], tok_sum[tl & 1]);
-                __syncthreads();
+                if (tid < k && ps[tid] >= 0) {
+                    unsigned long long row_sum = 0ull;
+                    for (int q = 0; q < kWarps; ++q) row_sum += wsum[tl & 1][q];
+                    atomicAdd(&chk_sm[ps[tid] / p.cap], row_sum);
+                }
             }
             if (kProto == kSW) {
                 // stop-and-wait: the row's stores are fenced before its flag is raised
@@ -248,42 +255,46 @@ __global__ void __launch_bounds__(kThreads, 1) sync_dispatch_kernel(const Params
         if (kProto == kTFF || kProto == kSP) {
             const int lo = (int)((long long)n_r * q / Q), hi = (int)((long long)n_r * (q + 1) / Q);
             duty = duty || hi > lo;
-            for (int row = lo; row < hi && !abort_flag; ++row) {
-                const size_t grow = (size_t)r * p.cap + row;
-                if (kProto == kTFF) {
-                    const uint8_t* w = sp.tff_wire + grow * wire_row;
-                    uint32_t* out = reinterpret_cast<uint32_t*>(p.recv_x + grow * p.rowB);
-                    for (int g = tid; g < sp.tff_blocks; g += kThreads) {
-                        uint4 blk;
-                        unsigned spins = 0;
-                        bool ok = true;
-                        for (;;) {
-                            blk = ld_relaxed_v4(w + (size_t)g * 16);
-                            if (blk.x == seq) break;
-                            if (!wt.keep_waiting(spins)) { ok = false; break; }
-                        }
-                        if (!ok) break;
-                        const int w0 = 3 * g;
-                        if (w0 < nwords) out[w0] = blk.y;
-                        if (w0 + 1 < nwords) out[w0 + 1] = blk.z;
-                        if (w0 + 2 < nwords) out[w0 + 2] = blk.w;
+            // The slice's DataBlocks as one index space; every thread keeps kBatch loads in
+            // flight and only then looks at what they brought (a block that has not arrived
+            // is polled on its own).
+            constexpr int kBatch = 4;
+            const int per_row = kProto == kTFF ? sp.tff_blocks : nvec;
+            const size_t row_stride = kProto == kTFF ? wire_row : (size_t)p.rowB;
+            uint8_t* const wire = (kProto == kTFF ? sp.tff_wire : sp.sp_wire) + ((size_t)r * p.cap + lo) * row_stride;
+            uint8_t* const region = p.recv_x + ((size_t)r * p.cap + lo) * p.rowB;
+            const int items = (hi - lo) * per_row;
+            const uint4 sentinel = make_uint4(0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu);
+            bool ok = true;
+            for (int i0 = tid; ok && i0 < items && !*wt.abort; i0 += kBatch * kThreads) {
+                uint4 blk[kBatch];
+                int row[kBatch], g[kBatch];
+#pragma unroll
+                for (int b = 0; b < kBatch; ++b) {
+                    const int i = i0 + b * kThreads;
+                    row[b] = i / per_row;
+                    g[b] = i - row[b] * per_row;
+                    if (i < items) blk[b] = ld_relaxed_v4(wire + row[b] * row_stride + (size_t)g[b] * 16);
+                }
+#pragma unroll
+                for (int b = 0; b < kBatch; ++b) {
+                    if (i0 + b * kThreads >= items) break;
+                    uint8_t* const src = wire + row[b] * row_stride + (size_t)g[b] * 16;
+                    unsigned spins = 0;
+                    while (kProto == kTFF ? blk[b].x != seq : is_sentinel(blk[b])) {
+                        if (!wt.keep_waiting(spins)) { ok = false; break; }
+                        blk[b] = ld_relaxed_v4(src);
                     }
-                } else {
-                    uint8_t* w = sp.sp_wire + grow * p.rowB;
-                    uint4* out = reinterpret_cast<uint4*>(p.recv_x + grow * p.rowB);
-                    const uint4 sentinel = make_uint4(0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu);
-                    for (int v = tid; v < nvec; v += kThreads) {
-                        uint4 d;
-                        unsigned spins = 0;
-                        bool ok = true;
-                        for (;;) {
-                            d = ld_relaxed_v4(w + (size_t)v * 16);
-                            if (!is_sentinel(d)) break;
-                            if (!wt.keep_waiting(spins)) { ok = false; break; }
-                        }
-                        if (!ok) break;
-                        out[v] = d;
-                        st_relaxed_v4(w + (size_t)v * 16, sentinel);   // consumed: ready for the next call
+                    if (!ok) break;
+                    if (kProto == kTFF) {
+                        uint32_t* out = reinterpret_cast<uint32_t*>(region + (size_t)row[b] * p.rowB);
+                        const int w0 = 3 * g[b];
+                        if (w0 < nwords) out[w0] = blk[b].y;
+                        if (w0 + 1 < nwords) out[w0 + 1] = blk[b].z;
+                        if (w0 + 2 < nwords) out[w0 + 2] = blk[b].w;
+                    } else {
+                        *reinterpret_cast<uint4*>(region + (size_t)row[b] * p.rowB + (size_t)g[b] * 16) = blk[b];
+                        st_relaxed_v4(src, sentinel);   // consumed: ready for the next call
                     }
                 }
             }
@@ -305,11 +316,13 @@ __global__ void __launch_bounds__(kThreads, 1) sync_dispatch_kernel(const Params
                             mine += marker_words(__ldcg(
                                 reinterpret_cast<const uint4*>(p.recv_x + ((size_t)r * p.cap + row) * p.rowB) + v));
                     }
-                    if (mine) atomicAdd(&rx_sum, mine);
+                    mine = warp_sum64(mine);
+                    if (lane == 0) wsum[0][warp] = mine;
                     __syncthreads();
                     if (tid == 0) {
-                        if (rx_sum != ld_relaxed_u64(sp.checksum + par * R + r)) report(p.status, kErrChecksum);
-                        rx_sum = 0ull;
+                        unsigned long long found = 0ull;
+                        for (int q = 0; q < kWarps; ++q) found += wsum[0][q];
+                        if (found != ld_relaxed_u64(sp.checksum + par * R + r)) report(p.status, kErrChecksum);
                     }
                 }
                 __syncthreads();
