@@ -404,7 +404,7 @@ int ubep_combine(ubep_buffer_t* buf, const void* y, const float* topk_w, int32_t
     buf->last_stream = st;
     cudaError_t e = ubep::launch_combine(static_cast<const uint16_t*>(y), at<int32_t>(buf, buf->lay.slot_pos), topk_w,
                                          T, buf->cfg.hidden, buf->cfg.topk, static_cast<uint16_t*>(out),
-                                         buf->num_sms, st);
+                                         buf->num_sms, (int64_t)T * buf->cfg.topk <= kLocalMaxSlots, st);
     if (e != cudaSuccess) return cuda_fail(buf, e);
     g_launches += 1;
     return UBEP_OK;
