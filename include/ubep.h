@@ -100,7 +100,10 @@ enum {
                                  /*                     captured CUDA graph needs no reset     */
     UBEP_VIEW_TRACE = 16,        /* u64 [chunks, 16]    per-CTA phase time stamps in ns of the */
                                  /*                     last traced dispatch (ubep_debug_trace)*/
-    UBEP_VIEW_COUNT_ = 17
+    UBEP_VIEW_SHARD_ARRIVAL = 17,/* u32 [2]             sharded use: rows announced to this    */
+                                 /*                     rank's region so far, rows expected so */
+                                 /*                     far (both modulo 2^32, never reset)    */
+    UBEP_VIEW_COUNT_ = 18
 };
 
 /*
@@ -310,6 +313,64 @@ int ubep_sync_view(ubep_buffer_t *buf, int which, void **dev_ptr /*[host]*/, int
  */
 int ubep_sync_scan_sentinel(ubep_buffer_t *buf, const void *x /*[dev]*/, int32_t T, int64_t *count /*[host]*/,
                             void *cuda_stream);
+
+/* ----------------------------------------------------------------------------------------
+ * Ranks on different GPUs (Sec. 2.3 and Sec. 4, "Global Load/Store for Point-to-Point
+ * Synchronization"): rank r is GPU r, S = R, every GPU holds an arena of the same
+ * configuration (hence the same layout) in memory its peers can address -- peer-to-peer
+ * mappings over NVLink, which the caller sets up and passes in as plain device pointers.
+ * Receive region r is used in arena r only.  One buffer handle per GPU and process.
+ *
+ * A dispatch of the global batch of T tokens then is, on every rank s:
+ *   1. (caller) all-gather of the routing table, so that every rank holds topk_idx and
+ *      topk_w of all T tokens -- 8 bytes per slot against 2H bytes per row;
+ *   2. ubep_dispatch_sharded: the rank derives the whole layout from the table (every rank
+ *      gets the same counts and offsets, each into its own arena), and stores the rows of its
+ *      own tokens, floor(s*T/R) <= t < floor((s+1)*T/R), and their metadata straight into the
+ *      regions of the ranks that host their experts (plain 128-bit stores to peer memory; no
+ *      multicast, no collective).  Then one system-scope fence and one release-add per
+ *      destination rank on that rank's arrival word;
+ *   3. ubep_wait_arrivals: a one-CTA kernel that waits (bounded, about 1.5 s, then
+ *      UBEP_ERR_TIMEOUT) until the local arrival word has reached the number of rows this
+ *      rank's region receives.  The arrival words only grow (modulo 2^32); nothing is reset
+ *      between calls, so a fast peer can never have its announcement wiped out.
+ * ubep_combine_sharded gathers, for the rank's own tokens, expert-output rows from the ranks
+ * that produced them with plain loads from peer memory.
+ *
+ * The caller orders the steps across ranks where data is reused: no rank may start dispatch
+ * n + 1 before every rank has finished reading what dispatch n delivered, and no rank may
+ * start combine before the y of every peer is complete (a barrier on the streams, e.g. an
+ * NCCL one).  Limits of this path: bf16 payload, T * k <= 8192, no FP8, no replicas beyond
+ * ubep_set_replicas.  Kernels of different ranks never wait for one another except in
+ * ubep_wait_arrivals, which therefore must not be emulated by launches queued on one GPU
+ * ahead of the senders it waits for.
+ */
+
+/*
+ * Puts the buffer in sharded use.  peer_arenas [host]: R device pointers, entry r = the
+ * arena of rank r as this GPU addresses it (entry my_rank = the buffer's own arena).
+ * Copies R offsets to the device on the stream of the last call and waits for it.
+ */
+int ubep_set_peers(ubep_buffer_t *buf, int32_t my_rank, void *const *peer_arenas /*[host]*/);
+
+/*
+ * Step 2 above.  x_local [dev] bf16 [T_local, H], the rank's own tokens in order; topk_idx,
+ * topk_w [dev]: the table of all T tokens.  Asynchronous on `cuda_stream`.
+ */
+int ubep_dispatch_sharded(ubep_buffer_t *buf, const void *x_local /*[dev]*/, const int32_t *topk_idx /*[dev]*/,
+                          const float *topk_w /*[dev]*/, int32_t T, void *cuda_stream);
+
+/* Step 3 above: one small launch on `cuda_stream` after the rank's own ubep_dispatch_sharded. */
+int ubep_wait_arrivals(ubep_buffer_t *buf, void *cuda_stream);
+
+/*
+ * out_local[t - t_begin] = bf16( sum_j topk_w[t][j] * y_r(j)[slot_row[t][j]] ) for the rank's
+ * own tokens; same arithmetic as ubep_combine.  y_peers [dev]: R device pointers, entry r =
+ * the expert-output buffer of rank r (bf16, laid out like the receive regions: [R, cap, H],
+ * of which rank r fills region r) as this GPU addresses it.  topk_w [dev]: all T tokens.
+ */
+int ubep_combine_sharded(ubep_buffer_t *buf, const void *const *y_peers /*[dev]*/, const float *topk_w /*[dev]*/,
+                         int32_t T, void *out_local /*[dev]*/, void *cuda_stream);
 
 /* Device address and shape (unused dims = 1) of one arena array; valid until destroy. */
 int ubep_view(ubep_buffer_t *buf, int which, void **dev_ptr /*[host]*/, int64_t shape[4] /*[host]*/);

@@ -34,10 +34,10 @@ UBEP_PIPELINE_AUTO, UBEP_PIPELINE_PHASED, UBEP_PIPELINE_FUSED, UBEP_PIPELINE_LOC
 
 VIEW_NAMES = ["recv_x", "recv_scale", "recv_src_idx", "recv_weight", "recv_topk_idx", "recv_topk_w",
               "expert_rows", "cnt", "src_offset", "expert_offset", "num_tokens_per_expert",
-              "num_rows_per_rank", "num_tokens_per_rank", "slot_row", "arrival", "epoch", "trace"]
+              "num_rows_per_rank", "num_tokens_per_rank", "slot_row", "arrival", "epoch", "trace", "shard_arrival"]
 _VIEW_DTYPES = [torch.uint8, torch.float32, torch.int32, torch.float32, torch.int32, torch.float32,
                 torch.int32, torch.int32, torch.int32, torch.int32, torch.int32, torch.int32, torch.int32,
-                torch.int32, torch.int32, torch.int32, torch.int64]
+                torch.int32, torch.int32, torch.int32, torch.int64, torch.int32]
 
 # every symbol include/ubep.h declares
 EXPORTS = ["ubep_buffer_bytes", "ubep_buffer_create", "ubep_buffer_destroy", "ubep_set_replicas",
@@ -46,7 +46,8 @@ EXPORTS = ["ubep_buffer_bytes", "ubep_buffer_create", "ubep_buffer_destroy", "ub
            "ubep_debug_set_quant_warps",
            "ubep_last_cuda_error", "ubep_strerror", "ubep_map_workers",
            "ubep_sync_wire_bytes", "ubep_sync_attach", "ubep_dispatch_sync", "ubep_sync_view",
-           "ubep_sync_scan_sentinel"]
+           "ubep_sync_scan_sentinel",
+           "ubep_set_peers", "ubep_dispatch_sharded", "ubep_wait_arrivals", "ubep_combine_sharded"]
 
 
 class ubep_config_t(ctypes.Structure):
@@ -100,6 +101,12 @@ def load() -> ctypes.CDLL:
     lib.ubep_sync_view.argtypes = [vp, ctypes.c_int, ctypes.POINTER(vp), ctypes.POINTER(ctypes.c_int64)]
     lib.ubep_sync_scan_sentinel.restype = ctypes.c_int
     lib.ubep_sync_scan_sentinel.argtypes = [vp, vp, i32, ctypes.POINTER(ctypes.c_int64), vp]
+    lib.ubep_set_peers.restype, lib.ubep_set_peers.argtypes = ctypes.c_int, [vp, i32, ctypes.POINTER(vp)]
+    lib.ubep_dispatch_sharded.restype = ctypes.c_int
+    lib.ubep_dispatch_sharded.argtypes = [vp, vp, vp, vp, i32, vp]
+    lib.ubep_wait_arrivals.restype, lib.ubep_wait_arrivals.argtypes = ctypes.c_int, [vp, vp]
+    lib.ubep_combine_sharded.restype = ctypes.c_int
+    lib.ubep_combine_sharded.argtypes = [vp, vp, vp, i32, vp, vp]
     _lib = lib
     return lib
 
@@ -265,20 +272,47 @@ def ubep_sync_scan_sentinel(buf, x: torch.Tensor, T: int, stream=None) -> int:
     return n.value
 
 
+def ubep_set_peers(buf, my_rank: int, peer_arena_ptrs) -> None:
+    """peer_arena_ptrs: R integers, the device address of every rank's arena as this GPU sees it."""
+    arr = (ctypes.c_void_p * len(peer_arena_ptrs))(*[int(v) for v in peer_arena_ptrs])
+    _check(load().ubep_set_peers(buf, my_rank, arr), "ubep_set_peers", buf)
+
+
+def ubep_dispatch_sharded(buf, x_local: torch.Tensor, topk_idx: torch.Tensor, topk_w: torch.Tensor, T: int,
+                          stream=None) -> None:
+    _check(load().ubep_dispatch_sharded(buf, _ptr(x_local), _ptr(topk_idx), _ptr(topk_w), T, _stream(stream)),
+           "ubep_dispatch_sharded", buf)
+
+
+def ubep_wait_arrivals(buf, stream=None) -> None:
+    _check(load().ubep_wait_arrivals(buf, _stream(stream)), "ubep_wait_arrivals", buf)
+
+
+def ubep_combine_sharded(buf, y_peers: torch.Tensor, topk_w: torch.Tensor, T: int, out_local: torch.Tensor,
+                         stream=None) -> None:
+    """y_peers: int64 device tensor of R addresses (every rank's expert-output buffer)."""
+    assert y_peers.dtype == torch.int64 and y_peers.is_cuda
+    _check(load().ubep_combine_sharded(buf, _ptr(y_peers), _ptr(topk_w), T, _ptr(out_local), _stream(stream)),
+           "ubep_combine_sharded", buf)
+
+
 # ------------------------------------------------------------------------ convenience
 
 class Buffer:
     """An arena tensor plus the library handle laid out inside it."""
 
     def __init__(self, *, num_ranks, num_experts, hidden, topk, max_tokens, rows_per_rank_cap,
-                 num_src_ranks=0, payload=0, dedup=0, device=0, pipeline=0, num_ctas=0, fill: Optional[int] = None):
+                 num_src_ranks=0, payload=0, dedup=0, device=0, pipeline=0, num_ctas=0, fill: Optional[int] = None,
+                 arena: Optional[torch.Tensor] = None):
         self.cfg = ubep_config_t(num_ranks, num_experts, hidden, topk, max_tokens, rows_per_rank_cap,
                                  num_src_ranks, payload, dedup, device, pipeline, num_ctas)
         nbytes = ubep_buffer_bytes(self.cfg)
         if nbytes == 0:
             raise UbepError(UBEP_ERR_ARG, "ubep_buffer_bytes")
         dev = torch.device("cuda", device)
-        self.arena = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+        if arena is not None:      # memory the caller obtained elsewhere (e.g. mapped for peer access)
+            assert arena.dtype == torch.uint8 and arena.numel() >= nbytes and arena.is_cuda
+        self.arena = arena if arena is not None else torch.empty(nbytes, dtype=torch.uint8, device=dev)
         if fill is not None:
             self.arena.fill_(fill)
         self.handle = ubep_buffer_create(self.cfg, self.arena)
@@ -293,7 +327,7 @@ class Buffer:
             rank = {"recv_x": 3, "recv_scale": 3, "recv_topk_idx": 3, "recv_topk_w": 3}.get(name)
             if rank is None:
                 rank = 1 if name in ("expert_offset", "num_tokens_per_expert", "num_rows_per_rank",
-                                     "num_tokens_per_rank", "epoch") else 2
+                                     "num_tokens_per_rank", "epoch", "shard_arrival") else 2
             shape = shape[:rank]
             n = 1
             for s in shape:

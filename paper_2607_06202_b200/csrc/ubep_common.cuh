@@ -82,6 +82,10 @@ struct Params {
     unsigned* claimed;    // [2] tokens handed out in this dispatch (half = epoch & 1)
     int32_t* status;
     unsigned long long* trace;  // optional [nchunks, kTraceSlots] globaltimer stamps, or null
+    // ranks on different GPUs (sharded use): this GPU is rank my_rank and moves tokens [tok0, tok1)
+    int my_rank, tok0, tok1;
+    const long long* peer_delta;  // [R] byte distance from this arena to the arena of rank r
+    unsigned* shard_arrival;      // [2] rows announced to this rank so far, rows expected so far
 };
 
 // ------------------------------------------------------------------ small helpers

@@ -10,6 +10,7 @@
 #include "../../include/ubep.h"
 #include "ubep_kernels.h"
 #include "ubep_sync.h"
+#include "ubep_sharded.h"
 
 using ubep::Params;
 
@@ -26,7 +27,7 @@ struct ArenaLayout {
     size_t off[UBEP_VIEW_COUNT_];
     size_t slot_pos, copy_pos, chunk_hist, partial, chunk_base, trace;
     size_t flags_begin, hist_flag, scan_flag, status, ticket, epoch_ctr, done_ticket, cursor, pos_flag, claimed,
-        order_pos, flags_end;
+        order_pos, flags_end, peer_delta;
     size_t total;
     int er_cap, nchunks, S, rowB, G, B;
 };
@@ -92,8 +93,10 @@ ArenaLayout make_layout(const ubep_config_t& c, int nchunks) {
     a.cursor = take(n * 4);
     a.pos_flag = take(n * 4);
     a.claimed = take(8);
+    a.off[UBEP_VIEW_SHARD_ARRIVAL] = take(8);
     a.flags_end = at;
     a.order_pos = take(R * 4);
+    a.peer_delta = take(R * 8);
     a.total = at;
     return a;
 }
@@ -142,6 +145,7 @@ struct ubep_buffer {
     const int32_t* phys;
     const int32_t* ncopies;
     int32_t E_log, C;
+    int32_t my_rank;    // sharded use (ubep_set_peers): this GPU's rank, -1 otherwise
     uint8_t* wire;      // readiness-protocol wire buffer (caller-owned) or null
     WireLayout wlay;
     bool sp_dirty;      // an earlier call may have left non-sentinel blocks in the SP wire
@@ -204,6 +208,11 @@ Params make_params(ubep_buffer* b, int T) {
     p.arrival = at<unsigned>(b, a.off[UBEP_VIEW_ARRIVAL]);
     p.status = at<int32_t>(b, a.status);
     p.trace = b->tracing ? at<unsigned long long>(b, a.trace) : nullptr;
+    p.my_rank = b->my_rank;
+    p.tok0 = 0;
+    p.tok1 = T;
+    p.peer_delta = at<long long>(b, a.peer_delta);
+    p.shard_arrival = at<unsigned>(b, a.off[UBEP_VIEW_SHARD_ARRIVAL]);
     return p;
 }
 
@@ -261,6 +270,7 @@ int ubep_buffer_create(const ubep_config_t* cfg, void* dev_arena, size_t bytes, 
     b->ncopies = nullptr;
     b->E_log = 0;
     b->C = 0;
+    b->my_rank = -1;
     b->wire = nullptr;
     b->wlay = WireLayout{};
     b->sp_dirty = false;
@@ -531,6 +541,96 @@ int ubep_sync_scan_sentinel(ubep_buffer_t* buf, const void* x, int32_t T, int64_
     return UBEP_OK;
 }
 
+int ubep_set_peers(ubep_buffer_t* buf, int32_t my_rank, void* const* peer_arenas) {
+    if (!buf || !peer_arenas || my_rank < 0 || my_rank >= buf->cfg.num_ranks) return UBEP_ERR_ARG;
+    const int R = buf->cfg.num_ranks;
+    if (buf->lay.S != R || buf->cfg.payload != UBEP_PAYLOAD_BF16) return UBEP_ERR_ARG;   // one source rank per GPU
+    if (peer_arenas[my_rank] != buf->arena) return UBEP_ERR_ARG;
+    std::vector<long long> delta(R);
+    for (int r = 0; r < R; ++r) {
+        if (!peer_arenas[r] || (reinterpret_cast<uintptr_t>(peer_arenas[r]) & (kAlign - 1)) != 0) return UBEP_ERR_ARENA;
+        delta[r] = (long long)(reinterpret_cast<intptr_t>(peer_arenas[r]) - reinterpret_cast<intptr_t>(buf->arena));
+    }
+    DeviceGuard guard(buf->cfg.device);
+    if (guard.err != cudaSuccess) return cuda_fail(buf, guard.err);
+    cudaError_t e = cudaMemcpyAsync(buf->arena + buf->lay.peer_delta, delta.data(), sizeof(long long) * R,
+                                    cudaMemcpyHostToDevice, buf->last_stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(buf->last_stream);
+    if (e != cudaSuccess) return cuda_fail(buf, e);
+    buf->my_rank = my_rank;
+    return UBEP_OK;
+}
+
+int ubep_dispatch_sharded(ubep_buffer_t* buf, const void* x_local, const int32_t* topk_idx, const float* topk_w,
+                          int32_t T, void* cuda_stream) {
+    if (!buf || buf->my_rank < 0) return UBEP_ERR_ARG;
+    if (T < 0 || T > buf->cfg.max_tokens || (int64_t)T * buf->cfg.topk > kLocalMaxSlots) return UBEP_ERR_ARG;
+    if (T > 0 && (!topk_idx || !topk_w)) return UBEP_ERR_ARG;
+    if (!aligned16(x_local) || !aligned16(topk_idx) || !aligned16(topk_w)) return UBEP_ERR_ARG;
+    DeviceGuard guard(buf->cfg.device);
+    if (guard.err != cudaSuccess) return cuda_fail(buf, guard.err);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    buf->last_stream = st;
+    if (T == 0) {
+        const size_t lo = buf->lay.off[UBEP_VIEW_CNT], hi = buf->lay.off[UBEP_VIEW_SLOT_ROW];
+        cudaError_t e0 = cudaMemsetAsync(buf->arena + lo, 0, hi - lo, st);
+        return e0 == cudaSuccess ? UBEP_OK : cuda_fail(buf, e0);
+    }
+    Params p = make_params(buf, T);
+    const int R = buf->cfg.num_ranks;
+    p.tok0 = (int)((int64_t)buf->my_rank * T / R);
+    p.tok1 = (int)((int64_t)(buf->my_rank + 1) * T / R);
+    if (p.tok1 > p.tok0 && !x_local) return UBEP_ERR_ARG;
+    p.x = static_cast<const uint16_t*>(x_local);
+    p.topk_idx = topk_idx;
+    p.topk_w = topk_w;
+    p.trace = nullptr;
+    p.parts = 1;
+    p.grid = p.nchunks;
+    ubep::SmemPlan pl{};
+    if (ubep::plan_dispatch(p, UBEP_PIPELINE_LOCAL, buf->max_smem - ubep::sharded_extra_smem(p), &pl) != 0)
+        return UBEP_ERR_ARG;
+    cudaError_t e = ubep::launch_sharded_dispatch(p, pl, st);
+    if (e != cudaSuccess) return cuda_fail(buf, e);
+    g_launches += 1;
+    return UBEP_OK;
+}
+
+int ubep_wait_arrivals(ubep_buffer_t* buf, void* cuda_stream) {
+    if (!buf || buf->my_rank < 0) return UBEP_ERR_ARG;
+    DeviceGuard guard(buf->cfg.device);
+    if (guard.err != cudaSuccess) return cuda_fail(buf, guard.err);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    buf->last_stream = st;
+    cudaError_t e = ubep::launch_wait_arrivals(at<unsigned>(buf, buf->lay.off[UBEP_VIEW_SHARD_ARRIVAL]),
+                                               at<int32_t>(buf, buf->lay.status), st);
+    if (e != cudaSuccess) return cuda_fail(buf, e);
+    g_launches += 1;
+    return UBEP_OK;
+}
+
+int ubep_combine_sharded(ubep_buffer_t* buf, const void* const* y_peers, const float* topk_w, int32_t T,
+                         void* out_local, void* cuda_stream) {
+    if (!buf || buf->my_rank < 0 || T < 0 || T > buf->cfg.max_tokens) return UBEP_ERR_ARG;
+    if (T == 0) return UBEP_OK;
+    const int R = buf->cfg.num_ranks;
+    const int tok0 = (int)((int64_t)buf->my_rank * T / R), tok1 = (int)((int64_t)(buf->my_rank + 1) * T / R);
+    if (!y_peers || !topk_w || (tok1 > tok0 && !out_local)) return UBEP_ERR_ARG;
+    if (!aligned16(topk_w) || !aligned16(out_local) || (reinterpret_cast<uintptr_t>(y_peers) & 7u) != 0) return UBEP_ERR_ARG;
+    if (tok1 == tok0) return UBEP_OK;
+    DeviceGuard guard(buf->cfg.device);
+    if (guard.err != cudaSuccess) return cuda_fail(buf, guard.err);
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    buf->last_stream = st;
+    cudaError_t e = ubep::launch_sharded_combine(reinterpret_cast<const uint16_t* const*>(y_peers),
+                                                 at<int32_t>(buf, buf->lay.slot_pos), topk_w, tok0, tok1,
+                                                 buf->cfg.hidden, buf->cfg.topk, buf->cfg.rows_per_rank_cap,
+                                                 static_cast<uint16_t*>(out_local), buf->num_sms, st);
+    if (e != cudaSuccess) return cuda_fail(buf, e);
+    g_launches += 1;
+    return UBEP_OK;
+}
+
 int ubep_view(ubep_buffer_t* buf, int which, void** dev_ptr, int64_t shape[4]) {
     if (!buf || !dev_ptr || !shape || which < 0 || which >= UBEP_VIEW_COUNT_) return UBEP_ERR_ARG;
     const ubep_config_t& c = buf->cfg;
@@ -556,6 +656,7 @@ int ubep_view(ubep_buffer_t* buf, int which, void** dev_ptr, int64_t shape[4]) {
         case UBEP_VIEW_ARRIVAL: s[0] = 2; s[1] = R; break;
         case UBEP_VIEW_EPOCH: s[0] = 1; break;
         case UBEP_VIEW_TRACE: s[0] = a.nchunks; s[1] = ubep::kTraceSlots; break;
+        case UBEP_VIEW_SHARD_ARRIVAL: s[0] = 2; break;
         default: return UBEP_ERR_ARG;
     }
     if (!present) {

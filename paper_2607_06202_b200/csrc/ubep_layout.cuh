@@ -274,10 +274,17 @@ static __device__ void scan_rank_sources(const Params& p, int r, const int* sm, 
 // global row to copy to (rank * cap + row), or -1, and in dst_key[] the place of that row's
 // rank in the destination-ordering table rotated by the worker id (R for "no copy").
 // w_sm: the tokens' gate weights, staged.  (Rows per rank are counted by whoever copies them.)
-template <typename RowsE, typename RowsR>
+// kPeers (ranks on different GPUs, arenas of identical layout): what belongs to the receiver
+// of a row -- its metadata and its expert row list -- is written into the arena of that rank,
+// peer_delta[r] bytes away from this GPU's own.
+template <bool kPeers, typename T>
+__device__ __forceinline__ T* toward_peer(T* ptr, long long delta) {
+    return kPeers ? reinterpret_cast<T*>(reinterpret_cast<char*>(ptr) + delta) : ptr;
+}
+template <bool kPeers = false, typename RowsE, typename RowsR>
 __device__ void finalize_chunk(const Params& p, int t0, int t1, const int* ids, const float* w_sm, RowsE rows_e,
                                RowsR rows_r, bool write_meta, int worker, const int* order_sm, int* pos,
-                               int* dst_key, int* arr, int gtid, int gn) {
+                               int* dst_key, int* arr, int gtid, int gn, const long long* peer_delta = nullptr) {
     const int k = p.k, L = p.L, R = p.R;
     const int rot = worker % R;
     const int nslots = (t1 - t0) * k;
@@ -290,6 +297,7 @@ __device__ void finalize_chunk(const Params& p, int t0, int t1, const int* ids, 
         if (packed >= 0) {
             const int e = slot_expert(packed);
             r = slot_rank(packed);
+            const long long pd = kPeers ? peer_delta[r] : 0;
             bool first = true;
             if (!p.dedup) {
                 row = rows_e(e, tl);
@@ -301,7 +309,7 @@ __device__ void finalize_chunk(const Params& p, int t0, int t1, const int* ids, 
                 row = rows_r(r, tl);
                 if (write_meta) {
                     const int at = rows_e(e, tl);
-                    if (at < p.er_cap) p.expert_rows[(size_t)r * p.er_cap + at] = row;
+                    if (at < p.er_cap) toward_peer<kPeers>(p.expert_rows, pd)[(size_t)r * p.er_cap + at] = row;
                     else report(p.status, kErrCapacity);
                 }
             }
@@ -313,16 +321,17 @@ __device__ void finalize_chunk(const Params& p, int t0, int t1, const int* ids, 
                     where = gpos;
                     if (arr) atomicAdd(&arr[r], 1);   // rows this CTA will copy to rank r (null: counted at copy time)
                     if (write_meta) {
-                        p.recv_src_idx[where] = t;
+                        toward_peer<kPeers>(p.recv_src_idx, pd)[where] = t;
                         if (!p.dedup) {
-                            p.recv_weight[where] = w_sm[li];
+                            toward_peer<kPeers>(p.recv_weight, pd)[where] = w_sm[li];
                         } else {
                             const int* row_ids = ids + tl * k;
                             for (int jj = 0; jj < k; ++jj) {
                                 const int v2 = row_ids[jj];
                                 const bool here = v2 >= 0 && slot_rank(v2) == r;
-                                p.recv_topk_idx[(size_t)where * k + jj] = here ? slot_expert(v2) - r * L : -1;
-                                p.recv_topk_w[(size_t)where * k + jj] =
+                                toward_peer<kPeers>(p.recv_topk_idx, pd)[(size_t)where * k + jj] =
+                                    here ? slot_expert(v2) - r * L : -1;
+                                toward_peer<kPeers>(p.recv_topk_w, pd)[(size_t)where * k + jj] =
                                     here ? w_sm[tl * k + jj] : 0.0f;
                             }
                         }

@@ -82,6 +82,10 @@ def test_null_arguments_are_rejected_without_a_gpu(lib):
     assert lib.ubep_dispatch_sync(None, 0, None, None, None, 0, None) == B.UBEP_ERR_ARG
     assert lib.ubep_sync_view(None, 0, None, None) == B.UBEP_ERR_ARG
     assert lib.ubep_sync_scan_sentinel(None, None, 0, None, None) == B.UBEP_ERR_ARG
+    assert lib.ubep_set_peers(None, 0, None) == B.UBEP_ERR_ARG
+    assert lib.ubep_dispatch_sharded(None, None, None, None, 0, None) == B.UBEP_ERR_ARG
+    assert lib.ubep_wait_arrivals(None, None) == B.UBEP_ERR_ARG
+    assert lib.ubep_combine_sharded(None, None, None, 0, None, None) == B.UBEP_ERR_ARG
 
 
 def test_wire_bytes_of_the_readiness_protocols(lib):
