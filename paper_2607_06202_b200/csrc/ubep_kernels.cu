@@ -86,7 +86,8 @@ struct Cta {
     float* w_sm;
     BinMaps bmaps;
     int *hist, *arr, *order_sm;
-    unsigned epoch, in_bytes, out_bytes;
+    unsigned epoch, in_bytes, out_bytes;   // (epoch: 0 in the flag-free kernel, which reads it late into *epoch_late)
+    unsigned* epoch_late;
     size_t in_off, out_off;
     bool fast_local;
     int issued;   // rows whose load the mover has started (thread 0's copy is used when leaving early)
@@ -393,6 +394,7 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
         if (gtid == 0) {
             mbar_arrive(&ready_bar);
             trace(p, c, kTrReady);
+            *x.epoch_late = read_epoch_and_check_in(p);   // nothing needs it before the kernel's last lines
         }
         if (part == 0) {
             float* w_own = reinterpret_cast<float*>(key);   // the ordering keys are no longer needed
@@ -445,6 +447,7 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
         if (gtid == 0) {
             mbar_arrive(&ready_bar);
             trace(p, c, kTrReady);
+            *x.epoch_late = read_epoch_and_check_in(p);   // nothing needs it before the kernel's last lines
         }
         // outputs nobody inside this kernel waits for
         if (c == 0) {
@@ -721,9 +724,11 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
     }
     for (int r = tid; r < p.R; r += kThreads) arr[r] = 0;
     griddep_wait();     // shared-memory set-up done; everything below reads what earlier kernels wrote
-    if (tid == 0) epoch_sm = read_epoch_and_check_in(p);
+    // The flag-free kernel uses the epoch only for the arrival counters at its very end, so there it
+    // is read after the movers have been released instead of in front of everything.
+    if (kMode != kModeLocal && tid == 0) epoch_sm = read_epoch_and_check_in(p);
     __syncthreads();
-    const unsigned epoch = epoch_sm;
+    const unsigned epoch = kMode == kModeLocal ? 0u : epoch_sm;
     if (tid == 0) trace(p, c, kTrStart);
 
     const unsigned in_bytes = (unsigned)(p.H * 2 / p.parts);   // this CTA's piece of a bf16 row
@@ -738,7 +743,7 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
           BinMaps{reinterpret_cast<unsigned*>(smem + pl.off_mask), reinterpret_cast<unsigned*>(smem + pl.off_bm),
                   pl.map_wb, pl.map_bp, pl.map_groups},
           reinterpret_cast<int*>(smem + pl.off_hist), arr, reinterpret_cast<int*>(smem + pl.off_order),
-          epoch, in_bytes, out_bytes, (size_t)part * in_bytes, (size_t)part * out_bytes,
+          epoch, in_bytes, out_bytes, &epoch_sm, (size_t)part * in_bytes, (size_t)part * out_bytes,
           kMode == kModeLocal && p.local_fast != 0, 0};
 
     if (x.warp == 0) {
@@ -759,12 +764,13 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
     // pieces of this CTA's rows have landed: add them to the per-region arrival counters
     // (unit: eighths of a row, so that the total does not depend on the column split)
     fence_proxy_async();   // rows written through the async proxy, counters through the generic one
+    const unsigned half = (kMode == kModeLocal ? epoch_sm : epoch) & 1u;
     for (int r = tid; r < p.R; r += kThreads)
-        if (arr[r]) red_release_add(p.arrival + (epoch & 1) * p.R + r, (unsigned)(arr[r] * (8 / p.parts)));
+        if (arr[r]) red_release_add(p.arrival + half * p.R + r, (unsigned)(arr[r] * (8 / p.parts)));
     // the arrival counters of the next call live in the other half; clear them now
     if (c == 0) {
-        for (int r = tid; r < p.R; r += kThreads) p.arrival[((epoch + 1) & 1) * p.R + r] = 0;
-        if (tid == 0) p.claimed[(epoch + 1) & 1] = 0;   // same for the count of tokens handed out
+        for (int r = tid; r < p.R; r += kThreads) p.arrival[(half ^ 1u) * p.R + r] = 0;
+        if (tid == 0) p.claimed[half ^ 1u] = 0;   // same for the count of tokens handed out
     }
     if (tid == 0) trace(p, c, kTrEnd);
 }
