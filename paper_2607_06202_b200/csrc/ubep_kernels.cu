@@ -79,14 +79,14 @@ struct Cta {
     const Params& p;
     const SmemPlan& pl;
     uint8_t* smem;
-    uint64_t *full_bar, *empty_bar, *out_full, *out_empty, *ready_bar;
+    uint64_t *full_bar, *empty_bar, *out_full, *out_empty, *ready_bar, *epoch_bar;
     int* abort_flag;
     int tid, lane, warp, c, part, ch, t0, t1, ntok, stages, nq;
     int *ids_sm, *pos, *pos_raw, *key;
     float* w_sm;
     BinMaps bmaps;
     int *hist, *arr, *order_sm;
-    unsigned epoch, in_bytes, out_bytes;   // (epoch: 0 in the flag-free kernel, which reads it late into *epoch_late)
+    unsigned epoch, in_bytes, out_bytes;   // (epoch: 0 until the role that needs it has learnt it from *epoch_late)
     unsigned* epoch_late;
     size_t in_off, out_off;
     bool fast_local;
@@ -130,6 +130,17 @@ struct Cta {
 // so the k copies of a row are issued side by side; for FP8 rows the warp only loads.
 template <int kMode, bool kFp8, bool kSteal>
 __device__ __forceinline__ void mover_warp(Cta& x) {
+    if (kMode != kModeLocal) {
+        // The epoch: one acquire load and one ticket, two round trips to L2.  This warp has nothing
+        // urgent to do yet, so it fetches it while the layout group already stages the routing table.
+        unsigned ep = 0;
+        if (x.lane == 0) {
+            ep = read_epoch_and_check_in(x.p);
+            *x.epoch_late = ep;
+            mbar_arrive(x.epoch_bar);
+        }
+        x.epoch = __shfl_sync(0xffffffffu, ep, 0);
+    }
     UBEP_CTA_LOCALS(x);
     // Lane 0 issues the TMA loads; for bf16 rows lane j issues the TMA store of slot j,
     // so the k copies of a row are issued side by side.  Tokens come from a feeder: the
@@ -480,13 +491,21 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
         build_bin_maps(p, ids_sm, ntok, bmaps, gw, nw, lane);
         group_sync(1, gn);
         int deferred = -1;
+        // The mover warp fetched the epoch while the table was staged; one thread makes sure it has
+        // arrived, the barrier that follows hands it to the others.
+        unsigned ep = 0;
+        auto learn_epoch = [&]() {
+            if (gtid == 0) (void)mbar_wait(x.epoch_bar, 0, abortp);
+            group_sync(1, gn);
+            ep = *reinterpret_cast<volatile unsigned*>(x.epoch_late);
+        };
         if (kMode == kModeFused) {
             publish_chunk_counts(p, ch, t0, t1, bmaps, gtid, gn);
-            group_sync(1, gn);
+            learn_epoch();
             if (gtid == 0) {
                 if (ch != p.withhold) {
                     __threadfence();
-                    st_release(p.hist_flag + ch, epoch);
+                    st_release(p.hist_flag + ch, ep);
                 }
                 trace(p, c, kTrCounted);
             }
@@ -494,13 +513,13 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
             bool lost = false;  // a wait of this thread ran out
             for (int r = ch; r < p.R; r += p.nchunks) {
                 for (int cc = gtid; cc < p.nchunks; cc += gn)
-                    if (!wait_flag(p.hist_flag + cc, epoch, abortp)) lost = true;
+                    if (!wait_flag(p.hist_flag + cc, ep, abortp)) lost = true;
                 if (group_or(1, gn, lost || *abortp)) { lost = true; break; }  // same answer for all
                 if (gtid == 0) trace(p, c, kTrHistSeen);
                 scan_rank_publish(p, r, hist, gw, nw, lane, 1);
                 if (gtid == 0) {
                     __threadfence();
-                    st_release(p.scan_flag + r, epoch);
+                    st_release(p.scan_flag + r, ep);
                     trace(p, c, kTrScanned);
                 }
                 if (r + p.nchunks < p.R) {
@@ -513,7 +532,7 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
             // every slot of this chunk may need any rank's bases
             if (!lost)
                 for (int r = gtid; r < p.R; r += gn)
-                    if (!wait_flag(p.scan_flag + r, epoch, abortp)) lost = true;
+                    if (!wait_flag(p.scan_flag + r, ep, abortp)) lost = true;
             ok = !group_or(1, gn, lost || *abortp);
             if (gtid == 0) trace(p, c, kTrScanSeen);
             if (!ok && gtid == 0) {
@@ -547,10 +566,11 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
         if (ok && kSteal) {
             // this chunk's destinations, for CTAs that run out of work and take over some of its tokens
             for (int i = gtid; i < ntok * p.k; i += gn) p.copy_pos[(size_t)t0 * p.k + i] = pos[i];
-            group_sync(1, gn);
+            if (kMode == kModeFused) group_sync(1, gn);
+            else learn_epoch();   // (with kernel boundaries instead of flags nothing has asked for it yet)
             if (gtid == 0) {
                 __threadfence();
-                st_release(p.pos_flag + ch, epoch);
+                st_release(p.pos_flag + ch, ep);
             }
         }
         if (ok && deferred >= 0) scan_rank_sources(p, deferred, hist, gtid, gn);
@@ -697,6 +717,7 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
     __shared__ __align__(8) uint64_t out_full[kOutStages];    // FP8: quantised row written
     __shared__ __align__(8) uint64_t out_empty[kOutStages];   // FP8: its stores have read it
     __shared__ __align__(8) uint64_t ready_bar;               // rows assigned, movers may go
+    __shared__ __align__(8) uint64_t epoch_bar;               // epoch_sm holds this launch's epoch
     __shared__ int abort_flag;
     __shared__ unsigned epoch_sm;
 
@@ -719,21 +740,22 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
             mbar_init(&out_empty[s], 1);
         }
         mbar_init(&ready_bar, 1);
+        mbar_init(&epoch_bar, 1);
         abort_flag = 0;
         mbar_fence_init();
     }
     for (int r = tid; r < p.R; r += kThreads) arr[r] = 0;
     griddep_wait();     // shared-memory set-up done; everything below reads what earlier kernels wrote
-    // The flag-free kernel uses the epoch only for the arrival counters at its very end, so there it
-    // is read after the movers have been released instead of in front of everything.
-    if (kMode != kModeLocal && tid == 0) epoch_sm = read_epoch_and_check_in(p);
+    // The epoch is not read here, in front of everything: the flag-free kernel needs it only for the
+    // arrival counters at its very end and reads it once the movers are released; in the other
+    // kernels the mover warp fetches it while the layout group stages the routing table.
     __syncthreads();
-    const unsigned epoch = kMode == kModeLocal ? 0u : epoch_sm;
+    const unsigned epoch = 0u;
     if (tid == 0) trace(p, c, kTrStart);
 
     const unsigned in_bytes = (unsigned)(p.H * 2 / p.parts);   // this CTA's piece of a bf16 row
     const unsigned out_bytes = (unsigned)(p.rowB / p.parts);   // and of a payload row
-    Cta x{p, pl, smem, full_bar, empty_bar, out_full, out_empty, &ready_bar, &abort_flag,
+    Cta x{p, pl, smem, full_bar, empty_bar, out_full, out_empty, &ready_bar, &epoch_bar, &abort_flag,
           tid, tid & 31, tid >> 5, c, part, ch, t0, t1, t1 - t0, stages, nq,
           reinterpret_cast<int*>(smem + pl.off_ids),
           reinterpret_cast<int*>(smem + pl.off_ord),    // destinations in issue order
@@ -764,7 +786,7 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
     // pieces of this CTA's rows have landed: add them to the per-region arrival counters
     // (unit: eighths of a row, so that the total does not depend on the column split)
     fence_proxy_async();   // rows written through the async proxy, counters through the generic one
-    const unsigned half = (kMode == kModeLocal ? epoch_sm : epoch) & 1u;
+    const unsigned half = epoch_sm & 1u;
     for (int r = tid; r < p.R; r += kThreads)
         if (arr[r]) red_release_add(p.arrival + half * p.R + r, (unsigned)(arr[r] * (8 / p.parts)));
     // the arrival counters of the next call live in the other half; clear them now
