@@ -504,8 +504,7 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
             learn_epoch();
             if (gtid == 0) {
                 if (ch != p.withhold) {
-                    __threadfence();
-                    st_release(p.hist_flag + ch, ep);
+                    st_release(p.hist_flag + ch, ep);   // release: cumulative over what the barrier above ordered
                 }
                 trace(p, c, kTrCounted);
             }
@@ -518,7 +517,6 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
                 if (gtid == 0) trace(p, c, kTrHistSeen);
                 scan_rank_publish(p, r, hist, gw, nw, lane, 1);
                 if (gtid == 0) {
-                    __threadfence();
                     st_release(p.scan_flag + r, ep);
                     trace(p, c, kTrScanned);
                 }
@@ -569,7 +567,6 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
             if (kMode == kModeFused) group_sync(1, gn);
             else learn_epoch();   // (with kernel boundaries instead of flags nothing has asked for it yet)
             if (gtid == 0) {
-                __threadfence();
                 st_release(p.pos_flag + ch, ep);
             }
         }
