@@ -312,36 +312,68 @@ def run_ours(args, cfg, rank: int, world: int, local_rank: int):
     disp_us, comb_us = kernel_us("dispatch"), kernel_us("combine")
 
     # end to end through the C ABI with host buffers: pinned inputs -> device -> dispatch ->
-    # combine over identity experts (bf16 payload) or the synthetic y (FP8) -> host
-    hx = torch.from_numpy(wl.x).view(torch.bfloat16).pin_memory()
-    hidx = torch.from_numpy(wl.topk_idx.astype(np.int32)).pin_memory()
-    hw = torch.from_numpy(wl.topk_w).pin_memory()
+    # combine over identity experts (bf16 payload) or the synthetic y (FP8) -> host.  Every step
+    # copies its own inputs in and its own result out; the copies run on streams of their own, so
+    # step n's result leaves and step n + 2's inputs arrive while step n + 1 computes (what a caller
+    # that feeds the library from host memory would do).  Inputs travel as one pinned block.
+    def aligned(n):
+        return (n + 255) // 256 * 256
+    nx, nidx, nw_ = cfg.T * cfg.H * 2, cfg.T * cfg.k * 4, cfg.T * cfg.k * 4
+    off_idx, off_w = aligned(nx), aligned(nx) + aligned(nidx)
+    block_bytes = off_w + aligned(nw_)
+    hin = torch.empty(block_bytes, dtype=torch.uint8).pin_memory()
+    hin[:nx] = torch.from_numpy(wl.x).view(torch.uint8).reshape(-1)
+    hin[off_idx:off_idx + nidx] = torch.from_numpy(wl.topk_idx.astype(np.int32)).view(torch.uint8).reshape(-1)
+    hin[off_w:off_w + nw_] = torch.from_numpy(wl.topk_w.astype(np.float32)).view(torch.uint8).reshape(-1)
     hout = torch.empty((cfg.T, cfg.H), dtype=torch.bfloat16).pin_memory()
+    for s in sets:
+        blk = torch.empty(block_bytes, dtype=torch.uint8, device=dev)
+        s["in_block"] = blk
+        s["ex"] = blk[:nx].view(torch.bfloat16).view(cfg.T, cfg.H)
+        s["eidx"] = blk[off_idx:off_idx + nidx].view(torch.int32).view(cfg.T, cfg.k)
+        s["ew"] = blk[off_w:off_w + nw_].view(torch.float32).view(cfg.T, cfg.k)
+        s["ev_in"], s["ev_cmp"], s["ev_out"] = (torch.cuda.Event() for _ in range(3))
+    s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
     n_e = min(args.steps, 200)
     ee0, ee1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
-    def e2e_step(s):
-        s["x"].copy_(hx, non_blocking=True)
-        s["idx"].copy_(hidx, non_blocking=True)
-        s["w"].copy_(hw, non_blocking=True)
-        B.ubep_dispatch(s["buf"].handle, s["x"], s["idx"], s["w"], cfg.T, stream)
+    def e2e_step(s, first_use):
+        if not first_use:
+            s_in.wait_event(s["ev_cmp"])        # the set's last dispatch / combine have read its inputs
+        with torch.cuda.stream(s_in):
+            s["in_block"].copy_(hin, non_blocking=True)
+            s["ev_in"].record(s_in)
+        stream.wait_event(s["ev_in"])
+        if not first_use:
+            stream.wait_event(s["ev_out"])      # the set's last result has left
+        B.ubep_dispatch(s["buf"].handle, s["ex"], s["eidx"], s["ew"], cfg.T, stream)
         yy = s["y"] if cfg.payload else s["buf"].recv_x.view(torch.bfloat16).view(cfg.R, cap, cfg.H)
-        B.ubep_combine(s["buf"].handle, yy, s["w"], cfg.T, s["out"], stream)
-        hout.copy_(s["out"], non_blocking=True)
+        B.ubep_combine(s["buf"].handle, yy, s["ew"], cfg.T, s["out"], stream)
+        s["ev_cmp"].record(stream)
+        s_out.wait_event(s["ev_cmp"])
+        with torch.cuda.stream(s_out):
+            hout.copy_(s["out"], non_blocking=True)
+            s["ev_out"].record(s_out)
 
-    with torch.cuda.stream(stream):
-        for i in range(3):
-            e2e_step(sets[i % nsets])
+    torch.cuda.synchronize(dev)
+    e2e_step(sets[0], True)
+    torch.cuda.synchronize(dev)
+    e2e_ref = hout.clone()                       # one step alone, to compare the pipelined steps with
+    for i in range(1, nsets + 3):                # warm-up: every set used once, then the steady pattern
+        e2e_step(sets[i % nsets], i < nsets)
+    torch.cuda.synchronize(dev)
     barrier()
-    with torch.cuda.stream(stream):
-        ee0.record(stream)
-        for i in range(n_e):
-            e2e_step(sets[i % nsets])
-        ee1.record(stream)
+    ee0.record(s_in)
+    for i in range(n_e):
+        e2e_step(sets[i % nsets], False)
+    ee1.record(s_out)
+    torch.cuda.synchronize(dev)
     barrier()
     e2e_ms = ee0.elapsed_time(ee1) / n_e
+    # every set holds the same inputs, so what came back last must be what the first step computed
+    assert torch.equal(hout.view(torch.int16), e2e_ref.view(torch.int16)), "end-to-end result differs"
     e2e_ms = max_over_ranks(e2e_ms, world, dev)
-    h2d = hx.numel() * 2 + hidx.numel() * 4 + hw.numel() * 4
+    h2d = block_bytes
     d2h = hout.numel() * 2
     e2e = {"value": whole_job_value(disp_b + comb_b, e2e_ms, world), "unit": "GB/s",
            "us_per_layer": e2e_ms * 1e3, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
