@@ -228,13 +228,19 @@ __device__ __forceinline__ void mover_warp(Cta& x) {
         ++head;
     };
     if (kSteal && lane == 0) p.cursor[ch] = 0;   // before anybody can claim from this chunk
+    // Rows fetched before the layout is done.  With flags the layout takes many microseconds in which a
+    // few small loads and stores of every CTA wait on one another; a ring-full of rows per CTA fetched
+    // meanwhile fills the memory system's queues in front of them.  Three rows start the copies, the
+    // rest follows once the movers are released.  (Not with stealing: there every block of rows costs a
+    // claim, a round trip each, and those are best paid while the layout runs.)
+    const int early = (kMode == kModeLocal || kSteal) ? kMaxStages : 3;
     if (!kFp8) {
         // loads run (stages - 3) rows ahead; up to 3 rows' stores stay in flight
         int tl = 0;
         if (kSteal) {
-            while (head < stages - 3 && next_token(tl, false) == 1) issue_item(tl);
+            while (head < min(stages - 3, early) && next_token(tl, false) == 1) issue_item(tl);
         } else {
-            while (head < min(stages - 3, ntok)) issue_item(head);
+            while (head < min(min(stages - 3, early), ntok)) issue_item(head);
         }
         issued = head;
         if (fast_local) {
@@ -245,6 +251,14 @@ __device__ __forceinline__ void mover_warp(Cta& x) {
         }
         ok = mbar_wait(&ready_bar, 0, abortp) && !*abortp;  // no rows without a layout
         ok = __all_sync(0xffffffffu, ok);
+        if (kMode != kModeLocal && ok) {   // the rest of the ring
+            if (kSteal) {
+                while (head < stages - 3 && next_token(tl, false) == 1) issue_item(tl);
+            } else {
+                while (head < min(stages - 3, ntok)) issue_item(head);
+            }
+            issued = head;
+        }
         if (!kSteal) {
             // the CTA's own rows, in order: row n sits in stage n % stages
             for (int n = 0; ok && n < ntok; ++n) {
@@ -314,6 +328,11 @@ __device__ __forceinline__ void mover_warp(Cta& x) {
         if (!kSteal) {
             // the CTA's own rows only: one thread, as far ahead as the ring allows
             while (ok && head < ntok) {
+                if (kMode != kModeLocal && head == early) {   // the rest once the layout is done
+                    if (lane == 0) ok = mbar_wait(&ready_bar, 0, abortp);
+                    ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+                    if (!ok) break;
+                }
                 if (head >= stages) {
                     if (lane == 0) ok = mbar_wait(&empty_bar[head % stages], ((head / stages) - 1) & 1, abortp);
                     ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
@@ -331,6 +350,11 @@ __device__ __forceinline__ void mover_warp(Cta& x) {
                 const int hs = head - 3;
                 drained = mbar_test_wait(&empty_bar[hs % stages], (hs / stages) & 1);
                 drained = __all_sync(0xffffffffu, drained);
+            }
+            if (head == early) {   // the rest once the layout is done
+                ok = mbar_wait(&ready_bar, 0, abortp);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
             }
             const int got = feeder_done ? 0 : next_token(tl, drained);
             if (got == 2) {
