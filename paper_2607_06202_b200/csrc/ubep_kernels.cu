@@ -79,7 +79,7 @@ struct Cta {
     const Params& p;
     const SmemPlan& pl;
     uint8_t* smem;
-    uint64_t *full_bar, *empty_bar, *out_full, *out_empty, *ready_bar, *epoch_bar;
+    uint64_t *full_bar, *empty_bar, *out_full, *out_empty, *ready_bar, *epoch_bar, *staged_bar;
     int* abort_flag;
     int tid, lane, warp, c, part, ch, t0, t1, ntok, stages, nq;
     int *ids_sm, *pos, *pos_raw, *key;
@@ -237,18 +237,23 @@ __device__ __forceinline__ void mover_warp(Cta& x) {
     if (!kFp8) {
         // loads run (stages - 3) rows ahead; up to 3 rows' stores stay in flight
         int tl = 0;
+        // Flag-free kernel: the routing table first, the rows after it.  The table is the one load the
+        // whole layout waits for; the rows of 148 CTAs queued in front of it cost about a microsecond.
+        if (fast_local) {
+            // lend a hand with the routing table
+            const RankMaps rm{bmaps.bm, bmaps.mask_t, (p.R + 31) / 32, ((p.R + 31) / 32) * 32, (p.T + 31) / 32};
+            local_stage_and_rank_maps(p, ids_sm, rm, 0, kWarps, lane);
+            group_sync(2, kThreads);
+        } else if (kMode == kModeLocal) {
+            ok = mbar_wait(x.staged_bar, 0, abortp);
+            ok = __all_sync(0xffffffffu, ok);
+        }
         if (kSteal) {
             while (head < min(stages - 3, early) && next_token(tl, false) == 1) issue_item(tl);
         } else {
             while (head < min(min(stages - 3, early), ntok)) issue_item(head);
         }
         issued = head;
-        if (fast_local) {
-            // lend a hand with the routing table, then wait for the layout group
-            const RankMaps rm{bmaps.bm, bmaps.mask_t, (p.R + 31) / 32, ((p.R + 31) / 32) * 32, (p.T + 31) / 32};
-            local_stage_and_rank_maps(p, ids_sm, rm, 0, kWarps, lane);
-            group_sync(2, kThreads);
-        }
         ok = mbar_wait(&ready_bar, 0, abortp) && !*abortp;  // no rows without a layout
         ok = __all_sync(0xffffffffu, ok);
         if (kMode != kModeLocal && ok) {   // the rest of the ring
@@ -316,11 +321,11 @@ __device__ __forceinline__ void mover_warp(Cta& x) {
     } else {
         if (fast_local) {
             const RankMaps rm{bmaps.bm, bmaps.mask_t, (p.R + 31) / 32, ((p.R + 31) / 32) * 32, (p.T + 31) / 32};
-            int tl = 0;
-            while (head < stages && next_token(tl, false) == 1) issue_item(tl);
-            issued = head;
-            local_stage_and_rank_maps(p, ids_sm, rm, 0, kWarps, lane);
+            local_stage_and_rank_maps(p, ids_sm, rm, 0, kWarps, lane);   // the table first, the rows after it
             group_sync(2, kThreads);
+        } else if (kMode == kModeLocal) {
+            ok = mbar_wait(x.staged_bar, 0, abortp);
+            ok = __all_sync(0xffffffffu, ok);
         }
         // loader only; the quantising warps free the stages.  A closing item with no row
         // tells them (and through them the store issuer) that nothing follows.
@@ -453,7 +458,10 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
         stage_ids(p, 0, p.T, ids_sm, gtid, gn);
         stage_small();
         group_sync(1, gn);
-        if (gtid == 0) trace(p, c, kTrCounted);
+        if (gtid == 0) {
+            mbar_arrive(x.staged_bar);   // the mover may fetch rows now
+            trace(p, c, kTrCounted);
+        }
         build_bin_maps(p, ids_sm, p.T, bmaps, gw, nw, lane);
         group_sync(1, gn);
         if (gtid == 0) trace(p, c, kTrHistSeen);
@@ -739,6 +747,7 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
     __shared__ __align__(8) uint64_t out_empty[kOutStages];   // FP8: its stores have read it
     __shared__ __align__(8) uint64_t ready_bar;               // rows assigned, movers may go
     __shared__ __align__(8) uint64_t epoch_bar;               // epoch_sm holds this launch's epoch
+    __shared__ __align__(8) uint64_t staged_bar;              // flag-free kernel: the routing table is in shared memory
     __shared__ int abort_flag;
     __shared__ unsigned epoch_sm;
 
@@ -762,6 +771,7 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
         }
         mbar_init(&ready_bar, 1);
         mbar_init(&epoch_bar, 1);
+        mbar_init(&staged_bar, 1);
         abort_flag = 0;
         mbar_fence_init();
     }
@@ -776,7 +786,7 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
 
     const unsigned in_bytes = (unsigned)(p.H * 2 / p.parts);   // this CTA's piece of a bf16 row
     const unsigned out_bytes = (unsigned)(p.rowB / p.parts);   // and of a payload row
-    Cta x{p, pl, smem, full_bar, empty_bar, out_full, out_empty, &ready_bar, &epoch_bar, &abort_flag,
+    Cta x{p, pl, smem, full_bar, empty_bar, out_full, out_empty, &ready_bar, &epoch_bar, &staged_bar, &abort_flag,
           tid, tid & 31, tid >> 5, c, part, ch, t0, t1, t1 - t0, stages, nq,
           reinterpret_cast<int*>(smem + pl.off_ids),
           reinterpret_cast<int*>(smem + pl.off_ord),    // destinations in issue order
