@@ -66,9 +66,9 @@ struct Params {
     int32_t* slot_row;   // [T, k] region-local row of each slot, -1 if none
     int32_t* slot_pos;   // [T, k] global row (rank * cap + row) of each slot, -1 if none
     // scratch
-    int32_t* chunk_hist;  // [nchunks, B]
+    int32_t* chunk_hist;  // [B, nchunks] histogram of every chunk, bin-major
     int32_t* partial;     // [S, B] running chunk histogram at each source-rank boundary
-    int32_t* chunk_base;  // [nchunks, B] final base of every bin for every chunk
+    int32_t* chunk_base;  // [B, nchunks] final base of every bin for every chunk, bin-major
     unsigned* hist_flag;  // [nchunks]
     unsigned* scan_flag;  // [R]
     unsigned* arrival;    // [2, R]

@@ -575,10 +575,10 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
             // region), published by the prefix-sum step, + earlier tokens of this chunk.
             // The published part is fetched once per bin into shared memory (one round
             // trip to L2), the rest is bit counting.
-            const int32_t* cb = p.chunk_base + (size_t)ch * p.B;
+            const int32_t* cb = p.chunk_base + ch;   // [bin][chunk]
             int* base_sm = hist + p.B;   // second half of the scratch (the first may hold scan totals)
             for (int b = gtid; b < p.B; b += gn)
-                base_sm[b] = __ldcg(cb + b) + (b < p.E ? __ldcg(p.expert_offset + b) : 0);
+                base_sm[b] = __ldcg(cb + (size_t)b * p.nchunks) + (b < p.E ? __ldcg(p.expert_offset + b) : 0);
             group_sync(1, gn);
             finalize_chunk(p, t0, t1, ids, w_sm,
                            [&](int e, int tl) { return base_sm[e] + bits_in_range(bmaps, e, 0, tl); },

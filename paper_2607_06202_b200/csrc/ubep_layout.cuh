@@ -181,7 +181,7 @@ static __device__ void publish_chunk_counts(const Params& p, int ch, int t0, int
         ++nbnd;
     }
     for (int b = gtid; b < B; b += gn) {
-        p.chunk_hist[(size_t)ch * B + b] = bits_in_range(bmaps, b, 0, t1 - t0);
+        p.chunk_hist[(size_t)b * p.nchunks + ch] = bits_in_range(bmaps, b, 0, t1 - t0);   // [bin][chunk]
         for (int q = 0; q < nbnd; ++q) {
             const int bs = q < 4 ? bnd[q] : src_begin(s_lo + q, T, S);
             p.partial[(size_t)(s_lo + q) * B + b] = bits_in_range(bmaps, b, 0, bs - t0);
@@ -193,11 +193,13 @@ static __device__ void publish_chunk_counts(const Params& p, int ch, int t0, int
 // Prefix sums for the bins of rank r (its L experts and its rank bin), run by a group of
 // nw warps that share barrier `bar_id`.  One pass over the chunk histograms gives, per bin,
 // the exclusive prefix over chunks (chunk_base) and the total; the expert offsets inside
-// the region follow from the totals.  `sm` holds L + 1 ints.  Inputs written by other CTAs
+// the region follow from the totals.  chunk_hist and chunk_base are stored [bin][chunk], so the
+// chunks of a bin -- what this step reads and writes, with all CTAs waiting for it -- lie side
+// by side.  `sm` holds L + 1 ints.  Inputs written by other CTAs
 // are read past L1 (__ldcg).  scan_rank_publish must complete before the rank's readiness
 // flag is released; scan_rank_sources only fills cnt / src_offset, which no mover needs.
 static __device__ void scan_rank_publish(const Params& p, int r, int* sm, int gw, int nw, int lane, int bar_id) {
-    const int n = p.nchunks, L = p.L, B = p.B, E = p.E;
+    const int n = p.nchunks, L = p.L, E = p.E;
     const int nb = L + 1;
     for (int bi = gw; bi < nb; bi += nw) {
         const int bin = bi < L ? r * L + bi : E + r;
@@ -209,7 +211,7 @@ static __device__ void scan_rank_publish(const Params& p, int r, int* sm, int gw
 #pragma unroll
         for (int i = 0; i < kMaxChunks / 32; ++i) {
             const int c = lane * per + i;
-            v[i] = (i < per && c < n) ? __ldcg(p.chunk_hist + (size_t)c * B + bin) : 0;
+            v[i] = (i < per && c < n) ? __ldcg(p.chunk_hist + (size_t)bin * n + c) : 0;
         }
 #pragma unroll
         for (int i = 0; i < kMaxChunks / 32; ++i) mine += v[i];
@@ -218,7 +220,7 @@ static __device__ void scan_rank_publish(const Params& p, int r, int* sm, int gw
 #pragma unroll
         for (int i = 0; i < kMaxChunks / 32; ++i) {
             const int c = lane * per + i;
-            if (i < per && c < n) p.chunk_base[(size_t)c * B + bin] = run;
+            if (i < per && c < n) p.chunk_base[(size_t)bin * n + c] = run;
             run += v[i];
         }
         const int carry = __shfl_sync(0xffffffffu, incl, 31);
@@ -253,12 +255,12 @@ static __device__ void scan_rank_sources(const Params& p, int r, const int* sm, 
         const int s = i / L, bi = i - s * L, bin = r * L + bi;
         const int eo = __ldcg(p.expert_offset + bin);
         const int b0 = src_begin(s, T, S);
-        const int pre0 = __ldcg(p.chunk_base + (size_t)chunk_of(b0, T, n) * B + bin) +
+        const int pre0 = __ldcg(p.chunk_base + (size_t)bin * n + chunk_of(b0, T, n)) +
                          __ldcg(p.partial + (size_t)s * B + bin);
         int pre1 = sm[bi];
         if (s + 1 < S) {
             const int b1 = src_begin(s + 1, T, S);
-            pre1 = __ldcg(p.chunk_base + (size_t)chunk_of(b1, T, n) * B + bin) +
+            pre1 = __ldcg(p.chunk_base + (size_t)bin * n + chunk_of(b1, T, n)) +
                    __ldcg(p.partial + (size_t)(s + 1) * B + bin);
         }
         p.src_offset[(size_t)s * E + bin] = eo + pre0;
