@@ -138,7 +138,9 @@ int ubep_set_replicas(ubep_buffer_t *buf, const int32_t *phys /*[dev]*/,
 /*
  * Destination-ordering table (Sec. 3.3: the re-mapped expert sequence each worker sends
  * in).  `order` [host] is a permutation of 0..R-1; worker w issues the copies of one row
- * in the table's order rotated by w.  Results never depend on it.  NULL = identity.
+ * in the table's order rotated by w.  Results never depend on it.  NULL = no table: the
+ * copies of a row are issued in slot order, which saves the ordering step of every dispatch
+ * (on one GPU all destinations are the same memory, so the order changes nothing measurable).
  */
 int ubep_set_dest_order(ubep_buffer_t *buf, const int32_t *order /*[host] [R]*/);
 

@@ -49,6 +49,7 @@ struct Params {
     const int32_t* ncopies;  // [E_log]
     int E_log, C;
     const int32_t* order_pos;  // [R] position of each rank in the destination-ordering table
+    int ordered;               // 1 = a table was set (ubep_set_dest_order): copies are issued in its order
     // arena outputs
     uint8_t* recv_x;
     float* recv_scale;

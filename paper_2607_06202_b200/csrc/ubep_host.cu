@@ -145,6 +145,7 @@ struct ubep_buffer {
     const int32_t* phys;
     const int32_t* ncopies;
     int32_t E_log, C;
+    int32_t ordered;    // a destination-ordering table has been set
     int32_t my_rank;    // sharded use (ubep_set_peers): this GPU's rank, -1 otherwise
     uint8_t* wire;      // readiness-protocol wire buffer (caller-owned) or null
     WireLayout wlay;
@@ -179,6 +180,7 @@ Params make_params(ubep_buffer* b, int T) {
     p.withhold = -1;
     p.phys = b->phys; p.ncopies = b->ncopies; p.E_log = b->E_log; p.C = b->C;
     p.order_pos = at<int32_t>(b, a.order_pos);
+    p.ordered = b->ordered;
     p.recv_x = at<uint8_t>(b, a.off[UBEP_VIEW_RECV_X]);
     p.recv_scale = at<float>(b, a.off[UBEP_VIEW_RECV_SCALE]);
     p.recv_src_idx = at<int32_t>(b, a.off[UBEP_VIEW_RECV_SRC_IDX]);
@@ -270,6 +272,7 @@ int ubep_buffer_create(const ubep_config_t* cfg, void* dev_arena, size_t bytes, 
     b->ncopies = nullptr;
     b->E_log = 0;
     b->C = 0;
+    b->ordered = 0;
     b->my_rank = -1;
     b->wire = nullptr;
     b->wlay = WireLayout{};
@@ -321,7 +324,9 @@ int ubep_set_dest_order(ubep_buffer_t* buf, const int32_t* order) {
     cudaError_t e = cudaMemcpyAsync(buf->arena + buf->lay.order_pos, posv.data(), sizeof(int32_t) * R,
                                     cudaMemcpyHostToDevice, buf->last_stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(buf->last_stream);
-    return e == cudaSuccess ? UBEP_OK : cuda_fail(buf, e);
+    if (e != cudaSuccess) return cuda_fail(buf, e);
+    buf->ordered = order != nullptr;
+    return UBEP_OK;
 }
 
 int ubep_get_dispatch_layout(ubep_buffer_t* buf, const int32_t* topk_idx, int32_t T, int32_t* num_tokens_per_rank,

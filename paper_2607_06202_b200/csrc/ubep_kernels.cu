@@ -429,8 +429,10 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
         local_rows_dedup(p, t0, t1, ids_sm, rm, c, order_sm, pos_raw, key, row_sm, arr, gtid, gn);
         group_sync(1, gn);
         if (gtid == 0) trace(p, c, kTrFinalized);
-        order_destinations(p, pos_raw, key, pos, ntok * p.k, gtid, gn);
-        group_sync(1, gn);
+        if (p.ordered) {   // a destination table is set: the copies of a token in its order (else pos_raw is pos)
+            order_destinations(p, pos_raw, key, pos, ntok * p.k, gtid, gn);
+            group_sync(1, gn);
+        }
         if (gtid == 0) {
             mbar_arrive(&ready_bar);
             trace(p, c, kTrReady);
@@ -485,8 +487,10 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
                        part == 0, c, order_sm, pos_raw, key, arr, gtid, gn);
         group_sync(1, gn);
         if (gtid == 0) trace(p, c, kTrFinalized);
-        order_destinations(p, pos_raw, key, pos, ntok * p.k, gtid, gn);
-        group_sync(1, gn);
+        if (p.ordered) {   // a destination table is set: the copies of a token in its order (else pos_raw is pos)
+            order_destinations(p, pos_raw, key, pos, ntok * p.k, gtid, gn);
+            group_sync(1, gn);
+        }
         if (gtid == 0) {
             mbar_arrive(&ready_bar);
             trace(p, c, kTrReady);
@@ -586,8 +590,10 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
                            true, c, order_sm, pos_raw, key, kSteal ? nullptr : arr, gtid, gn);
             group_sync(1, gn);
             if (gtid == 0) trace(p, c, kTrFinalized);
-            order_destinations(p, pos_raw, key, pos, ntok * p.k, gtid, gn);
-            group_sync(1, gn);
+            if (p.ordered) {   // a destination table is set: the copies of a token in its order (else pos_raw is pos)
+                order_destinations(p, pos_raw, key, pos, ntok * p.k, gtid, gn);
+                group_sync(1, gn);
+            }
         }
         if (gtid == 0) {
             mbar_arrive(&ready_bar);
@@ -790,7 +796,8 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
           tid, tid & 31, tid >> 5, c, part, ch, t0, t1, t1 - t0, stages, nq,
           reinterpret_cast<int*>(smem + pl.off_ids),
           reinterpret_cast<int*>(smem + pl.off_ord),    // destinations in issue order
-          reinterpret_cast<int*>(smem + pl.off_pos),    // destinations in slot order
+          reinterpret_cast<int*>(smem + (p.ordered ? pl.off_pos : pl.off_ord)),   // in slot order (the same array
+                                                                                  // when no table reorders them)
           reinterpret_cast<int*>(smem + pl.off_key),
           reinterpret_cast<float*>(smem + pl.off_w),
           BinMaps{reinterpret_cast<unsigned*>(smem + pl.off_mask), reinterpret_cast<unsigned*>(smem + pl.off_bm),
