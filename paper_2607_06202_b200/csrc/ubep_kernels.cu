@@ -464,21 +464,7 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
             mbar_arrive(x.staged_bar);   // the mover may fetch rows now
             trace(p, c, kTrCounted);
         }
-        build_bin_maps(p, ids_sm, p.T, bmaps, gw, nw, lane);
-        group_sync(1, gn);
-        if (gtid == 0) trace(p, c, kTrHistSeen);
-        for (int b = gtid; b < p.B; b += gn) {
-            const int before = bits_in_range(bmaps, b, 0, t0);
-            pre[b] = before;
-            tot[b] = before + bits_in_range(bmaps, b, t0, p.T);
-        }
-        group_sync(1, gn);
-        for (int e = gtid; e < p.E; e += gn) {
-            int o = 0;
-            for (int q = (e / p.L) * p.L; q < e; ++q) o += tot[q];
-            eo[e] = o;
-        }
-        group_sync(1, gn);
+        local_counts_all_bins(p, ids_sm, bmaps, t0, tot, pre, eo, gtid, gn, gw, nw, lane, 1);
         if (gtid == 0) trace(p, c, kTrScanSeen);
         ids = ids_sm + (size_t)t0 * p.k;
         finalize_chunk(p, t0, t1, ids, w_sm,
@@ -497,29 +483,9 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
             *x.epoch_late = read_epoch_and_check_in(p);   // nothing needs it before the kernel's last lines
         }
         // outputs nobody inside this kernel waits for
-        if (c == 0) {
-            for (int e = gtid; e < p.E; e += gn) {
-                p.expert_offset[e] = eo[e];
-                p.num_tokens_per_expert[e] = tot[e];
-            }
-            for (int r = gtid; r < p.R; r += gn) {
-                p.num_tokens_per_rank[r] = tot[p.E + r];
-                int rows = tot[p.E + r];
-                if (!p.dedup) {
-                    rows = 0;
-                    for (int q = r * p.L; q < (r + 1) * p.L; ++q) rows += tot[q];
-                }
-                p.num_rows_per_rank[r] = rows;
-            }
-        }
+        if (c == 0) write_totals(p, tot, eo, gtid, gn);
         if (part == 0)
-            for (int s = ch; s < p.S; s += p.nchunks) {   // source ranks this CTA reports
-                const int b0 = src_begin(s, p.T, p.S), b1 = src_begin(s + 1, p.T, p.S);
-                for (int e = gtid; e < p.E; e += gn) {
-                    p.cnt[(size_t)s * p.E + e] = bits_in_range(bmaps, e, b0, b1);
-                    p.src_offset[(size_t)s * p.E + e] = eo[e] + bits_in_range(bmaps, e, 0, b0);
-                }
-            }
+            for (int s = ch; s < p.S; s += p.nchunks) write_source_from_maps(p, s, bmaps, eo, gtid, gn);   // source ranks this CTA reports
     } else {
         stage_ids(p, t0, t1, ids_sm, gtid, gn);
         stage_small();

@@ -355,6 +355,59 @@ __device__ void finalize_chunk(const Params& p, int t0, int t1, const int* ids, 
     }
 }
 
+// ------------------------------------------------- flag-free layout, every bin
+// From the staged table of all T tokens (ids: T * k slots): the bitmaps of every bin, then per bin
+// the total (tot), the count among the tokens before t0 (pre) and per expert the offset inside its
+// rank's region (eo).  Run by the gn threads (nw warps) that share barrier `bar`; ends with that
+// barrier.  Used by every kernel in which a CTA derives the layout alone.
+static __device__ void local_counts_all_bins(const Params& p, const int* ids, const BinMaps& bmaps, int t0, int* tot,
+                                             int* pre, int* eo, int gtid, int gn, int gw, int nw, int lane, int bar) {
+    build_bin_maps(p, ids, p.T, bmaps, gw, nw, lane);
+    group_sync(bar, gn);
+    for (int b = gtid; b < p.B; b += gn) {
+        const int before = bits_in_range(bmaps, b, 0, t0);
+        pre[b] = before;
+        tot[b] = before + bits_in_range(bmaps, b, t0, p.T);
+    }
+    group_sync(bar, gn);
+    for (int e = gtid; e < p.E; e += gn) {
+        int o = 0;
+        for (int q = (e / p.L) * p.L; q < e; ++q) o += tot[q];
+        eo[e] = o;
+    }
+    group_sync(bar, gn);
+}
+
+// Rows region r receives, from the totals.
+__device__ __forceinline__ int rows_of_rank(const Params& p, const int* tot, int r) {
+    if (p.dedup) return tot[p.E + r];
+    int rows = 0;
+    for (int q = r * p.L; q < (r + 1) * p.L; ++q) rows += tot[q];
+    return rows;
+}
+
+// The counts and offsets that are the same for everybody, written by one CTA.
+static __device__ void write_totals(const Params& p, const int* tot, const int* eo, int gtid, int gn) {
+    for (int e = gtid; e < p.E; e += gn) {
+        p.expert_offset[e] = eo[e];
+        p.num_tokens_per_expert[e] = tot[e];
+    }
+    for (int r = gtid; r < p.R; r += gn) {
+        p.num_tokens_per_rank[r] = tot[p.E + r];
+        p.num_rows_per_rank[r] = rows_of_rank(p, tot, r);
+    }
+}
+
+// What source rank s reports (cnt, src_offset), from bitmaps over the whole table.
+static __device__ void write_source_from_maps(const Params& p, int s, const BinMaps& bmaps, const int* eo, int gtid,
+                                              int gn) {
+    const int b0 = src_begin(s, p.T, p.S), b1 = src_begin(s + 1, p.T, p.S);
+    for (int e = gtid; e < p.E; e += gn) {
+        p.cnt[(size_t)s * p.E + e] = bits_in_range(bmaps, e, b0, b1);
+        p.src_offset[(size_t)s * p.E + e] = eo[e] + bits_in_range(bmaps, e, 0, b0);
+    }
+}
+
 // --------------------------------------------- flag-free layout, dedup fast path
 // With one row per (token, rank) the movers only need rank-level rows: row of token t in
 // region r = number of earlier tokens that visit r.  One 32-bit word per token and 32 ranks

@@ -56,27 +56,8 @@ __global__ void __launch_bounds__(kThreads, 1) sharded_dispatch_kernel(const Par
     stage_ids(p, 0, p.T, ids_sm, tid, kThreads);
     for (int i = tid; i < ntok * k; i += kThreads) w_sm[i] = __ldg(p.topk_w + (size_t)t0 * k + i);
     __syncthreads();
-    build_bin_maps(p, ids_sm, p.T, bmaps, warp, kWarps, lane);
-    __syncthreads();
-    for (int b = tid; b < p.B; b += kThreads) {
-        const int before = bits_in_range(bmaps, b, 0, t0);
-        pre[b] = before;
-        tot[b] = before + bits_in_range(bmaps, b, t0, p.T);
-    }
-    __syncthreads();
-    for (int e = tid; e < p.E; e += kThreads) {
-        int o = 0;
-        for (int q = (e / p.L) * p.L; q < e; ++q) o += tot[q];
-        eo[e] = o;
-    }
-    for (int r = tid; r < R; r += kThreads) {
-        int rows = tot[p.E + r];
-        if (!p.dedup) {
-            rows = 0;
-            for (int q = r * p.L; q < (r + 1) * p.L; ++q) rows += tot[q];
-        }
-        nrows[r] = rows;
-    }
+    local_counts_all_bins(p, ids_sm, bmaps, t0, tot, pre, eo, tid, kThreads, warp, kWarps, lane, 0);
+    for (int r = tid; r < R; r += kThreads) nrows[r] = rows_of_rank(p, tot, r);
     __syncthreads();
     // rows of this CTA's slots; the metadata of every row goes to the arena of the rank that receives it
     finalize_chunk<true>(p, t0, t1, ids_sm + (size_t)t0 * k, w_sm,
@@ -86,24 +67,11 @@ __global__ void __launch_bounds__(kThreads, 1) sharded_dispatch_kernel(const Par
     __syncthreads();
     // counts and offsets: every rank keeps the whole set in its own arena
     if (c == 0) {
-        for (int e = tid; e < p.E; e += kThreads) {
-            p.expert_offset[e] = eo[e];
-            p.num_tokens_per_expert[e] = tot[e];
-        }
-        for (int r = tid; r < R; r += kThreads) {
-            p.num_tokens_per_rank[r] = tot[p.E + r];
-            p.num_rows_per_rank[r] = nrows[r];
-        }
+        write_totals(p, tot, eo, tid, kThreads);
         // what the local receiver has to wait for (read by wait_arrivals_kernel, later in this stream)
         if (tid == 0) atomicAdd(p.shard_arrival + 1, (unsigned)(nrows[p.my_rank] < p.cap ? nrows[p.my_rank] : p.cap));
     }
-    for (int s = c; s < p.S; s += p.grid) {
-        const int b0 = src_begin(s, p.T, p.S), b1 = src_begin(s + 1, p.T, p.S);
-        for (int e = tid; e < p.E; e += kThreads) {
-            p.cnt[(size_t)s * p.E + e] = bits_in_range(bmaps, e, b0, b1);
-            p.src_offset[(size_t)s * p.E + e] = eo[e] + bits_in_range(bmaps, e, 0, b0);
-        }
-    }
+    for (int s = c; s < p.S; s += p.grid) write_source_from_maps(p, s, bmaps, eo, tid, kThreads);
 
     // ---- sender: one token at a time, all threads on its row, one 128-bit store per copy
     const int nvec = p.rowB / 16;
