@@ -4,10 +4,9 @@
  * The expert-parallel ranks are virtual: R disjoint receive regions inside one device
  * arena that the caller allocates.  The library allocates no device memory, creates no
  * stream and synchronises the host only where a call says so (ubep_status, and the set-up
- * calls ubep_set_dest_order, ubep_set_peers, ubep_sync_attach, ubep_sync_scan_sentinel).  Every
- * pointer below
- * is marked [host] or [dev]; all device pointers must be 16-byte aligned; `cuda_stream`
- * is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ * calls ubep_set_dest_order, ubep_set_peers, ubep_sync_attach, ubep_sync_scan_sentinel).
+ * Every pointer below is marked [host] or [dev]; all device pointers must be 16-byte aligned;
+ * `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  *
  * Notation: T tokens, H hidden size, E physical experts, R ranks, L = E / R experts per
  * rank (expert p lives on rank p / L), k = top-k, S source ranks (token t belongs to the

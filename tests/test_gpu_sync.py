@@ -201,3 +201,40 @@ def test_argument_errors():
     # T == 0 leaves zero counts like the main dispatch
     buf.dispatch_sync("dc", x[:0], idx[:0], w[:0])
     assert int(buf.num_rows_per_rank.sum()) == 0 and buf.status() == 0
+
+
+def test_one_captured_graph_of_all_protocols_replays_with_new_routing():
+    """The sequence number that flags and counter halves go by lives on the device, so a captured
+    graph of protocol dispatches can be replayed; inputs are rewritten in place between replays."""
+    cfg = W.Config("graph", T=160, H=512, E=32, R=8, k=4, seed=4500)
+    base = W.make_workload(cfg)
+    cap = 256
+    bufs = {proto: Hn.make_buffer(cfg, cap) for proto in PROTOCOLS}
+    for b in bufs.values():
+        b.attach_sync()
+    x, idx, w, _, _ = Hn.device_inputs(base)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):                      # warm-up outside capture
+        for proto, b in bufs.items():
+            b.dispatch_sync(proto, x, idx, w, stream)
+    stream.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        for proto, b in bufs.items():
+            b.dispatch_sync(proto, x, idx, w, stream)
+    for it in range(3):
+        wl = W.make_workload(dataclasses.replace(cfg, seed=4600 + it))
+        x.copy_(Hn.to_dev(wl.x, torch.bfloat16))
+        idx.copy_(Hn.to_dev(wl.topk_idx.astype(np.int32)))
+        w.copy_(Hn.to_dev(wl.topk_w))
+        for b in bufs.values():
+            for name in ("recv_x", "recv_src_idx", "recv_weight"):
+                b.views[name].view(torch.uint8).fill_(Hn.FILL)
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        ids, lay, _, recv = Hn.oracle_reference(wl, cap=cap)
+        for proto, b in bufs.items():
+            Hn.check_dispatch(b, wl, lay, cap, recv, arrival=False)
+            wire_checks(b, proto, cfg, lay, recv, b.sync_views["times"].shape[0])
+            assert int(b.sync_views["seq"].item()) == 2 + it     # one warm-up call, then one per replay
