@@ -70,7 +70,10 @@ typedef struct {
                                /* 1: one row per (token, rank), ascending token                */
     int32_t device;            /* CUDA device ordinal                                          */
     int32_t pipeline;          /* UBEP_PIPELINE_*                                              */
-    int32_t num_ctas;          /* persistent CTAs / token chunks; 0 = number of SMs            */
+    int32_t num_ctas;          /* persistent CTAs / token chunks; 0 = number of SMs.  The      */
+                               /* bookkeeping of one chunk lives in shared memory: a dispatch  */
+                               /* whose T / num_ctas tokens do not fit there (a few thousand   */
+                               /* slots per CTA) returns UBEP_ERR_ARG and launches nothing     */
 } ubep_config_t;
 
 /* Arrays that live in the arena; ubep_view() returns their device address and shape. */
