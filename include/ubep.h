@@ -346,8 +346,8 @@ int ubep_sync_scan_sentinel(ubep_buffer_t *buf, const void *x /*[dev]*/, int32_t
  * The caller orders the steps across ranks where data is reused: no rank may start dispatch
  * n + 1 before every rank has finished reading what dispatch n delivered, and no rank may
  * start combine before the y of every peer is complete (a barrier on the streams, e.g. an
- * NCCL one).  Limits of this path: bf16 payload, T * k <= 8192, no FP8, no replicas beyond
- * ubep_set_replicas.  Kernels of different ranks never wait for one another except in
+ * NCCL one).  Limit of this path: T * k <= 8192.  Both payloads (FP8 rows are quantised by
+ * the sender; scales land in the receiver's scale array).  Kernels of different ranks never wait for one another except in
  * ubep_wait_arrivals, which therefore must not be emulated by launches queued on one GPU
  * ahead of the senders it waits for.
  */

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libubep.so")
 SOURCES = ["ubep_kernels.cu", "ubep_host.cu", "ubep_static.cu", "ubep_mapper.cu", "ubep_sync.cu", "ubep_sharded.cu"]
-DEPENDS = SOURCES + ["ubep_common.cuh", "ubep_layout.cuh", "ubep_kernels.h", "ubep_sync.h", "ubep_sharded.h", "../../include/ubep.h"]
+DEPENDS = SOURCES + ["ubep_common.cuh", "ubep_layout.cuh", "ubep_quant.cuh", "ubep_kernels.h", "ubep_sync.h", "ubep_sharded.h", "../../include/ubep.h"]
 
 
 def up_to_date() -> bool:

@@ -549,7 +549,7 @@ int ubep_sync_scan_sentinel(ubep_buffer_t* buf, const void* x, int32_t T, int64_
 int ubep_set_peers(ubep_buffer_t* buf, int32_t my_rank, void* const* peer_arenas) {
     if (!buf || !peer_arenas || my_rank < 0 || my_rank >= buf->cfg.num_ranks) return UBEP_ERR_ARG;
     const int R = buf->cfg.num_ranks;
-    if (buf->lay.S != R || buf->cfg.payload != UBEP_PAYLOAD_BF16) return UBEP_ERR_ARG;   // one source rank per GPU
+    if (buf->lay.S != R) return UBEP_ERR_ARG;   // one source rank per GPU
     if (peer_arenas[my_rank] != buf->arena) return UBEP_ERR_ARG;
     std::vector<long long> delta(R);
     for (int r = 0; r < R; ++r) {

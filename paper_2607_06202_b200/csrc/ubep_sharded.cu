@@ -2,13 +2,14 @@
 // "Global Load/Store for Point-to-Point Synchronization"): rank r = GPU r, every GPU holds an
 // arena of the same layout that its peers address over NVLink, rows and their metadata are
 // stored straight into the receiving rank's arena, expert outputs are loaded straight from the
-// producing rank's buffer.  Plain 128-bit loads and stores only: no TMA, no multicast, no
-// collective.  No kernel here waits for another rank except wait_arrivals_kernel.
+// producing rank's buffer.  Plain loads and stores only: no TMA, no multicast, no collective.
+// FP8 rows are quantised by the sender, payload and scales go to the receiver's arrays.  No kernel here waits for another rank except wait_arrivals_kernel.
 //
 // Every rank derives the whole layout from the all-gathered routing table, alone, with the
 // same device functions and in the same order as the flag-free instance of the main dispatch
 // kernel, so all ranks agree on every row without exchanging a count.
 #include "ubep_layout.cuh"
+#include "ubep_quant.cuh"
 #include "ubep_sharded.h"
 
 namespace ubep {
@@ -73,18 +74,30 @@ __global__ void __launch_bounds__(kThreads, 1) sharded_dispatch_kernel(const Par
     }
     for (int s = c; s < p.S; s += p.grid) write_source_from_maps(p, s, bmaps, eo, tid, kThreads);
 
-    // ---- sender: one token at a time, all threads on its row, one 128-bit store per copy
-    const int nvec = p.rowB / 16;
+    // ---- sender: one token at a time, all threads on its row, one store per copy and vector
+    const int nvec = p.H / 8;   // 16-byte vectors of the bf16 input row
     for (int tl = 0; tl < ntok; ++tl) {
         const int* ps = pos + tl * k;
         const uint4* src = reinterpret_cast<const uint4*>(p.x + (size_t)(t0 + tl - p.tok0) * p.H);
-        for (int v = tid; v < nvec; v += kThreads) {
-            const uint4 d = __ldg(src + v);
+        for (int v0 = 0; v0 < nvec; v0 += kThreads) {   // same trip count for every thread (the quantiser shuffles)
+            const int v = v0 + tid;
+            const bool in = v < nvec;
+            const uint4 d = in ? __ldg(src + v) : make_uint4(0, 0, 0, 0);
+            uint2 q = make_uint2(0, 0);
+            float scale = 0.0f;
+            if (p.payload) quantize8(d, in, q, scale);
+            if (!in) continue;
             for (int j = 0; j < k; ++j) {
                 const int where = ps[j];
                 if (where < 0) continue;
-                uint8_t* region = p.recv_x + delta[where / p.cap];
-                *reinterpret_cast<uint4*>(region + (size_t)where * p.rowB + (size_t)v * 16) = d;
+                const long long pd = delta[where / p.cap];
+                uint8_t* row = p.recv_x + pd + (size_t)where * p.rowB;
+                if (p.payload) {
+                    *reinterpret_cast<uint2*>(row + (size_t)v * 8) = q;
+                    if ((v & 15) == 0) toward_peer<true>(p.recv_scale, pd)[(size_t)where * p.G + (v >> 4)] = scale;
+                } else {
+                    *reinterpret_cast<uint4*>(row + (size_t)v * 16) = d;
+                }
             }
         }
     }

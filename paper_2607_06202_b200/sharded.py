@@ -63,20 +63,20 @@ class ShardedEP:
     """This process's rank of an expert-parallel group: R = world size, experts p of rank p // L."""
 
     def __init__(self, *, num_experts: int, hidden: int, topk: int, max_tokens: int, rows_per_rank_cap: int,
-                 dedup: int = 0, group=None, device: Optional[torch.device] = None,
+                 dedup: int = 0, payload: int = 0, group=None, device: Optional[torch.device] = None,
                  alloc: Callable = symmetric_alloc):
         self.group = group
         self.rank, self.world = dist.get_rank(group), dist.get_world_size(group)
         self.device = device if device is not None else torch.device("cuda", torch.cuda.current_device())
-        self.H, self.k, self.cap = hidden, topk, rows_per_rank_cap
-        cfg = B.ubep_config_t(self.world, num_experts, hidden, topk, max_tokens, rows_per_rank_cap, 0, 0, dedup,
+        self.H, self.k, self.cap, self.payload = hidden, topk, rows_per_rank_cap, payload
+        cfg = B.ubep_config_t(self.world, num_experts, hidden, topk, max_tokens, rows_per_rank_cap, 0, payload, dedup,
                               self.device.index or 0, 0, 0)
         nbytes = B.ubep_buffer_bytes(cfg)
         if nbytes == 0:
             raise B.UbepError(B.UBEP_ERR_ARG, "ubep_buffer_bytes")
         arena, arena_ptrs = alloc(nbytes, self.device, group)
         self.buf = B.Buffer(num_ranks=self.world, num_experts=num_experts, hidden=hidden, topk=topk,
-                            max_tokens=max_tokens, rows_per_rank_cap=rows_per_rank_cap, dedup=dedup,
+                            max_tokens=max_tokens, rows_per_rank_cap=rows_per_rank_cap, dedup=dedup, payload=payload,
                             device=self.device.index or 0, arena=arena)
         B.ubep_set_peers(self.buf.handle, self.rank, arena_ptrs)
         # expert outputs, laid out like the receive regions; this rank fills region `rank`
@@ -93,8 +93,11 @@ class ShardedEP:
             dist.all_reduce(self._token, group=self.group)
 
     @property
-    def region(self) -> torch.Tensor:
-        """The rows this rank received: bf16 [cap, H] (num_rows_per_rank[rank] of them are valid)."""
+    def region(self):
+        """The rows this rank received (num_rows_per_rank[rank] of them are valid): bf16 [cap, H], or for
+        FP8 rows the pair (e4m3 bytes [cap, H], fp32 scales [cap, H / 128])."""
+        if self.payload:
+            return self.buf.recv_x[self.rank], self.buf.recv_scale[self.rank]
         return self.buf.recv_x[self.rank].view(torch.bfloat16).view(self.cap, self.H)
 
     def dispatch(self, x_local: torch.Tensor, idx_local: torch.Tensor, w_local: torch.Tensor, T: int):

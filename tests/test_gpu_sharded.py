@@ -23,6 +23,8 @@ CASES = {
     "fewer_tokens_than_ranks": W.Config("few", T=5, H=128, E=16, R=8, k=2, dedup=1, seed=5103),
     "one_rank": W.Config("one_rank", T=19, H=64, E=4, R=1, k=2, seed=5104),
     "replicas": W.Config("replicas", T=96, H=512, E=36, R=4, k=4, seed=5105, E_logical=32),
+    "fp8": W.Config("fp8", T=96, H=384, E=16, R=4, k=4, payload=1, seed=5106),
+    "fp8_dedup": W.Config("fp8_dedup", T=70, H=1024, E=32, R=8, k=4, payload=1, dedup=1, seed=5107),
 }
 
 
@@ -56,6 +58,8 @@ def check_rank(bufs, r, cfg, lay, recv, times=1):
         assert torch.equal(b.recv_x[q], want), f"arena {r} region {q}"
     n = int(lay.num_rows_per_rank[r])
     Hn._eq(f"recv_src_idx[{r}]", b.recv_src_idx[r, :n], recv.recv_src_idx[r, :n])
+    if cfg.payload:
+        Hn._eq(f"recv_scale[{r}]", b.recv_scale[r, :n].view(torch.int32), recv.recv_scale[r, :n].view(np.int32))
     if cfg.dedup:
         Hn._eq("recv_topk_idx", b.recv_topk_idx[r, :n], recv.recv_topk_idx[r, :n])
         Hn._eq("recv_topk_w", b.recv_topk_w[r, :n].view(torch.int32), recv.recv_topk_w[r, :n].view(np.int32))
@@ -138,9 +142,6 @@ def test_argument_errors():
     other = Hn.make_buffer(cfg, cap)
     with pytest.raises(B.UbepError):                      # the table's own entry must be this buffer's arena
         B.ubep_set_peers(buf.handle, 0, [other.arena.data_ptr()] + ptrs[1:])
-    fp8 = Hn.make_buffer(dataclasses.replace(cfg, payload=1), cap)
-    with pytest.raises(B.UbepError):
-        B.ubep_set_peers(fp8.handle, 0, [fp8.arena.data_ptr()] * cfg.R)
     fewer_sources = Hn.make_buffer(dataclasses.replace(cfg, num_src_ranks=2), cap)
     with pytest.raises(B.UbepError):                      # one source rank per GPU
         B.ubep_set_peers(fewer_sources.handle, 0, [fewer_sources.arena.data_ptr()] * cfg.R)
