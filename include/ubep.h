@@ -46,7 +46,8 @@ enum { UBEP_PAYLOAD_BF16 = 0, UBEP_PAYLOAD_FP8_E4M3 = 1 };
 
 /* How ubep_dispatch schedules its steps. */
 enum {
-    UBEP_PIPELINE_AUTO = 0,   /* LOCAL while T*k <= 8192, else FUSED                           */
+    UBEP_PIPELINE_AUTO = 0,   /* LOCAL for small routing tables (how small depends on whether */
+                              /* the one-row-per-rank fast path applies), else FUSED          */
     UBEP_PIPELINE_PHASED = 1, /* count -> prefix sums -> scatter as three launches; the        */
                               /* kernel boundaries play the role of the global barriers of    */
                               /* the bulk-synchronous dispatch (Sec. 2.3, phases 2-5)         */

@@ -20,7 +20,10 @@ std::atomic<uint64_t> g_launches{0};
 
 constexpr size_t kAlign = 256;
 constexpr int kStealMinTokensPerChunk = 40;  // shorter slices: the hand-out costs more than the tail it removes (measured)
-constexpr int64_t kLocalMaxSlots = 8192;  // AUTO uses the flag-free kernel up to this many (token, slot) pairs
+constexpr int64_t kLocalMaxSlots = 8192;        // small-T limit of the combine launch mode and of the protocol / sharded paths
+constexpr int64_t kLocalFastMaxSlots = 14336;   // AUTO: flag-free kernel with the rank-level fast path up to this many slots
+constexpr int64_t kLocalMaxWeight = 18432;      // AUTO: flag-free kernel over every bin up to this many slots x bin words
+constexpr int64_t kLocalFp8MaxWeight = 9216;    // the same with FP8 rows
 inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 
 struct ArenaLayout {
@@ -370,8 +373,17 @@ int ubep_dispatch(ubep_buffer_t* buf, const void* x, const int32_t* topk_idx, co
     // AUTO: a routing table that fits in shared memory is cheaper to recount in every CTA
     // than to exchange through flags; larger ones use the decomposed kernel.
     int mode = buf->cfg.pipeline;
-    if (mode == UBEP_PIPELINE_AUTO)
-        mode = (int64_t)T * p.k <= kLocalMaxSlots ? UBEP_PIPELINE_LOCAL : UBEP_PIPELINE_FUSED;
+    if (mode == UBEP_PIPELINE_AUTO) {
+        // Measured crossovers (H = 7168, 256 experts on 32 ranks, top-8).  With the rank-level fast path
+        // the flag-free kernel wins up to about 1800 tokens; when every CTA has to build the bitmaps of
+        // every bin its cost grows with slots x bin words and it wins only for a few hundred tokens, and
+        // with FP8 rows (whose quantising warps are the layout warps, so nothing moves before the layout
+        // and its outputs are done) for about a hundred.
+        const int64_t slots = (int64_t)T * p.k, weight = slots * ((p.B + 31) / 32);
+        const bool local = p.local_fast ? slots <= kLocalFastMaxSlots
+                                        : weight <= (p.payload ? kLocalFp8MaxWeight : kLocalMaxWeight);
+        mode = local ? UBEP_PIPELINE_LOCAL : UBEP_PIPELINE_FUSED;
+    }
     ubep::SmemPlan pl{};
     int launches = 0;
     p.parts = 1;
@@ -379,14 +391,20 @@ int ubep_dispatch(ubep_buffer_t* buf, const void* x, const int32_t* topk_idx, co
     if (mode == UBEP_PIPELINE_LOCAL) {
         // split rows into column parts until the slices of work are balanced to ~5 %
         const int n = buf->lay.nchunks;
+        // The CTA with the most work sets the pace: ceil(T / chunks) tokens of 1 / parts of a row each.
+        // Smaller pieces cost more per byte (measured on the decode shape: 4 parts + 8 %, 8 parts + 60 %).
         int best = 1;
-        for (int parts = 1; parts <= 8; parts *= 2) {
+        double best_cost = 0.0;
+        static const double kPiecePenalty[4] = {1.0, 1.0, 1.08, 1.6};
+        for (int parts = 1, i = 0; parts <= 8; parts *= 2, ++i) {
             const int chunks = n / parts;
             if (chunks < 1 || (p.H * 2 / parts) % 16 != 0 || (p.H * 2) % parts != 0) break;
             if (p.payload && ((p.H / parts) % 128 != 0 || p.H % parts != 0)) break;
-            best = parts;
-            const double per = (double)T / chunks;
-            if (per / (double)((T + chunks - 1) / chunks) >= 0.95) break;
+            const double cost = (double)((T + chunks - 1) / chunks) / parts * kPiecePenalty[i];
+            if (parts == 1 || cost < best_cost * 0.999) {
+                best = parts;
+                best_cost = cost;
+            }
         }
         p.parts = best;
         p.nchunks = n / best;
