@@ -5,7 +5,12 @@ One "step" = one ubep_dispatch followed by one ubep_combine over one batch of sy
 input of the decode-shaped configuration (T=512, H=7168 bf16, E=256 over R=32 virtual
 ranks, top-8, per-rank token de-duplication).  `value` is the algorithmic bytes the two
 calls must move divided by the measured time (GB/s, whole job), next to microseconds per
-layer.  Rotating buffer sets larger than L2 keep every step cold.
+layer.  Rotating buffer sets larger than L2 keep every step cold.  Beside it in the JSON line:
+`roofline` (the dominant kernel against the measured HBM copy bandwidth), `cpu_baseline` (the CPU
+oracle on the host cores), `e2e` (the same step fed from pinned host memory: one host -> device and one
+device -> host copy per step inside the timed region, copies and kernels on streams of their own) and
+`identity_experts` (the layer when combine reads the rows dispatch has just delivered, still in L2;
+not the headline).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload decode|prefill|...]
 
