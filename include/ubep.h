@@ -55,7 +55,9 @@ enum {
                               /* offsets through release/acquire flags while mover warps      */
                               /* already stream rows (kernel decomposition, Sec. 3.2)         */
     UBEP_PIPELINE_LOCAL = 3   /* one persistent kernel in which every CTA derives its offsets */
-                              /* from the whole routing table itself (no flags; small T*k)    */
+                              /* from the whole routing table itself (no flags; small T*k:    */
+                              /* asked for explicitly with a table that does not fit in       */
+                              /* shared memory, ubep_dispatch returns UBEP_ERR_ARG)           */
 };
 
 typedef struct {
@@ -265,8 +267,9 @@ int ubep_map_workers(const int32_t *order /*[dev]*/, const int32_t *counts /*[de
  * promises for vector accesses.  All waits are bounded (about 1.5 s); a wait that runs out
  * records UBEP_ERR_TIMEOUT and the kernel returns.
  *
- * Limits: bf16 payload only, T * k <= 8192 (every CTA derives the layout from the whole
- * routing table, as UBEP_PIPELINE_LOCAL does), one CTA per SM at most.  Everything
+ * Limits: bf16 payload only; T * k <= 8192 and the routing table with the bitmaps of all its
+ * bins (T x (E + R) bits) must fit in a CTA's shared memory, since every CTA derives the layout
+ * from the whole table, as UBEP_PIPELINE_LOCAL does; one CTA per SM at most.  Everything
  * ubep_dispatch leaves in the arena is left here too, with identical contents; ubep_combine
  * may follow.  The arrival counters of ubep_dispatch (UBEP_VIEW_ARRIVAL) are not touched.
  */
@@ -304,7 +307,8 @@ int ubep_sync_attach(ubep_buffer_t *buf, void *dev_wire /*[dev]*/, size_t bytes,
  * Dispatch with readiness protocol `protocol` (UBEP_SYNC_*); arguments as ubep_dispatch.
  * One kernel launch (a memset before it when an earlier call left the SP wire dirty, which
  * the library learns when ubep_status reports that call's error).  UBEP_ERR_ARG if no wire
- * buffer is attached, the payload is not bf16 or T * k > 8192.
+ * buffer is attached, the payload is not bf16, T * k > 8192 or the table does not fit in shared
+ * memory.
  */
 int ubep_dispatch_sync(ubep_buffer_t *buf, int protocol, const void *x /*[dev]*/,
                        const int32_t *topk_idx /*[dev]*/, const float *topk_w /*[dev]*/, int32_t T,
@@ -347,10 +351,11 @@ int ubep_sync_scan_sentinel(ubep_buffer_t *buf, const void *x /*[dev]*/, int32_t
  * The caller orders the steps across ranks where data is reused: no rank may start dispatch
  * n + 1 before every rank has finished reading what dispatch n delivered, and no rank may
  * start combine before the y of every peer is complete (a barrier on the streams, e.g. an
- * NCCL one).  Limit of this path: T * k <= 8192.  Both payloads (FP8 rows are quantised by
- * the sender; scales land in the receiver's scale array).  Kernels of different ranks never wait for one another except in
- * ubep_wait_arrivals, which therefore must not be emulated by launches queued on one GPU
- * ahead of the senders it waits for.
+ * NCCL one).  Limit of this path: T * k <= 8192 and the table with the bitmaps of all its
+ * bins must fit in a CTA's shared memory (else UBEP_ERR_ARG).  Both payloads (FP8 rows are
+ * quantised by the sender; scales land in the receiver's scale array).  Kernels of different
+ * ranks never wait for one another except in ubep_wait_arrivals, which therefore must not be
+ * emulated by launches queued on one GPU ahead of the senders it waits for.
  */
 
 /*
