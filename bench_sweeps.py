@@ -1,0 +1,228 @@
+#!/usr/bin/env python
+"""Measurement sweeps beside bench.py (each needs a GPU; the library itself does not use this file).
+
+    python bench_sweeps.py spread [--workload skewed prefill] [--rows 4] [--markdown]
+    python bench_sweeps.py sync   [--tokens 128] [--iters 200] [--markdown]
+
+spread: per-CTA latency spread of dispatch under different destination-ordering tables -- the
+analogue, on one GPU, of the paper's per-worker token-transmission latencies with and without
+expert re-mapping (Sec. 5.4, "Impact of Token Scheduling").
+sync: latency of the readiness protocols (stop-and-wait, Token-Flag Fusion, Data-for-Checksum,
+Sentinel Polling; Sec. 3.4) over synchronisation granularity and rank count.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2607_06202_b200 import binding as B
+from paper_2607_06202_b200 import workload as W
+
+SPREAD_DOC = """Every CTA of the persistent dispatch kernel is one worker with an equal slice of the tokens.
+The library's phase trace (ubep_debug_trace) gives, per CTA, when its layout was ready, when its last
+copy was issued and when it left.  The tables compared are the identity order, the paper's logical
+matrix transposition with `rows` rows (Sec. 3.3) and the reversed order."""
+
+SYNC_DOC = """For every (row bytes, ranks, protocol): kernel = mean time of one ubep_dispatch_sync launch
+(CUDA events around `iters` launches); sent / ready = inside the last launch, from the first CTA's
+entry to the last sender finishing and to the last receiver having confirmed its region (device
+nanosecond timer); wire = bytes put on the wire per payload byte.  Inputs are seeded and synthetic
+(Gaussian routing, top-8 of 256 experts)."""
+
+# ------------------------------------------------------------------------------------ spread
+
+READY, ISSUED, STORED, END = 6, 8, 9, 10   # phase slots of the trace (see ubep_debug_trace)
+
+
+def stride_order(n: int, rows: int) -> np.ndarray:
+    """Visiting order of n destinations after the logical matrix transposition of Sec. 3.3: the ids
+    fill a matrix of `rows` rows row by row and are read column by column."""
+    cols = -(-n // rows)
+    grid = np.full(rows * cols, -1, np.int64)
+    grid[:n] = np.arange(n)
+    order = grid.reshape(rows, cols).T.reshape(-1)
+    return order[order >= 0].astype(np.int32)
+
+
+def spread(cfg: W.Config, order, repeats: int = 5):
+    dev = torch.device("cuda", 0)
+    wl = W.make_workload(cfg)
+    idx = torch.from_numpy(wl.topk_idx.astype(np.int32)).to(dev)
+    x = torch.from_numpy(wl.x).view(torch.bfloat16).to(dev)
+    w = torch.from_numpy(wl.topk_w.astype(np.float32)).to(dev)
+    common = dict(num_ranks=cfg.R, num_experts=cfg.E, hidden=cfg.H, topk=cfg.k, max_tokens=cfg.T,
+                  num_src_ranks=cfg.S, payload=cfg.payload, dedup=cfg.dedup)
+    probe = B.Buffer(rows_per_rank_cap=1, **common)
+    phys = ncopies = None
+    if wl.phys is not None:
+        phys, ncopies = torch.from_numpy(wl.phys).to(dev), torch.from_numpy(wl.ncopies).to(dev)
+        probe.set_replicas(phys, ncopies)
+    npr, npe, _ = probe.get_dispatch_layout(idx)
+    rows_per_rank = npr if cfg.dedup else npe.view(cfg.R, cfg.L).sum(1)
+    cap = W.round_up(max(1, int(rows_per_rank.max().item())), 128)
+    probe.close()
+    buf = B.Buffer(rows_per_rank_cap=cap, **common)
+    if phys is not None:
+        buf.set_replicas(phys, ncopies)
+    buf.set_dest_order(order)
+    B.ubep_debug_trace(buf.handle, True)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    runs = []
+    for it in range(repeats + 1):
+        flush.fill_(it)                    # cold L2 for every run
+        buf.dispatch(x, idx, w)
+        torch.cuda.synchronize()
+        if it == 0:
+            continue                       # first run: warm-up
+        tr = buf.trace.cpu().numpy().astype(np.int64)
+        t0 = tr[:, 0].min()
+        runs.append(np.stack([(tr[:, s] - t0) / 1e3 for s in (READY, ISSUED, STORED, END)], axis=1))
+    status = buf.status()
+    buf.close()
+    if status != 0:
+        raise RuntimeError(f"device status {status} ({B.ubep_strerror(status)})")
+    return np.median(np.stack(runs), axis=0)   # [CTAs, 4], median over the repeats
+
+
+def main_spread(argv):
+    ap = argparse.ArgumentParser(prog="bench_sweeps.py spread", description=SPREAD_DOC,
+                                 formatter_class=argparse.RawDescriptionHelpFormatter)
+    ap.add_argument("--workload", nargs="*", default=["skewed", "prefill"], choices=list(W.CONFIGS))
+    ap.add_argument("--rows", type=int, default=4, help="rows of the transposition matrix")
+    ap.add_argument("--markdown", action="store_true")
+    args = ap.parse_args(argv)
+    B.load()
+    if args.markdown:
+        print("| workload | table | layout ready us (median / max) | sending us: min / median / p95 / max | "
+              "max / median | kernel end us (max) |")
+        print("|---|---|---|---|---|---|")
+    for name in args.workload:
+        cfg = W.CONFIGS[name]
+        tables = {"identity": None, f"transposed ({args.rows} rows)": stride_order(cfg.R, args.rows),
+                  "reversed": np.arange(cfg.R - 1, -1, -1, dtype=np.int32)}
+        for label, order in tables.items():
+            t = spread(cfg, order)
+            send = t[:, 3] - t[:, 0]          # layout ready (movers released) -> CTA done, all its copies complete
+            line = (name, label, np.median(t[:, 0]), t[:, 0].max(), send.min(), np.median(send),
+                    np.percentile(send, 95), send.max(), send.max() / np.median(send), t[:, 3].max())
+            if args.markdown:
+                print("| %s | %s | %.1f / %.1f | %.1f / %.1f / %.1f / %.1f | %.2f | %.1f |" % line)
+            else:
+                print("%s %-22s ready %.1f/%.1f  sending min %.1f med %.1f p95 %.1f max %.1f  max/med %.2f  end %.1f"
+                      % line)
+
+
+
+# -------------------------------------------------------------------------------------- sync
+
+PROTOCOLS = ["sw", "tff", "dc", "sp"]
+
+
+def wire_ratio(proto: str, row_bytes: int) -> float:
+    if proto == "tff":
+        payload = B.UBEP_SYNC_BLOCK_BYTES - B.UBEP_SYNC_FLAG_BYTES
+        return B.UBEP_SYNC_BLOCK_BYTES * -(-row_bytes // payload) / row_bytes
+    return 1.0
+
+
+def measure(cfg: W.Config, iters: int, warmup: int = 20):
+    dev = torch.device("cuda", 0)
+    wl = W.make_workload(cfg)
+    idx = torch.from_numpy(wl.topk_idx.astype(np.int32)).to(dev)
+    x = torch.from_numpy(wl.x).view(torch.bfloat16).to(dev)
+    w = torch.from_numpy(wl.topk_w.astype(np.float32)).to(dev)
+    probe = B.Buffer(num_ranks=cfg.R, num_experts=cfg.E, hidden=cfg.H, topk=cfg.k, max_tokens=cfg.T,
+                     rows_per_rank_cap=1, dedup=cfg.dedup)
+    npr, npe, _ = probe.get_dispatch_layout(idx)
+    rows_per_rank = npr if cfg.dedup else npe.view(cfg.R, cfg.L).sum(1)
+    cap = W.round_up(max(1, int(rows_per_rank.max().item())), 16)
+    n_rows = int(rows_per_rank.sum().item())
+    probe.close()
+    buf = B.Buffer(num_ranks=cfg.R, num_experts=cfg.E, hidden=cfg.H, topk=cfg.k, max_tokens=cfg.T,
+                   rows_per_rank_cap=cap, dedup=cfg.dedup)
+    views = buf.attach_sync()
+    out = {}
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for proto in PROTOCOLS + ["main"]:
+        def call():
+            if proto == "main":
+                buf.dispatch(x, idx, w)
+            else:
+                buf.dispatch_sync(proto, x, idx, w)
+        for _ in range(warmup):
+            call()
+        torch.cuda.synchronize()
+        start.record()
+        for _ in range(iters):
+            call()
+        stop.record()
+        torch.cuda.synchronize()
+        status = buf.status()
+        if status != 0:
+            raise RuntimeError(f"{proto}: device status {status} ({B.ubep_strerror(status)})")
+        rec = {"kernel_us": start.elapsed_time(stop) * 1e3 / iters}
+        if proto != "main":
+            t = views["times"].cpu().numpy()
+            t_first = int(t[:, 0].min())
+            rec["layout_us"] = (int(t[:, 1].max()) - t_first) / 1e3
+            rec["sent_us"] = (int(t[:, 2].max()) - t_first) / 1e3
+            rec["ready_us"] = (int(t[:, 3].max()) - t_first) / 1e3
+            rec["wire_ratio"] = wire_ratio(proto, 2 * cfg.H)
+        out[proto] = rec
+    buf.close()
+    return out, n_rows
+
+
+def main_sync(argv):
+    ap = argparse.ArgumentParser(prog="bench_sweeps.py sync", description=SYNC_DOC,
+                                 formatter_class=argparse.RawDescriptionHelpFormatter)
+    ap.add_argument("--tokens", type=int, default=128)
+    ap.add_argument("--iters", type=int, default=200)
+    ap.add_argument("--hidden", type=int, nargs="*", default=[256, 1024, 4096, 7168])
+    ap.add_argument("--ranks", type=int, nargs="*", default=[8, 32, 128])
+    ap.add_argument("--markdown", action="store_true")
+    args = ap.parse_args(argv)
+    B.load()
+    rows = []
+    for R in args.ranks:
+        for H in args.hidden:
+            cfg = W.Config(f"sync_T{args.tokens}_H{H}_R{R}", T=args.tokens, H=H, E=256, R=R, k=8, seed=7000 + R + H)
+            res, n_rows = measure(cfg, args.iters)
+            rows.append({"tokens": args.tokens, "row_bytes": 2 * H, "ranks": R, "rows": n_rows, **res})
+    if not args.markdown:
+        for r in rows:
+            print(json.dumps(r))
+        return
+    print("| row bytes | ranks | rows | protocol | kernel us | layout us | sent us | ready us | wire bytes / payload byte |")
+    print("|---|---|---|---|---|---|---|---|---|")
+    for r in rows:
+        for proto in PROTOCOLS + ["main"]:
+            m = r[proto]
+            if proto == "main":
+                print(f"| {r['row_bytes']} | {r['ranks']} | {r['rows']} | main path | {m['kernel_us']:.2f} | | | | 1.000 |")
+            else:
+                print(f"| {r['row_bytes']} | {r['ranks']} | {r['rows']} | {proto.upper()} | {m['kernel_us']:.2f} | "
+                      f"{m['layout_us']:.2f} | {m['sent_us']:.2f} | {m['ready_us']:.2f} | {m['wire_ratio']:.3f} |")
+
+
+SWEEPS = {"spread": main_spread, "sync": main_sync}
+
+
+def main():
+    if len(sys.argv) < 2 or sys.argv[1] not in SWEEPS:
+        print(__doc__)
+        sys.exit(2)
+    SWEEPS[sys.argv[1]](sys.argv[2:])
+
+
+if __name__ == "__main__":
+    main()

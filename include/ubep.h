@@ -15,7 +15,7 @@
  * All functions return UBEP_OK (0) or a negative error code.  Argument errors are
  * reported synchronously and nothing is launched.  Conditions found on the device
  * (a region overflowing its capacity, a bounded flag wait running out, an expert id out
- * of range) never trap: the kernel records the first such code in a device status word,
+ * of range or repeated within a token) never trap: the kernel records the first such code in a device status word,
  * skips the offending access and returns; ubep_status() reads and clears that word.
  */
 #ifndef UBEP_H
@@ -36,7 +36,8 @@ enum {
     UBEP_ERR_CUDA = -2,      /* a CUDA runtime call failed (see ubep_last_cuda_error)         */
     UBEP_ERR_CAPACITY = -3,  /* device: a region needs more than cap rows; extra rows dropped */
     UBEP_ERR_TIMEOUT = -4,   /* device: a bounded wait on a readiness flag ran out            */
-    UBEP_ERR_BAD_INDEX = -5, /* device: an expert id outside [-1, E) was skipped              */
+    UBEP_ERR_BAD_INDEX = -5, /* device: an expert id outside [-1, E), or an expert named a    */
+                             /* second time by one token, was treated as an empty slot        */
     UBEP_ERR_ARENA = -6,     /* arena too small or not 256-byte aligned                       */
     UBEP_ERR_CHECKSUM = -7   /* device: the marker sum a receiver computed differs from the   */
                              /* checksum its senders announced (ubep_dispatch_sync, DC)       */
@@ -155,7 +156,8 @@ int ubep_set_dest_order(ubep_buffer_t *buf, const int32_t *order /*[host] [R]*/)
  * TokenCnt only (Sec. 3.2; Sec. 2.3: ranges follow from per-expert counts): counts how
  * many distinct tokens go to each rank and how many tokens select each expert, and marks
  * which ranks each token visits.  topk_idx [dev] int32 [T, k] (expert id, or -1 = empty
- * slot; ids of one token distinct).  Outputs [dev], caller-owned:
+ * slot; the ids of one token are distinct -- a repeated id is reported as UBEP_ERR_BAD_INDEX
+ * and the later slot counts as empty).  Outputs [dev], caller-owned:
  * num_tokens_per_rank [R], num_tokens_per_expert [E], is_token_in_rank u8 [T, R]
  * (any of them may be NULL).  One launch on `cuda_stream`.
  */
@@ -198,7 +200,9 @@ int ubep_get_dispatch_layout_static(const int32_t *topk_idx /*[dev]*/, int32_t T
  * assignment, optional FP8 quantisation, and the copy of every token row into the receive
  * regions of the ranks that host its experts.  x [dev] bf16 [T, H]; topk_idx [dev] int32
  * [T, k]; topk_w [dev] fp32 [T, k].  Results land in the arena (ubep_view).  Rows at or
- * beyond a region's row count are not written.  Asynchronous on `cuda_stream`; calls on
+ * beyond a region's row count are not written.  An id outside [-1, E) and the second
+ * occurrence of an expert within one token are reported (UBEP_ERR_BAD_INDEX) and handled as
+ * if the slot held -1: every output equals that of the corrected table.  Asynchronous on `cuda_stream`; calls on
  * one buffer must be stream-ordered.
  */
 int ubep_dispatch(ubep_buffer_t *buf, const void *x /*[dev]*/, const int32_t *topk_idx /*[dev]*/,

@@ -741,7 +741,7 @@ const char* ubep_strerror(int code) {
         case UBEP_ERR_CUDA: return "CUDA runtime error";
         case UBEP_ERR_CAPACITY: return "a receive region needs more rows than rows_per_rank_cap";
         case UBEP_ERR_TIMEOUT: return "a bounded wait on a readiness flag ran out";
-        case UBEP_ERR_BAD_INDEX: return "expert id out of range";
+        case UBEP_ERR_BAD_INDEX: return "expert id out of range, or an expert named twice by one token";
         case UBEP_ERR_ARENA: return "arena too small or misaligned";
         case UBEP_ERR_CHECKSUM: return "marker sum of a receive region differs from the announced checksum";
         default: return "unknown error";

@@ -10,6 +10,8 @@
 //                                     from the whole routing table (small T*k, no flags).
 //   combine_kernel<K>                 gather + fp32 weighted sum + one bf16 rounding
 //   layout_kernel                     counts only (ubep_get_dispatch_layout)
+#include <atomic>
+
 #include "ubep_kernels.h"
 #include "ubep_layout.cuh"
 #include "ubep_quant.cuh"
@@ -711,6 +713,7 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
         mbar_init(&epoch_bar, 1);
         mbar_init(&staged_bar, 1);
         abort_flag = 0;
+        epoch_sm = 0u;
         mbar_fence_init();
     }
     for (int r = tid; r < p.R; r += kThreads) arr[r] = 0;
@@ -745,6 +748,14 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
         if (kFp8 && ok) fp8_consumers<kSteal>(x);
     }
     __syncthreads();
+    const unsigned half = epoch_sm & 1u;
+    // The arrival counters of the next call live in the other half; clear them now.  This also runs
+    // when the call gives up below: otherwise the call after the next one would add to stale totals.
+    // (epoch_sm == 0: the call gave up before it learnt its epoch, so it has not used either half.)
+    if (c == 0 && epoch_sm != 0u) {
+        for (int r = tid; r < p.R; r += kThreads) p.arrival[(half ^ 1u) * p.R + r] = 0;
+        if (tid == 0) p.claimed[half ^ 1u] = 0;   // same for the count of tokens handed out
+    }
     if (abort_flag) {
         // leaving early: the newest load of every ring stage may still be landing
         if (tid == 0) {
@@ -756,14 +767,8 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
     // pieces of this CTA's rows have landed: add them to the per-region arrival counters
     // (unit: eighths of a row, so that the total does not depend on the column split)
     fence_proxy_async();   // rows written through the async proxy, counters through the generic one
-    const unsigned half = epoch_sm & 1u;
     for (int r = tid; r < p.R; r += kThreads)
         if (arr[r]) red_release_add(p.arrival + half * p.R + r, (unsigned)(arr[r] * (8 / p.parts)));
-    // the arrival counters of the next call live in the other half; clear them now
-    if (c == 0) {
-        for (int r = tid; r < p.R; r += kThreads) p.arrival[(half ^ 1u) * p.R + r] = 0;
-        if (tid == 0) p.claimed[half ^ 1u] = 0;   // same for the count of tokens handed out
-    }
     if (tid == 0) trace(p, c, kTrEnd);
 }
 
@@ -853,9 +858,15 @@ __global__ void __launch_bounds__(256) layout_kernel(const Params p, int32_t* nu
     }
     __syncthreads();
     for (int t = t0 + threadIdx.x; t < t1; t += blockDim.x) {
-        int seen[kMaxTopk];
+        int seen[kMaxTopk], seen_e[kMaxTopk];
         for (int j = 0; j < k; ++j) {
-            const int e = resolve_expert(p, t, __ldg(p.topk_idx + (size_t)t * k + j));
+            int e = resolve_expert(p, t, __ldg(p.topk_idx + (size_t)t * k + j));
+            for (int jj = 0; jj < j; ++jj)
+                if (e >= 0 && seen_e[jj] == e) {   // an expert named twice: reported, the later slot counts as empty
+                    report(p.status, kErrBadIndex);
+                    e = -1;
+                }
+            seen_e[j] = e;
             int r = -1;
             if (e >= 0) {
                 atomicAdd(&sm_i[e], 1);
@@ -957,10 +968,26 @@ static cudaError_t launch_overlapped(void (*kern)(KArgs...), int grid, int block
     return cudaLaunchKernelEx(&cfg, kern, args...);
 }
 
+// The dynamic shared-memory limit of a kernel is a sticky attribute: per kernel instance and
+// device only a larger request has to reach the runtime (the call costs host time that an
+// enqueue-bound caller sees on every dispatch).  `granted` belongs to one kernel instance.
+constexpr int kAttrDevices = 64;
+static cudaError_t allow_dynamic_smem(const void* kern, int bytes, std::atomic<int>* granted) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const bool cached = dev >= 0 && dev < kAttrDevices;
+    if (cached && granted[dev].load(std::memory_order_relaxed) >= bytes) return cudaSuccess;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess && cached) granted[dev].store(bytes, std::memory_order_relaxed);
+    return e;
+}
+
 template <int kMode, bool kFp8, bool kSteal>
 static cudaError_t launch_dispatch_s(const Params& p, const SmemPlan& pl, cudaStream_t st) {
     auto kern = dispatch_kernel<kMode, kFp8, kSteal>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl.total);
+    static std::atomic<int> granted[kAttrDevices];
+    cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(kern), pl.total, granted);
     if (e != cudaSuccess) return e;
     return launch_overlapped(kern, p.grid, kThreads, (size_t)pl.total, st, p, pl);
 }
@@ -976,8 +1003,8 @@ cudaError_t launch_dispatch(const Params& p, int mode, const SmemPlan& pl, cudaS
     *launches = 1;
     if (mode == kModePhased) {
         const int count_smem = pl.off_pos - pl.off_ids;   // ids + both bitmap arrays
-        if ((e = cudaFuncSetAttribute(count_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, count_smem)) !=
-            cudaSuccess)
+        static std::atomic<int> granted[kAttrDevices];
+        if ((e = allow_dynamic_smem(reinterpret_cast<const void*>(count_kernel), count_smem, granted)) != cudaSuccess)
             return e;
         count_kernel<<<p.nchunks, 256, count_smem, st>>>(p, pl);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;

@@ -135,7 +135,13 @@ __device__ __forceinline__ unsigned transpose32(unsigned x, int lane) {
 // that word its token selected, the warp transposes the tile and stores it bin-major.
 // With many units per warp (a whole routing table) a unit covers four words instead: the token's
 // slots are read once and sorted into four registers, which costs a third of the instructions.
-static __device__ void build_bin_maps(const Params& p, const int* ids, int ntok, const BinMaps& bmaps, int gw, int nw,
+//
+// A token may name an expert once.  A second slot with the same expert finds the expert's bit
+// already set: it is reported (kErrBadIndex) and its staged id is overwritten with -1, so that
+// every later step treats it as an empty slot.  (Warps working on other words of the same tokens
+// may still read the old value meanwhile; they only take the rank bit from it, which the first
+// occurrence sets as well.)
+static __device__ void build_bin_maps(const Params& p, int* ids, int ntok, const BinMaps& bmaps, int gw, int nw,
                                int lane) {
     const int k = p.k;
     const int units = bmaps.groups * bmaps.wb;
@@ -152,6 +158,14 @@ static __device__ void build_bin_maps(const Params& p, const int* ids, int ntok,
                     const int e = slot_expert(v), rb = p.E + slot_rank(v);
                     const int we = (e >> 5) - w0, wr = (rb >> 5) - w0;
                     const unsigned be = 1u << (e & 31), br = 1u << (rb & 31);
+                    bool dup = false;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) dup = dup || (we == q && (m[q] & be) != 0u);
+                    if (dup) {
+                        report(p.status, kErrBadIndex);
+                        ids[tl * k + j] = -1;
+                        continue;
+                    }
 #pragma unroll
                     for (int q = 0; q < 4; ++q) m[q] |= (we == q ? be : 0u) | (wr == q ? br : 0u);
                 }
@@ -171,7 +185,13 @@ static __device__ void build_bin_maps(const Params& p, const int* ids, int ntok,
                 const int v = ids[tl * k + j];
                 if (v < 0) continue;
                 const int e = slot_expert(v), rb = p.E + slot_rank(v);
-                m |= ((e >> 5) == w ? 1u << (e & 31) : 0u) | ((rb >> 5) == w ? 1u << (rb & 31) : 0u);
+                const unsigned be = (e >> 5) == w ? 1u << (e & 31) : 0u;
+                if (m & be) {
+                    report(p.status, kErrBadIndex);
+                    ids[tl * k + j] = -1;
+                    continue;
+                }
+                m |= be | ((rb >> 5) == w ? 1u << (rb & 31) : 0u);
             }
         }
         bmaps.bm[(size_t)g * bmaps.bp + w * 32 + lane] = transpose32(m, lane);
@@ -385,7 +405,7 @@ __device__ void finalize_chunk(const Params& p, int t0, int t1, const int* ids, 
 // the total (tot), the count among the tokens before t0 (pre) and per expert the offset inside its
 // rank's region (eo).  Run by the gn threads (nw warps) that share barrier `bar`; ends with that
 // barrier.  Used by every kernel in which a CTA derives the layout alone.
-static __device__ void local_counts_all_bins(const Params& p, const int* ids, const BinMaps& bmaps, int t0, int* tot,
+static __device__ void local_counts_all_bins(const Params& p, int* ids, const BinMaps& bmaps, int t0, int* tot,
                                              int* pre, int* eo, int gtid, int gn, int gw, int nw, int lane, int bar) {
     build_bin_maps(p, ids, p.T, bmaps, gw, nw, lane);
     group_sync(bar, gn);
@@ -473,10 +493,24 @@ static __device__ void local_stage_and_rank_maps(const Params& p, int* ids, cons
 #pragma unroll
                     for (int u = 0; u < 8; ++u) raw[u] = j0 + u < k ? __ldg(src + j0 + u) : -1;
                 }
+                int res[8];
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
                     if (j0 + u >= k) break;
-                    const int e = resolve_expert(p, t, raw[u]);
+                    int e = resolve_expert(p, t, raw[u]);
+                    // an expert named twice by one token: the later slot is reported and left empty
+                    bool dup = false;
+#pragma unroll
+                    for (int u2 = 0; u2 < u; ++u2) dup = dup || (e >= 0 && res[u2] == e);
+                    for (int jj = 0; jj < j0; ++jj) {
+                        const int v2 = ids[t * k + jj];
+                        dup = dup || (e >= 0 && v2 >= 0 && slot_expert(v2) == e);
+                    }
+                    if (dup) {
+                        report(p.status, kErrBadIndex);
+                        e = -1;
+                    }
+                    res[u] = e;
                     int packed = -1;
                     if (e >= 0) {
                         const int r = fast_div(e, p.L_magic);

@@ -229,6 +229,49 @@ def test_out_of_range_expert_id_is_reported_and_skipped():
     assert np.array_equal(buf.slot_row[:cfg.T].cpu().numpy(), lay.slot_row)
 
 
+@pytest.mark.parametrize("pipeline", [PHASED, FUSED, LOCAL])
+@pytest.mark.parametrize("payload,dedup,k", [(0, 0, 4), (0, 1, 8), (1, 0, 3), (0, 1, 12)])
+def test_expert_named_twice_by_a_token_is_reported_and_the_later_slot_left_empty(pipeline, payload, dedup, k):
+    """The ids of one token must be distinct.  A repeated id is reported and the later slot is
+    handled as empty: every output equals what the oracle gives for the table with that slot -1
+    (the oracle itself rejects the uncorrected table)."""
+    cfg = W.Config("dup", T=210, H=256, E=48, R=6, k=k, payload=payload, dedup=dedup, seed=40 + k)
+    wl = W.with_empty_slots(W.make_workload(cfg), 0.1, seed=5)
+    bad = wl.topk_idx.copy()
+    fixed = wl.topk_idx.copy()
+    rng = np.random.default_rng(9)
+    n_dup = 0
+    for t in rng.choice(cfg.T, size=25, replace=False):
+        live = np.nonzero(bad[t] >= 0)[0]
+        if len(live) < 2:
+            continue
+        a, b = sorted(rng.choice(live, size=2, replace=False))
+        bad[t, b] = bad[t, a]          # slot b repeats slot a's expert
+        fixed[t, b] = -1
+        n_dup += 1
+    assert n_dup > 10
+    with pytest.raises(Exception):
+        oracle.layout(bad, cfg.E, cfg.R, cfg.S, cfg.dedup)
+    ref = W.Workload(cfg, wl.x, fixed, wl.topk_w)
+    ids, lay, cap, recv = Hn.oracle_reference(ref)
+    buf = Hn.make_buffer(cfg, cap, pipeline=pipeline)
+    x, _, w, _, _ = Hn.device_inputs(wl)
+    idx = Hn.to_dev(bad.astype(np.int32))
+    buf.dispatch(x, idx, w)
+    assert buf.status() == B.UBEP_ERR_BAD_INDEX
+    Hn.check_dispatch(buf, ref, lay, cap, recv)
+    y_bits = W.make_expert_outputs(cfg, cap)
+    out = buf.combine(Hn.to_dev(y_bits, torch.bfloat16), w)
+    want, _ = oracle.combine(y_bits, fixed, wl.topk_w, lay.slot_row, cfg.E, cfg.R)
+    Hn.check_combine(out, want)
+    # the counts-only entry point sees the same table the same way
+    npr, npe, itr = buf.get_dispatch_layout(idx)
+    assert buf.status() == B.UBEP_ERR_BAD_INDEX
+    assert np.array_equal(npr.cpu().numpy(), lay.num_tokens_per_rank)
+    assert np.array_equal(npe.cpu().numpy(), lay.num_tokens_per_expert)
+    assert np.array_equal(itr.cpu().numpy(), lay.is_token_in_rank)
+
+
 def test_bad_arguments_are_rejected_synchronously():
     cfg = small(64)
     wl = W.make_workload(cfg)
@@ -292,3 +335,12 @@ def test_bounded_wait_reports_timeout_and_the_context_survives():
     assert buf.status() == B.UBEP_ERR_TIMEOUT
     buf.dispatch(x, idx, w)
     Hn.check_dispatch(buf, wl, lay, cap, recv)
+    # A call that gives up after calls that went through: the arrival counters of the calls that
+    # follow must start from zero again (the call that gave up still clears the other half).
+    buf.dispatch(x, idx, w)                       # ok, leaves its totals in one half
+    B.ubep_debug_withhold_flag(buf.handle, 1)
+    buf.dispatch(x, idx, w)                       # gives up; uses the other half
+    assert buf.status() == B.UBEP_ERR_TIMEOUT
+    for _ in range(2):                            # both halves come round once more
+        buf.dispatch(x, idx, w)
+        Hn.check_dispatch(buf, wl, lay, cap, recv, arrival=True)

@@ -5,11 +5,13 @@ memory plan and are handed input and output tensors only, so they cannot give th
 an arena either.  `ubep_get_dispatch_layout_static` serves them from a fixed scratch array
 inside the library.  This test calls it through the C ABI twice in a row (different routing
 each time, so stale scratch from the first call would show) and requires exactly the output
-of the ordinary entry point.  It is collected last on purpose."""
+of the ordinary entry point -- and, so that a fault shared by both would not pass, exactly the
+counts of the CPU oracle.  It is collected last on purpose."""
 import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2607_06202_b200 import binding as B
 from paper_2607_06202_b200 import workload as W
 
@@ -38,6 +40,10 @@ def test_static_scratch_entry_point_matches_the_ordinary_one_twice():
         B.ubep_get_dispatch_layout_static(idx, cfg.T, cfg.k, cfg.E, cfg.R, got_r, got_e, got_m)
         torch.cuda.synchronize()
         assert torch.equal(got_r, npr) and torch.equal(got_e, npe) and torch.equal(got_m, itr)
+        lay = oracle.layout(wl.topk_idx, cfg.E, cfg.R, cfg.S, 0)
+        assert np.array_equal(got_r.cpu().numpy(), lay.num_tokens_per_rank)
+        assert np.array_equal(got_e.cpu().numpy(), lay.num_tokens_per_expert)
+        assert np.array_equal(got_m.cpu().numpy(), lay.is_token_in_rank)
 
 
 def test_static_scratch_entry_point_rejects_sizes_beyond_its_array():
