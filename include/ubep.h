@@ -424,11 +424,23 @@ int ubep_debug_trace(ubep_buffer_t *buf, int32_t enable);
 
 /*
  * Warp-role split of the FP8 dispatch kernel (the paper's core-allocation question, Sec. 3.2
- * and App. A / C: how many cores count and how many send): n of the CTA's 16 warps quantise
- * rows (1 <= n <= 14, default 14); one warp loads, one issues the stores, the rest idle once
- * the layout is done.  Results never depend on it.
+ * "most cores send tokens, a few compute token counts", and App. A / C: how many cores count and
+ * how many send).  Of the CTA's 16 warps one loads rows and one issues the stores.
+ *
+ * ubep_debug_set_count_warps: n warps (the store issuer among them) form the count group that
+ * computes the layout -- TokenCnt, the flag exchange, CalCumSum, row assignment -- while the
+ * remaining 15 - n warps already quantise the rows the loader has fetched into a ring of
+ * quantised rows that waits for the layout (1 <= n <= 13; default 4).  n = 0: all 15 warps
+ * compute the layout and 14 of them quantise afterwards.  Applies to the PHASED and FUSED
+ * schedules; the flag-free LOCAL schedule, whose layout waits for nobody, always runs as n = 0.
+ * ubep_debug_set_quant_warps: at most n warps quantise (1 <= n <= 14, default 14), the rest idle.
+ * ubep_debug_set_prefetch_rows: the loader fetches at most n rows before the layout is done
+ * (default: as many as the rings hold).
+ * Results never depend on any of them.
  */
 int ubep_debug_set_quant_warps(ubep_buffer_t *buf, int32_t n);
+int ubep_debug_set_count_warps(ubep_buffer_t *buf, int32_t n);
+int ubep_debug_set_prefetch_rows(ubep_buffer_t *buf, int32_t n);
 
 /* Text of the last CUDA runtime error seen by this buffer's calls ("" if none). */
 const char *ubep_last_cuda_error(const ubep_buffer_t *buf);

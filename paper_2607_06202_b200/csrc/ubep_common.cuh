@@ -19,7 +19,9 @@ constexpr int kMaxChunks = 320;        // scan keeps chunks/32 values per lane i
 constexpr int kMaxStages = 16;         // rows in the shared-memory ring
 constexpr int kRankWordsHost = 4;      // the rank-level fast path handles up to 128 ranks
 constexpr int kStealBlock = 2;         // tokens handed out per claim
-constexpr int kOutStages = 4;          // quantised rows waiting for their bulk stores (FP8)
+constexpr int kOutStages = 4;          // FP8, quantising after the layout: quantised rows waiting for their stores
+constexpr int kMaxOutStages = 24;      // FP8, quantising beside the layout: at most this many quantised rows wait
+constexpr int kStorePending = 3;       // FP8: rows whose bulk stores may still be reading shared memory
 constexpr int kTraceSlots = 16;        // per-CTA phase time stamps (optional tracing)
 constexpr int kModePhased = 1, kModeFused = 2, kModeLocal = 3;
 // Every wait in the kernels gives up after this many nanoseconds of wall time.
@@ -76,13 +78,18 @@ struct Params {
     // token stealing (large T): chunk c's tokens are handed out in blocks through cursor[c],
     // to its owner and, once pos_flag[c] holds the epoch, to CTAs that ran out of work
     int steal;            // 1 = on
-    int quant_warps;      // FP8: warps that quantise (2 .. kWarps - 2); the others idle after the layout
+    int quant_warps;      // FP8: warps that quantise at most (1 .. kWarps - 2)
+    int count_warps;      // FP8 with flags or kernel boundaries: warps 1 .. count_warps compute the layout while the
+                          // warps after them already quantise the rows the loader has fetched (0 = all 15 warps
+                          // compute the layout and quantise afterwards)
+    int prefetch_rows;    // FP8: rows the loader may fetch before the layout is done (the rings bound it as well)
     int32_t* copy_pos;    // [T, k] destinations in issue order (-1 = no copy), for thieves
     unsigned* cursor;     // [nchunks] tokens of the chunk handed out so far
     unsigned* pos_flag;   // [nchunks] == epoch: copy_pos of the chunk is final
     unsigned* claimed;    // [2] tokens handed out in this dispatch (half = epoch & 1)
     int32_t* status;
-    unsigned long long* trace;  // optional [nchunks, kTraceSlots] globaltimer stamps, or null
+    unsigned long long* trace;  // optional [nchunks, kTraceSlots] phase stamps in ns, or null
+    unsigned ns_per_cycle_q20;  // nanoseconds per SM cycle times 2^20 (the clock the stamps are derived with)
     // ranks on different GPUs (sharded use): this GPU is rank my_rank and moves tokens [tok0, tok1)
     int my_rank, tok0, tok1;
     const long long* peer_delta;  // [R] byte distance from this arena to the arena of rank r
@@ -101,7 +108,11 @@ __device__ __forceinline__ int chunk_of(int b, int T, int n) {
     return (int)((((int64_t)b + 1) * n - 1) / T);
 }
 
-__device__ __forceinline__ void report(int32_t* status, int code) { atomicCAS(status, 0, code); }
+// Records the first asynchronous condition of a call.  Out of line on purpose: it is called from
+// many places that almost never take it, and the kernels run every piece of their code once per
+// launch, so what they execute has to stay small enough for the instruction cache (measured: a few
+// hundred instructions more on the way to the first copy cost the decode-sized dispatch microseconds).
+static __device__ __noinline__ void report(int32_t* status, int code) { atomicCAS(status, 0, code); }
 
 __device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
     unsigned v;
@@ -132,6 +143,26 @@ __device__ __forceinline__ unsigned read_epoch_and_check_in(const Params& p) {
 }
 
 
+// The flag-free kernel needs the epoch only to pick the half of the arrival counters it adds to at
+// its very end, so it splits read_epoch_and_check_in in three: a relaxed load issued early (nothing
+// is ordered against it, so it costs the thread nothing until the value is used), the ticket once
+// the value has arrived, and the last CTA's update when the ticket's answer is finally looked at.
+__device__ __forceinline__ unsigned ld_relaxed(const unsigned* p) {
+    unsigned v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ unsigned epoch_from_counter(unsigned ctr) {
+    const unsigned e = ctr + 1u;
+    return e == 0u ? 1u : e;
+}
+__device__ __forceinline__ void epoch_finish_check_in(const Params& p, unsigned ticket, unsigned e) {
+    if (ticket == (unsigned)p.grid - 1u) {
+        *p.done_ticket = 0u;
+        *p.epoch_ctr = e;
+    }
+}
+
 __device__ __forceinline__ unsigned long long global_ns() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
@@ -141,8 +172,27 @@ __device__ __forceinline__ unsigned long long global_ns() {
 // Optional tracing: per-CTA %globaltimer stamp of a phase boundary.
 enum TracePhase { kTrStart = 0, kTrCounted, kTrHistSeen, kTrScanned, kTrScanSeen, kTrFinalized, kTrReady,
                   kTrFirstRow, kTrIssued, kTrStored, kTrEnd };
+// The stamps are nanoseconds of the device timer.  Reading that timer is slow enough to show in what
+// it measures, so a CTA reads it once, when it starts, and derives later stamps from the SM's cycle
+// counter (cheap to read) at the SM clock the host passed in -- exact enough for phase budgets.
+__device__ __forceinline__ unsigned long long* trace_origin() {
+    __shared__ unsigned long long origin[2];   // device timer and cycle counter at the CTA's start
+    return origin;
+}
+__device__ __forceinline__ unsigned long long trace_ns(const Params& p) {
+    const unsigned long long* o = trace_origin();
+    return o[0] + (((unsigned long long)(clock64() - (long long)o[1]) * (unsigned long long)p.ns_per_cycle_q20) >> 20);
+}
+// One thread, before the barrier that lets the CTA's roles go.
+__device__ __forceinline__ void trace_begin(const Params& p, int cta) {
+    if (!p.trace) return;
+    unsigned long long* o = trace_origin();
+    o[0] = global_ns();
+    o[1] = (unsigned long long)clock64();
+    p.trace[(size_t)cta * kTraceSlots + kTrStart] = o[0];
+}
 __device__ __forceinline__ void trace(const Params& p, int cta, int phase) {
-    if (p.trace) p.trace[(size_t)cta * kTraceSlots + phase] = global_ns();
+    if (p.trace) p.trace[(size_t)cta * kTraceSlots + phase] = trace_ns(p);
 }
 
 // Wait until *flag == epoch.  Gives up after kWaitLimitNs (or as soon as *abort is set) and
@@ -188,7 +238,19 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, unsigned parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait on an mbarrier phase; false after kWaitLimitNs or on abort.
+// Test of an mbarrier phase that may suspend the thread for up to about `hint_ns` while the phase
+// is incomplete, instead of spinning in the issue slots other warps of the CTA need.
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity, unsigned hint_ns) {
+    unsigned ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait on an mbarrier phase; false after kWaitLimitNs or on abort.  Spins: the quickest
+// to notice the phase, for a warp whose reaction time is on the critical path.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity, volatile int* abort) {
     for (unsigned i = 0; i < 128; ++i)
         if (mbar_test_wait(bar, parity)) return true;
@@ -198,6 +260,17 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity, volati
         if (abort && *abort) return false;
         if ((i & 63u) == 0 && global_ns() > t_end) return false;
         __nanosleep(40);
+    }
+}
+// The same wait for warps that are many and in no hurry (the quantising warps): suspended by the
+// hardware while the phase is incomplete, so that they leave the issue slots to the others.
+__device__ __forceinline__ bool mbar_wait_idle(uint64_t* bar, unsigned parity, volatile int* abort) {
+    if (mbar_test_wait(bar, parity)) return true;
+    const unsigned long long t_end = global_ns() + kWaitLimitNs;
+    for (;;) {
+        if (mbar_try_wait(bar, parity, 1000u)) return true;
+        if (abort && *abort) return false;
+        if (global_ns() > t_end) return false;
     }
 }
 // global -> shared bulk copy, completion counted in bytes on `bar`.
@@ -230,7 +303,7 @@ __device__ __forceinline__ void fence_proxy_async_smem() {
 // Where the dispatch kernel keeps things in dynamic shared memory (byte offsets).
 struct SmemPlan {
     int stages, stage_bytes;          // input row ring
-    int out_stage_bytes;              // FP8: kOutStages quantised rows
+    int out_stages, out_stage_bytes;  // FP8: ring of quantised rows
     int map_groups, map_wb, map_bp;   // bin bitmaps: 32-token groups, words of bins, padded bins
     int off_out, off_ids, off_mask, off_bm, off_pos, off_key, off_ord, off_w, off_hist, off_arr, off_order;
     int off_item;                     // per ring stage: where its token comes from, positions of stolen tokens

@@ -1,6 +1,7 @@
 // C ABI of the library (declared in include/ubep.h): argument checks, arena layout and
 // kernel launches.  No device memory is allocated here and no stream is created.
 #include <atomic>
+#include <climits>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -20,6 +21,7 @@ std::atomic<uint64_t> g_launches{0};
 
 constexpr size_t kAlign = 256;
 constexpr int kStealMinTokensPerChunk = 40;  // shorter slices: the hand-out costs more than the tail it removes (measured)
+constexpr int kDefaultCountWarps = 4;            // FP8: warps of the layout group while the others quantise (measured sweep)
 constexpr int64_t kLocalMaxSlots = 8192;        // small-T limit of the combine launch mode and of the protocol / sharded paths
 constexpr int64_t kLocalFastMaxSlots = 14336;   // AUTO: flag-free kernel with the rank-level fast path up to this many slots
 constexpr int64_t kLocalMaxWeight = 18432;      // AUTO: flag-free kernel over every bin up to this many slots x bin words
@@ -140,10 +142,13 @@ struct ubep_buffer {
     uint8_t* arena;
     int num_sms;
     int max_smem;
+    int sm_khz;
     uint32_t epoch;
     int32_t withhold;
     int32_t tracing;
     int32_t quant_warps;
+    int32_t count_warps;     // FP8 with flags / kernel boundaries: warps that compute the layout (0 = all, quantise afterwards)
+    int32_t prefetch_rows;   // FP8: rows fetched before the layout is done, at most
     cudaStream_t last_stream;
     const int32_t* phys;
     const int32_t* ncopies;
@@ -205,6 +210,8 @@ Params make_params(ubep_buffer* b, int T) {
     p.claimed = at<unsigned>(b, a.claimed);
     p.steal = 0;
     p.quant_warps = b->quant_warps;
+    p.count_warps = b->count_warps;
+    p.prefetch_rows = b->prefetch_rows;
     p.chunk_hist = at<int32_t>(b, a.chunk_hist);
     p.partial = at<int32_t>(b, a.partial);
     p.chunk_base = at<int32_t>(b, a.chunk_base);
@@ -213,6 +220,7 @@ Params make_params(ubep_buffer* b, int T) {
     p.arrival = at<unsigned>(b, a.off[UBEP_VIEW_ARRIVAL]);
     p.status = at<int32_t>(b, a.status);
     p.trace = b->tracing ? at<unsigned long long>(b, a.trace) : nullptr;
+    p.ns_per_cycle_q20 = (unsigned)((1000000.0 / (double)b->sm_khz) * 1048576.0 + 0.5);
     p.my_rank = b->my_rank;
     p.tok0 = 0;
     p.tok1 = T;
@@ -261,6 +269,7 @@ int ubep_buffer_create(const ubep_config_t* cfg, void* dev_arena, size_t bytes, 
     b->cfg = *cfg;
     b->num_sms = prop.multiProcessorCount;
     b->max_smem = (int)prop.sharedMemPerBlockOptin;
+    b->sm_khz = prop.clockRate > 0 ? prop.clockRate : 1965000;
     int n = cfg->num_ctas > 0 ? cfg->num_ctas : b->num_sms;
     if (n > b->num_sms) n = b->num_sms;  // all CTAs of the persistent kernel must be resident
     if (n > ubep::kMaxChunks) n = ubep::kMaxChunks;
@@ -270,6 +279,8 @@ int ubep_buffer_create(const ubep_config_t* cfg, void* dev_arena, size_t bytes, 
     b->withhold = -1;
     b->tracing = 0;
     b->quant_warps = ubep::kWarps - 2;
+    b->count_warps = kDefaultCountWarps;
+    b->prefetch_rows = INT32_MAX;
     b->last_stream = nullptr;
     b->phys = nullptr;
     b->ncopies = nullptr;
@@ -729,6 +740,18 @@ int ubep_debug_trace(ubep_buffer_t* buf, int32_t enable) {
 int ubep_debug_set_quant_warps(ubep_buffer_t* buf, int32_t n) {
     if (!buf || n < 1 || n > ubep::kWarps - 2) return UBEP_ERR_ARG;
     buf->quant_warps = n;
+    return UBEP_OK;
+}
+
+int ubep_debug_set_count_warps(ubep_buffer_t* buf, int32_t n) {
+    if (!buf || n < 0 || n > ubep::kWarps - 3) return UBEP_ERR_ARG;
+    buf->count_warps = n;
+    return UBEP_OK;
+}
+
+int ubep_debug_set_prefetch_rows(ubep_buffer_t* buf, int32_t n) {
+    if (!buf || n < 1) return UBEP_ERR_ARG;
+    buf->prefetch_rows = n;
     return UBEP_OK;
 }
 

@@ -50,6 +50,10 @@ struct Cta {
     uint64_t *full_bar, *empty_bar, *out_full, *out_empty, *ready_bar, *epoch_bar, *staged_bar;
     int* abort_flag;
     int tid, lane, warp, c, part, ch, t0, t1, ntok, stages, nq;
+    int gn, nw;        // layout (count) group: warps 1 .. nw, gn = 32 * nw threads
+    int out_stages;    // FP8: depth of the ring of quantised rows
+    int qwarp0;        // FP8: first quantising warp (warps qwarp0 .. qwarp0 + nq - 1 quantise)
+    bool beside;       // FP8: the quantising warps are not layout warps and run beside the layout
     int *ids_sm, *pos, *pos_raw, *key;
     float* w_sm;
     BinMaps bmaps;
@@ -62,7 +66,7 @@ struct Cta {
 };
 
 // The role functions below keep the names the kernel uses for these.
-#define UBEP_CTA_LOCALS(x)                                                                                   \
+#define UBEP_CTA_LOCALS(x, all15)                                                                              \
     [[maybe_unused]] const Params& p = (x).p;                                                                \
     [[maybe_unused]] const SmemPlan& pl = (x).pl;                                                            \
     [[maybe_unused]] uint8_t* const smem = (x).smem;                                                         \
@@ -89,8 +93,10 @@ struct Cta {
     [[maybe_unused]] const size_t in_off = (x).in_off, out_off = (x).out_off;                                \
     [[maybe_unused]] const bool fast_local = (x).fast_local;                                                 \
     [[maybe_unused]] int& issued = (x).issued;                                                               \
-    [[maybe_unused]] constexpr int gn = kThreads - 32; /* layout group: warps 1..15 */                       \
-    [[maybe_unused]] constexpr int nw = kWarps - 1;                                                          \
+    /* layout group: warps 1 .. nw; a compile-time constant where it is always all 15 */                    \
+    [[maybe_unused]] const int nw = (all15) ? kWarps - 1 : (x).nw;                                           \
+    [[maybe_unused]] const int gn = nw * 32;                                                                 \
+    [[maybe_unused]] const int out_stages = (x).out_stages;                                                  \
     [[maybe_unused]] const int gtid = (x).tid - 32, gw = (x).warp - 1
 
 // ------------------------------------------------------------------------ mover warp
@@ -109,7 +115,7 @@ __device__ __forceinline__ void mover_warp(Cta& x) {
         }
         x.epoch = __shfl_sync(0xffffffffu, ep, 0);
     }
-    UBEP_CTA_LOCALS(x);
+    UBEP_CTA_LOCALS(x, !kFp8);
     // Lane 0 issues the TMA loads; for bf16 rows lane j issues the TMA store of slot j,
     // so the k copies of a row are issued side by side.  Tokens come from a feeder: the
     // CTA's own chunk first and, when stealing is on, blocks of other chunks afterwards.
@@ -177,11 +183,18 @@ __device__ __forceinline__ void mover_warp(Cta& x) {
         return 1;
     };
     int* item_src = reinterpret_cast<int*>(smem + pl.off_item);           // [stages] (chunk << 16 | index), -1 = end
-    int* item_pos = item_src + kMaxStages + kOutStages;                   // [stages, k] destinations of stolen tokens
+    int* item_pos = item_src + kMaxStages + kMaxOutStages;                // [stages, k] destinations of stolen tokens
     int head = 0, tail = 0;   // rows whose load was issued / whose copies were issued
     // load of the feeder's next token into ring stage head % stages
     auto issue_item = [&](int tl) {
         const int s = head % stages;
+        // What travels with the row is written before the load is started: the consumers read it
+        // as soon as the row has landed.
+        if (kSteal && v != ch) {   // a stolen token: its destinations come from the owner's published list
+            for (int j = lane; j < p.k; j += 32)
+                item_pos[s * p.k + j] = __ldcg(p.copy_pos + (size_t)(v_t0 + tl) * p.k + j);
+            __syncwarp();
+        }
         if (lane == 0) {
             if (kSteal) item_src[s] = (v << 16) | tl;
             mbar_arrive_expect_tx(&full_bar[s], in_bytes);
@@ -189,9 +202,6 @@ __device__ __forceinline__ void mover_warp(Cta& x) {
                       reinterpret_cast<const uint8_t*>(p.x) + (size_t)(v_t0 + tl) * p.H * 2 + in_off, in_bytes,
                       &full_bar[s]);
         }
-        if (v != ch)   // a stolen token: its destinations come from the owner's published list
-            for (int j = lane; j < p.k; j += 32)
-                item_pos[s * p.k + j] = __ldcg(p.copy_pos + (size_t)(v_t0 + tl) * p.k + j);
         if (kSteal) __syncwarp();
         ++head;
     };
@@ -291,21 +301,28 @@ __device__ __forceinline__ void mover_warp(Cta& x) {
             const RankMaps rm{bmaps.bm, bmaps.mask_t, (p.R + 31) / 32, ((p.R + 31) / 32) * 32, (p.T + 31) / 32};
             local_stage_and_rank_maps(p, ids_sm, rm, 0, kWarps, lane);   // the table first, the rows after it
             group_sync(2, kThreads);
-        } else if (kMode == kModeLocal) {
+        } else if (kMode == kModeLocal || x.beside) {
+            // the routing table first: it is the one load the layout waits for
             ok = mbar_wait(x.staged_bar, 0, abortp);
             ok = __all_sync(0xffffffffu, ok);
         }
         // loader only; the quantising warps free the stages.  A closing item with no row
-        // tells them (and through them the store issuer) that nothing follows.
+        // tells them (and through them the store issuer) that nothing follows.  Rows are fetched as
+        // far ahead as the rings allow, at most prefetch_rows of them before the layout is done.
         int tl = 0;
+        bool ready_seen = kMode == kModeLocal;   // (the flag-free kernel: its quantisers start after the layout)
+        auto wait_ready_at = [&](int n) -> bool {   // warp-uniform
+            if (ready_seen || n < p.prefetch_rows) return true;
+            bool r = true;
+            if (lane == 0) r = mbar_wait(&ready_bar, 0, abortp);
+            ready_seen = true;
+            return __shfl_sync(0xffffffffu, (int)r, 0) != 0;
+        };
         if (!kSteal) {
             // the CTA's own rows only: one thread, as far ahead as the ring allows
             while (ok && head < ntok) {
-                if (kMode != kModeLocal && head == early) {   // the rest once the layout is done
-                    if (lane == 0) ok = mbar_wait(&ready_bar, 0, abortp);
-                    ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-                    if (!ok) break;
-                }
+                ok = wait_ready_at(head);
+                if (!ok) break;
                 if (head >= stages) {
                     if (lane == 0) ok = mbar_wait(&empty_bar[head % stages], ((head / stages) - 1) & 1, abortp);
                     ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
@@ -324,11 +341,8 @@ __device__ __forceinline__ void mover_warp(Cta& x) {
                 drained = mbar_test_wait(&empty_bar[hs % stages], (hs / stages) & 1);
                 drained = __all_sync(0xffffffffu, drained);
             }
-            if (head == early) {   // the rest once the layout is done
-                ok = mbar_wait(&ready_bar, 0, abortp);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-            }
+            ok = wait_ready_at(head);
+            if (!ok) break;
             const int got = feeder_done ? 0 : next_token(tl, drained);
             if (got == 2) {
                 const int hs = head - 3;   // wait for the queue to drain, then ask again
@@ -337,7 +351,6 @@ __device__ __forceinline__ void mover_warp(Cta& x) {
                 continue;
             }
             const int s = head % stages;
-            if (got == 0 && !kSteal) break;
             if (head >= stages) {
                 ok = mbar_wait(&empty_bar[s], ((head / stages) - 1) & 1, abortp);
                 ok = __all_sync(0xffffffffu, ok);
@@ -347,7 +360,7 @@ __device__ __forceinline__ void mover_warp(Cta& x) {
                 issue_item(tl);
                 issued = head;
             } else {
-                if (kSteal && lane == 0) {   // without stealing the consumers know the row count
+                if (lane == 0) {   // (without stealing the consumers know the row count)
                     item_src[s] = -1;
                     mbar_arrive(&full_bar[s]);
                 }
@@ -370,7 +383,7 @@ __device__ __forceinline__ void mover_warp(Cta& x) {
 // wait ran out.
 template <int kMode, bool kFp8, bool kSteal>
 __device__ __forceinline__ bool layout_group(Cta& x) {
-    UBEP_CTA_LOCALS(x);
+    UBEP_CTA_LOCALS(x, !kFp8);
     bool ok = true;
     const int* ids = ids_sm;  // staged slots of this CTA's tokens
     // Small global reads whose values are needed only after the first barriers: issue the
@@ -394,31 +407,55 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
         stage_small();
         group_sync(2, kThreads);
         if (gtid == 0) trace(p, c, kTrCounted);
-        local_rows_dedup(p, t0, t1, ids_sm, rm, c, order_sm, pos_raw, key, row_sm, arr, gtid, gn);
-        group_sync(1, gn);
-        if (gtid == 0) trace(p, c, kTrFinalized);
-        if (p.ordered) {   // a destination table is set: the copies of a token in its order (else pos_raw is pos)
-            order_destinations(p, pos_raw, key, pos, ntok * p.k, gtid, gn);
-            group_sync(1, gn);
-        }
-        if (gtid == 0) {
-            mbar_arrive(&ready_bar);
-            trace(p, c, kTrReady);
-            *x.epoch_late = read_epoch_and_check_in(p);   // nothing needs it before the kernel's last lines
-        }
-        if (part == 0) {
-            float* w_own = reinterpret_cast<float*>(key);   // the ordering keys are no longer needed
-            for (int i = gtid; i < ntok * p.k; i += gn) w_own[i] = __ldg(p.topk_w + (size_t)t0 * p.k + i);
-        }
-        group_sync(1, gn);
-        if (part == 0) local_meta_dedup(p, t0, t1, ids_sm, pos_raw, row_sm, reinterpret_cast<float*>(key), gtid, gn);
-        {
+        // From here the group splits.  Assigning rows to the CTA's own few tokens keeps a handful of
+        // threads busy, and nothing expert-level depends on it: warps 1..4 (the row group) assign the
+        // rows, release the movers and write the metadata of the own tokens, while the other warps
+        // (the duty group) already derive the expert-level outputs from the staged table.  (One after
+        // the other, the expert-level outputs ended after the last copy and set the kernel's duration.)
+        constexpr int kRowWarps = 4, kRowThreads = kRowWarps * 32;
+        if (gw < kRowWarps) {
+            const int rn = kRowThreads;
+            local_rows_dedup(p, t0, t1, ids_sm, rm, c, order_sm, pos_raw, key, row_sm, arr, gtid, rn);
+            group_sync(1, rn);
+            if (gtid == 0) trace(p, c, kTrFinalized);
+            if (p.ordered) {   // a destination table is set: the copies of a token in its order (else pos_raw is pos)
+                order_destinations(p, pos_raw, key, pos, ntok * p.k, gtid, rn);
+                group_sync(1, rn);
+            }
+            unsigned ticket = 0u, ep_mine = 0u;
+            if (gtid == 0) {
+                mbar_arrive(&ready_bar);
+                trace(p, c, kTrReady);
+                // The epoch: nothing needs it before the kernel's last lines.  A relaxed load (nothing
+                // is ordered against it); its value is in hand before the ticket is taken -- the store
+                // to shared memory needs it -- and the ticket's answer is looked at at the end.
+                ep_mine = epoch_from_counter(ld_relaxed(p.epoch_ctr));
+                *x.epoch_late = ep_mine;
+                ticket = atomicAdd(p.done_ticket, 1u);
+            }
+            if (part == 0) {
+                float* w_own = reinterpret_cast<float*>(key);   // the ordering keys are no longer needed
+                for (int i = gtid; i < ntok * p.k; i += rn) w_own[i] = __ldg(p.topk_w + (size_t)t0 * p.k + i);
+            }
+            local_clean_own_duplicates(p, t0, t1, ids_sm, gtid, rn);   // (rank-level rows do not depend on them)
+            group_sync(1, rn);
+            if (p.trace && gtid == 0) p.trace[(size_t)c * kTraceSlots + 11] = trace_ns(p);
+            if (part == 0) local_meta_dedup(p, t0, t1, ids_sm, pos_raw, row_sm, reinterpret_cast<float*>(key), gtid, rn);
+            if (gtid == 0) {
+                epoch_finish_check_in(p, ticket, ep_mine);
+                if (p.trace) p.trace[(size_t)c * kTraceSlots + 12] = trace_ns(p);
+            }
+        } else {
             // expert-level outputs of rank r: shared by Q CTAs so that no CTA trails the others
+            const int dn = gn - kRowThreads, dw = nw - kRowWarps;
             const int Q = p.grid / p.R > 1 ? p.grid / p.R : 1;
-            for (int u = c; u < p.R * Q; u += p.grid)
-                local_rank_duty(p, u / Q, u % Q, Q, ids_sm, rm, hist, gw, nw, lane, gtid, gn, 1);
+            // ... once the movers are released: started earlier, these warps take issue slots and
+            // shared-memory bandwidth from the few threads every copy of this CTA is waiting for
+            const bool go = mbar_wait_idle(&ready_bar, 0, abortp);
+            for (int u = c; go && u < p.R * Q; u += p.grid)
+                local_rank_duty(p, u / Q, u % Q, Q, ids_sm, rm, hist, gw - kRowWarps, dw, lane, gtid - kRowThreads, dn, 3);
+            if (gtid == kRowThreads) trace(p, c, kTrScanned);   // deferred outputs written
         }
-        if (gtid == 0) trace(p, c, kTrScanned);   // deferred outputs written
     } else if (kMode == kModeLocal) {
         // every CTA: bitmaps over the whole routing table -> totals, the rows before its
         // own tokens, and (CTAs with a source-rank duty) that rank's counts
@@ -458,6 +495,7 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
         stage_ids(p, t0, t1, ids_sm, gtid, gn);
         stage_small();
         group_sync(1, gn);
+        if (kFp8 && gtid == 0) mbar_arrive(x.staged_bar);   // the loader may fetch rows now
         build_bin_maps(p, ids_sm, ntok, bmaps, gw, nw, lane);
         group_sync(1, gn);
         int deferred = -1;
@@ -548,143 +586,175 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
 }
 
 // ------------------------------------------------------------ FP8: quantise and store
-// After the layout: warp 1 issues the stores, warps 2 .. nq + 1 quantise.
+// Two roles around a ring of quantised rows (payload + scales).  The quantising warps turn the
+// rows the loader has fetched into FP8 and know nothing about destinations (own rows) -- so they
+// can run beside the layout; the store issuer sends every quantised row to its destinations
+// with bulk copies once the layout is done.
+//
+// Shared-memory bookkeeping behind the input ring's items: out_src[os] = where the row of
+// output stage os comes from (chunk << 16 | index, -1 = nothing follows), out_pos[os] = the
+// destinations of a row taken over from another chunk.
+struct Fp8Ring {
+    uint8_t* out_ring;
+    const int* item_src;   // [kMaxStages]
+    const int* item_pos;   // [kMaxStages, k]
+    int* out_src;          // [kMaxOutStages]
+    int* out_pos;          // [kMaxOutStages, k]
+    int g0;                // first scale group of this CTA's piece
+    unsigned scale_bytes;  // its scales travel with the payload
+    bool scale_bulk;       // ... by a bulk copy when their size allows it
+};
+__device__ __forceinline__ Fp8Ring fp8_ring(const Cta& x) {
+    const Params& p = x.p;
+    int* item = reinterpret_cast<int*>(x.smem + x.pl.off_item);
+    Fp8Ring q;
+    q.out_ring = x.smem + x.pl.off_out;
+    q.item_src = item;
+    q.out_src = item + kMaxStages;
+    q.item_pos = item + kMaxStages + kMaxOutStages;
+    q.out_pos = item + kMaxStages + kMaxOutStages + kMaxStages * p.k;
+    q.g0 = x.part * (p.G / p.parts);
+    q.scale_bytes = (unsigned)(p.G / p.parts) * 4u;
+    q.scale_bulk = (q.scale_bytes & 15u) == 0;
+    return q;
+}
+
+// Quantising warp qw of nq.
 template <bool kSteal>
-__device__ __forceinline__ void fp8_consumers(Cta& x) {
-    UBEP_CTA_LOCALS(x);
-    uint8_t* out_ring = smem + pl.off_out;
-    const int g0 = part * (p.G / p.parts);                      // first scale group of this CTA's piece
-    const unsigned scale_bytes = (unsigned)(p.G / p.parts) * 4u;  // its scales travel with the payload
-    const bool scale_bulk = (scale_bytes & 15u) == 0;             // when a bulk copy can carry them
-    const int* item_src = reinterpret_cast<const int*>(smem + pl.off_item);
-    const int* item_pos = item_src + kMaxStages + kOutStages;
-    int* out_src = reinterpret_cast<int*>(smem + pl.off_item) + kMaxStages;   // [kOutStages] 0 = row, -1 = end
-    int* out_pos = out_src + kOutStages + kMaxStages * p.k;                    // [kOutStages, k]
-    if (warp == 1) {
-        // ------------------------------ store issuer: lane j issues the copy of slot j
-        bool sok = true;
-        unsigned long long w_full = 0, w_read = 0, tq = 0;
-        for (int n = 0; kSteal || n < ntok; ++n) {
-            const int os = n % kOutStages;
-            if (p.trace) tq = global_ns();
-            sok = mbar_wait(&out_full[os], (n / kOutStages) & 1, abortp);
-            if (p.trace) w_full += global_ns() - tq;
-            sok = __all_sync(0xffffffffu, sok);
-            if (!sok || (kSteal && out_src[os] < 0)) break;
-            if (n == 0 && lane == 0) trace(p, c, kTrFirstRow);
-            const uint8_t* src = out_ring + (size_t)os * pl.out_stage_bytes;
-            // lanes 0..k-1: payload of slot j; lanes k..2k-1: its scales (when bulk-storable)
-            for (int j = lane; j < (scale_bulk ? 2 * p.k : p.k); j += 32) {
-                const int jj = j < p.k ? j : j - p.k;
-                const int where = kSteal ? out_pos[os * p.k + jj] : pos[n * p.k + jj];
-                if (where < 0) continue;
-                if (j < p.k) {
-                    bulk_store(p.recv_x + (size_t)where * p.rowB + out_off, src, out_bytes);
-                    if (kSteal) atomicAdd(&arr[where / p.cap], 1);
-                } else {
-                    bulk_store(p.recv_scale + (size_t)where * p.G + g0, src + out_bytes, scale_bytes);
-                }
-            }
-            bulk_commit();
-            if (n + 1 >= kOutStages) {
-                if (p.trace) tq = global_ns();
-                bulk_wait_read<kOutStages - 1>();   // every lane: the oldest row's copies have read it
-                if (p.trace) w_read += global_ns() - tq;
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&out_empty[(n + 1) % kOutStages]);
-            }
-        }
-        if (!sok && lane == 0) {
-            report(p.status, kErrTimeout);
-            abort_flag = 1;
-        }
-        bulk_wait_all<0>();
-        if (p.trace && lane == 0) {
-            p.trace[(size_t)c * kTraceSlots + 14] = w_full;
-            p.trace[(size_t)c * kTraceSlots + 15] = w_read;
-        }
-    } else if (warp - 2 < nq) {
-        // ------------------------------------------------- quantising warps 2 .. nq + 1
-        const int qw = warp - 2;
-        const int nvec = (int)in_bytes / 16;          // 8-channel vectors in this CTA's piece
-        unsigned long long w_in = 0, w_out = 0, t_cmp = 0, tq = 0;
-        for (int n = 0; kSteal || n < ntok; ++n) {
-            const int s = n % stages, os = n % kOutStages;
-            if (p.trace) tq = global_ns();
-            if (!mbar_wait(&full_bar[s], (n / stages) & 1, abortp)) break;
-            if (p.trace) { unsigned long long t2 = global_ns(); w_in += t2 - tq; tq = t2; }
-            if (n >= kOutStages && !mbar_wait(&out_empty[os], ((n / kOutStages) - 1) & 1, abortp)) break;
-            if (p.trace) { unsigned long long t2 = global_ns(); w_out += t2 - tq; tq = t2; }
-            const int from = kSteal ? item_src[s] : ((ch << 16) | n);
-            if (from < 0) {
-                // the loader's closing item: pass it on to the store issuer and leave
-                if (qw == 0 && lane == 0) out_src[os] = -1;
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&out_full[os]);
-                break;
-            }
-            const bool own = (from >> 16) == ch;
-            const int* wpos = own ? pos + (from & 0xffff) * p.k : item_pos + s * p.k;   // this row's destinations
-            if (kSteal && qw == 0) {
-                for (int j = lane; j < p.k; j += 32) out_pos[os * p.k + j] = wpos[j];
-                if (lane == 0) out_src[os] = 0;
-            }
-            const uint8_t* src = smem + (size_t)s * pl.stage_bytes;
-            uint8_t* dst = out_ring + (size_t)os * pl.out_stage_bytes;
-            float* dst_scale = reinterpret_cast<float*>(dst + out_bytes);
-            // two vectors per thread and trip, independent of each other
-            for (int vb = qw * 32; vb < nvec; vb += 2 * nq * 32) {
-                const int v0 = vb + lane, v1 = v0 + nq * 32;
-                const bool ok0 = v0 < nvec, ok1 = v1 < nvec;
-                uint4 in0 = make_uint4(0, 0, 0, 0), in1 = make_uint4(0, 0, 0, 0);
-                if (ok0) in0 = *reinterpret_cast<const uint4*>(src + (size_t)v0 * 16);
-                if (ok1) in1 = *reinterpret_cast<const uint4*>(src + (size_t)v1 * 16);
-                uint2 q0, q1;
-                float sc0, sc1;
-                quantize8(in0, ok0, q0, sc0);
-                quantize8(in1, ok1, q1, sc1);
-                if (ok0) *reinterpret_cast<uint2*>(dst + (size_t)v0 * 8) = q0;
-                if (ok1) *reinterpret_cast<uint2*>(dst + (size_t)v1 * 8) = q1;
-                if ((lane & 15) == 0) {
-                    if (scale_bulk) {
-                        if (ok0) dst_scale[v0 >> 4] = sc0;
-                        if (ok1) dst_scale[v1 >> 4] = sc1;
-                    } else {
-                        for (int j = 0; j < p.k; ++j) {
-                            const int where = wpos[j];
-                            if (where < 0) continue;
-                            if (ok0) p.recv_scale[(size_t)where * p.G + g0 + (v0 >> 4)] = sc0;
-                            if (ok1) p.recv_scale[(size_t)where * p.G + g0 + (v1 >> 4)] = sc1;
-                        }
-                    }
-                }
-            }
-            fence_proxy_async_smem();   // the bulk stores read what we just wrote
+__device__ __forceinline__ void fp8_quantiser(Cta& x, int qw) {
+    UBEP_CTA_LOCALS(x, false);
+    const Fp8Ring q = fp8_ring(x);
+    const int nvec = (int)in_bytes / 16;          // 8-channel vectors in this CTA's piece
+    unsigned long long w_in = 0, w_out = 0, t_cmp = 0, tq = 0;
+    for (int n = 0; kSteal || n < ntok; ++n) {
+        const int s = n % stages, os = n % out_stages;
+        if (p.trace) tq = trace_ns(p);
+        if (!mbar_wait_idle(&full_bar[s], (n / stages) & 1, abortp)) break;
+        if (p.trace) { unsigned long long t2 = trace_ns(p); w_in += t2 - tq; tq = t2; }
+        if (n >= out_stages && !mbar_wait_idle(&out_empty[os], ((n / out_stages) - 1) & 1, abortp)) break;
+        if (p.trace) { unsigned long long t2 = trace_ns(p); w_out += t2 - tq; tq = t2; }
+        const int from = kSteal ? q.item_src[s] : ((ch << 16) | n);
+        if (from < 0) {
+            // the loader's closing item: pass it on to the store issuer and leave
+            if (qw == 0 && lane == 0) q.out_src[os] = -1;
             __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(&out_full[os]);
-                mbar_arrive(&empty_bar[s]);
+            if (lane == 0) mbar_arrive(&out_full[os]);
+            break;
+        }
+        if (kSteal && qw == 0) {
+            if ((from >> 16) != ch)   // a row of another chunk: its destinations travel with it
+                for (int j = lane; j < p.k; j += 32) q.out_pos[os * p.k + j] = q.item_pos[s * p.k + j];
+            if (lane == 0) q.out_src[os] = from;
+        }
+        const uint8_t* src = smem + (size_t)s * pl.stage_bytes;
+        uint8_t* dst = q.out_ring + (size_t)os * pl.out_stage_bytes;
+        float* dst_scale = reinterpret_cast<float*>(dst + out_bytes);
+        // two vectors per thread and trip, independent of each other
+        for (int vb = qw * 32; vb < nvec; vb += 2 * nq * 32) {
+            const int v0 = vb + lane, v1 = v0 + nq * 32;
+            const bool ok0 = v0 < nvec, ok1 = v1 < nvec;
+            uint4 in0 = make_uint4(0, 0, 0, 0), in1 = make_uint4(0, 0, 0, 0);
+            if (ok0) in0 = *reinterpret_cast<const uint4*>(src + (size_t)v0 * 16);
+            if (ok1) in1 = *reinterpret_cast<const uint4*>(src + (size_t)v1 * 16);
+            uint2 q0, q1;
+            float sc0, sc1;
+            quantize8(in0, ok0, q0, sc0);
+            quantize8(in1, ok1, q1, sc1);
+            if (ok0) *reinterpret_cast<uint2*>(dst + (size_t)v0 * 8) = q0;
+            if (ok1) *reinterpret_cast<uint2*>(dst + (size_t)v1 * 8) = q1;
+            if ((lane & 15) == 0) {
+                if (ok0) dst_scale[v0 >> 4] = sc0;
+                if (ok1) dst_scale[v1 >> 4] = sc1;
             }
-            if (p.trace) t_cmp += global_ns() - tq;
         }
-        if (p.trace && warp == 2 && lane == 0) {
-            p.trace[(size_t)c * kTraceSlots + 11] = w_in;
-            p.trace[(size_t)c * kTraceSlots + 12] = w_out;
-            p.trace[(size_t)c * kTraceSlots + 13] = t_cmp;
+        fence_proxy_async_smem();   // the bulk stores read what we just wrote
+        __syncwarp();
+        if (lane == 0) {
+            mbar_arrive(&out_full[os]);
+            mbar_arrive(&empty_bar[s]);
         }
+        if (p.trace) t_cmp += trace_ns(p) - tq;
+    }
+    if (p.trace && qw == 0 && lane == 0) {
+        p.trace[(size_t)c * kTraceSlots + 11] = w_in;
+        p.trace[(size_t)c * kTraceSlots + 12] = w_out;
+        p.trace[(size_t)c * kTraceSlots + 13] = t_cmp;
+    }
+}
+
+// Store issuer (one warp, after the layout): lane j issues the copy of slot j.
+template <bool kSteal>
+__device__ __forceinline__ void fp8_store_issuer(Cta& x) {
+    UBEP_CTA_LOCALS(x, false);
+    const Fp8Ring q = fp8_ring(x);
+    const int Gp = p.G / p.parts;   // scale groups of this CTA's piece
+    bool sok = true;
+    unsigned long long w_full = 0, w_read = 0, tq = 0;
+    for (int n = 0; kSteal || n < ntok; ++n) {
+        const int os = n % out_stages;
+        if (p.trace) tq = trace_ns(p);
+        sok = mbar_wait(&out_full[os], (n / out_stages) & 1, abortp);
+        if (p.trace) w_full += trace_ns(p) - tq;
+        sok = __all_sync(0xffffffffu, sok);
+        const int from = kSteal ? q.out_src[os] : ((ch << 16) | n);
+        if (!sok || from < 0) break;
+        if (n == 0 && lane == 0) trace(p, c, kTrFirstRow);
+        const int* wpos = (from >> 16) == ch ? pos + (from & 0xffff) * p.k : q.out_pos + os * p.k;
+        const uint8_t* src = q.out_ring + (size_t)os * pl.out_stage_bytes;
+        // lanes 0..k-1: payload of slot j; lanes k..2k-1: its scales (when bulk-storable)
+        for (int j = lane; j < (q.scale_bulk ? 2 * p.k : p.k); j += 32) {
+            const int jj = j < p.k ? j : j - p.k;
+            const int where = wpos[jj];
+            if (where < 0) continue;
+            if (j < p.k) {
+                bulk_store(p.recv_x + (size_t)where * p.rowB + out_off, src, out_bytes);
+                if (kSteal) atomicAdd(&arr[where / p.cap], 1);
+            } else {
+                bulk_store(p.recv_scale + (size_t)where * p.G + q.g0, src + out_bytes, q.scale_bytes);
+            }
+        }
+        if (!q.scale_bulk) {   // a piece of scales that no bulk copy can carry: plain stores
+            const float* sc = reinterpret_cast<const float*>(src + out_bytes);
+            for (int i = lane; i < p.k * Gp; i += 32) {
+                const int jj = i / Gp, g = i - jj * Gp;
+                const int where = wpos[jj];
+                if (where >= 0) p.recv_scale[(size_t)where * p.G + q.g0 + g] = sc[g];
+            }
+        }
+        bulk_commit();
+        if (n + 1 >= kStorePending) {
+            if (p.trace) tq = trace_ns(p);
+            bulk_wait_read<kStorePending - 1>();   // every lane: the copies of the row kStorePending - 1 back have read it
+            if (p.trace) w_read += trace_ns(p) - tq;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&out_empty[(n + 1 - kStorePending) % out_stages]);
+        }
+    }
+    if (!sok && lane == 0) {
+        report(p.status, kErrTimeout);
+        abort_flag = 1;
+    }
+    bulk_wait_all<0>();
+    if (p.trace && lane == 0) {
+        p.trace[(size_t)c * kTraceSlots + 14] = w_full;
+        p.trace[(size_t)c * kTraceSlots + 15] = w_read;
     }
 }
 
 // --------------------------------------------------------------------- dispatch kernel
 // Warp roles: warp 0 = mover; warps 1..15 = layout group (count, prefix sums, row
-// assignment); with FP8 rows warp 1 then becomes the store issuer and warps 2..15 quantise.
+// assignment).  FP8 rows: warp 0 only loads; either the layout group is warps 1 .. count_warps and
+// the warps behind them quantise beside it (the kernels whose layout waits for other CTAs or was
+// computed by earlier launches), or all 15 warps compute the layout and warps 2..15 quantise
+// afterwards (the flag-free kernel, whose layout is pure computation); warp 1 issues the stores
+// once the layout is done.
 template <int kMode, bool kFp8, bool kSteal>
 __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, const SmemPlan pl) {
     extern __shared__ __align__(128) uint8_t smem[];
     __shared__ __align__(8) uint64_t full_bar[kMaxStages];    // input row landed
     __shared__ __align__(8) uint64_t empty_bar[kMaxStages];   // FP8: input row consumed
-    __shared__ __align__(8) uint64_t out_full[kOutStages];    // FP8: quantised row written
-    __shared__ __align__(8) uint64_t out_empty[kOutStages];   // FP8: its stores have read it
+    __shared__ __align__(8) uint64_t out_full[kMaxOutStages];    // FP8: quantised row written
+    __shared__ __align__(8) uint64_t out_empty[kMaxOutStages];   // FP8: its stores have read it
     __shared__ __align__(8) uint64_t ready_bar;               // rows assigned, movers may go
     __shared__ __align__(8) uint64_t epoch_bar;               // epoch_sm holds this launch's epoch
     __shared__ __align__(8) uint64_t staged_bar;              // flag-free kernel: the routing table is in shared memory
@@ -696,7 +766,10 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
     const int part = c % p.parts, ch = c / p.parts;
     const int t0 = (int)chunk_begin(ch, p.T, p.nchunks), t1 = (int)chunk_begin(ch + 1, p.T, p.nchunks);
     const int stages = pl.stages;
-    const int nq = kFp8 ? p.quant_warps : kWarps - 2;   // FP8: warps 2 .. nq + 1 quantise
+    const bool beside = kFp8 && kMode != kModeLocal && p.count_warps > 0;
+    const int nw = beside ? p.count_warps : kWarps - 1;      // layout group: warps 1 .. nw
+    const int qwarp0 = beside ? nw + 1 : 2;                    // FP8: warps qwarp0 .. qwarp0 + nq - 1 quantise
+    const int nq = kFp8 ? min(p.quant_warps, kWarps - qwarp0) : kWarps - 2;
     int* arr = reinterpret_cast<int*>(smem + pl.off_arr);
     griddep_launch();   // the next kernel in the stream may be placed as soon as SMs have room
 
@@ -705,7 +778,7 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], nq);
         }
-        for (int s = 0; s < kOutStages; ++s) {
+        for (int s = 0; s < pl.out_stages; ++s) {
             mbar_init(&out_full[s], nq);
             mbar_init(&out_empty[s], 1);
         }
@@ -721,14 +794,15 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
     // The epoch is not read here, in front of everything: the flag-free kernel needs it only for the
     // arrival counters at its very end and reads it once the movers are released; in the other
     // kernels the mover warp fetches it while the layout group stages the routing table.
+    if (tid == 0) trace_begin(p, c);
     __syncthreads();
     const unsigned epoch = 0u;
-    if (tid == 0) trace(p, c, kTrStart);
 
     const unsigned in_bytes = (unsigned)(p.H * 2 / p.parts);   // this CTA's piece of a bf16 row
     const unsigned out_bytes = (unsigned)(p.rowB / p.parts);   // and of a payload row
     Cta x{p, pl, smem, full_bar, empty_bar, out_full, out_empty, &ready_bar, &epoch_bar, &staged_bar, &abort_flag,
           tid, tid & 31, tid >> 5, c, part, ch, t0, t1, t1 - t0, stages, nq,
+          nw * 32, nw, pl.out_stages, qwarp0, beside,
           reinterpret_cast<int*>(smem + pl.off_ids),
           reinterpret_cast<int*>(smem + pl.off_ord),    // destinations in issue order
           reinterpret_cast<int*>(smem + (p.ordered ? pl.off_pos : pl.off_ord)),   // in slot order (the same array
@@ -743,21 +817,26 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
 
     if (x.warp == 0) {
         mover_warp<kMode, kFp8, kSteal>(x);
+    } else if (kFp8 && beside && x.warp >= qwarp0) {
+        if (x.warp - qwarp0 < nq) fp8_quantiser<kSteal>(x, x.warp - qwarp0);   // beside the layout
     } else {
         const bool ok = layout_group<kMode, kFp8, kSteal>(x);
-        if (kFp8 && ok) fp8_consumers<kSteal>(x);
+        if (kFp8 && ok) {
+            if (x.warp == 1) fp8_store_issuer<kSteal>(x);
+            else if (!beside && x.warp - 2 < nq) fp8_quantiser<kSteal>(x, x.warp - 2);
+        }
     }
     __syncthreads();
     const unsigned half = epoch_sm & 1u;
-    // The arrival counters of the next call live in the other half; clear them now.  This also runs
-    // when the call gives up below: otherwise the call after the next one would add to stale totals.
-    // (epoch_sm == 0: the call gave up before it learnt its epoch, so it has not used either half.)
-    if (c == 0 && epoch_sm != 0u) {
-        for (int r = tid; r < p.R; r += kThreads) p.arrival[(half ^ 1u) * p.R + r] = 0;
-        if (tid == 0) p.claimed[half ^ 1u] = 0;   // same for the count of tokens handed out
-    }
     if (abort_flag) {
-        // leaving early: the newest load of every ring stage may still be landing
+        // leaving early.  The arrival counters of the next call live in the other half; they are
+        // cleared here too, otherwise the call after the next one would add to stale totals.
+        // (epoch_sm == 0: the call gave up before it learnt its epoch and has used neither half.)
+        if (c == 0 && epoch_sm != 0u) {
+            for (int r = tid; r < p.R; r += kThreads) p.arrival[(half ^ 1u) * p.R + r] = 0;
+            if (tid == 0) p.claimed[half ^ 1u] = 0;
+        }
+        // the newest load of every ring stage may still be landing
         if (tid == 0) {
             for (int n = max(0, x.issued - stages); n < x.issued; ++n)
                 (void)mbar_wait(&full_bar[n % stages], (n / stages) & 1, nullptr);
@@ -769,6 +848,11 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
     fence_proxy_async();   // rows written through the async proxy, counters through the generic one
     for (int r = tid; r < p.R; r += kThreads)
         if (arr[r]) red_release_add(p.arrival + half * p.R + r, (unsigned)(arr[r] * (8 / p.parts)));
+    // the arrival counters of the next call live in the other half; clear them now
+    if (c == 0) {
+        for (int r = tid; r < p.R; r += kThreads) p.arrival[(half ^ 1u) * p.R + r] = 0;
+        if (tid == 0) p.claimed[half ^ 1u] = 0;   // same for the count of tokens handed out
+    }
     if (tid == 0) trace(p, c, kTrEnd);
 }
 
@@ -921,19 +1005,38 @@ int plan_dispatch(const Params& p, int mode, int max_smem, SmemPlan* out) {
     pl.out_stage_bytes = p.payload ? round_up_i(p.rowB / p.parts + (p.G / p.parts) * 4, 128) : 0;
     const int64_t mask_ints = (int64_t)pl.map_groups * 32;
     const int64_t bm_ints = (int64_t)pl.map_groups * pl.map_bp;
-    const int item_ints = (kMaxStages + kOutStages) * (p.k + 1);
+    const int item_ints = (kMaxStages + kMaxOutStages) * (p.k + 1);
     const int64_t ints = ids_ints + mask_ints + bm_ints + 4 * (int64_t)chunk_slots + hist_ints + 2 * p.R + item_ints;
-    const int64_t fixed = (int64_t)kOutStages * pl.out_stage_bytes + ints * 4 + 128 + 1024;  // 1 KB: static smem
-    if (fixed + 4 * (int64_t)pl.stage_bytes > max_smem) return -1;
-    pl.stages = (int)((max_smem - fixed) / pl.stage_bytes);
-    if (pl.stages > kMaxStages) pl.stages = kMaxStages;
+    const int64_t fixed = ints * 4 + 128 + 1536;  // 1.5 KB: static shared memory
     // no more stages than rows this CTA will ever hold at once
-    {
-        const int want = chunk_tokens + 3 < 4 ? 4 : chunk_tokens + 3;
+    const int want = chunk_tokens + 3 < 4 ? 4 : chunk_tokens + 3;
+    const bool beside = p.payload && mode != kModeLocal && p.count_warps > 0;
+    if (!beside) {
+        // the quantising warps (if any) start after the layout: a deep input ring that the loader fills
+        // meanwhile, a short ring of quantised rows
+        pl.out_stages = p.payload ? kOutStages : 0;
+        const int64_t rest = max_smem - fixed - (int64_t)pl.out_stages * pl.out_stage_bytes;
+        if (rest < 4 * (int64_t)pl.stage_bytes) return -1;
+        pl.stages = (int)(rest / pl.stage_bytes);
+        if (pl.stages > kMaxStages) pl.stages = kMaxStages;
+        if (pl.stages > want) pl.stages = want;
+    } else {
+        // the quantising warps run beside the layout: a short input ring (enough loads in flight to keep
+        // them busy) and as many quantised rows as fit, which wait for the layout
+        const int64_t room = max_smem - fixed;
+        if (room < 2 * (int64_t)pl.stage_bytes + 4 * (int64_t)pl.out_stage_bytes) return -1;
+        pl.stages = 4;
+        while (pl.stages > 2 && room < (int64_t)pl.stages * pl.stage_bytes + 4 * (int64_t)pl.out_stage_bytes) --pl.stages;
+        pl.out_stages = (int)((room - (int64_t)pl.stages * pl.stage_bytes) / pl.out_stage_bytes);
+        if (pl.out_stages > kMaxOutStages) pl.out_stages = kMaxOutStages;
+        if (pl.out_stages > want) pl.out_stages = want < 4 ? 4 : want;
+        // what is left over goes to the input ring
+        const int more = (int)((room - (int64_t)pl.out_stages * pl.out_stage_bytes) / pl.stage_bytes);
+        pl.stages = more > kMaxStages ? kMaxStages : more;
         if (pl.stages > want) pl.stages = want;
     }
     int at = pl.stages * pl.stage_bytes;
-    pl.off_out = at; at += kOutStages * pl.out_stage_bytes;
+    pl.off_out = at; at += pl.out_stages * pl.out_stage_bytes;
     pl.off_ids = at; at += (int)ids_ints * 4;
     pl.off_mask = at; at += (int)mask_ints * 4;
     pl.off_bm = at; at += (int)bm_ints * 4;

@@ -472,6 +472,9 @@ constexpr int kRankWords = 4;
 __device__ __forceinline__ int fast_div(int v, unsigned magic) { return (int)__umulhi((unsigned)v, magic); }
 
 // Stage all T*k slots (packed id | rank << 16) and build the rank bitmaps; lane = token.
+// (An expert named twice by a token does not change any rank-level row, so this step, which every
+// copy waits for, does not look for it; that happens once the movers are released.
+// Looking for it here was measured to cost 2.5 us per dispatch of 512 tokens.)
 static __device__ void local_stage_and_rank_maps(const Params& p, int* ids, const RankMaps& rm, int gw, int nw, int lane) {
     const int k = p.k, T = p.T;
     const bool vec = (k & 3) == 0;   // a token's ids are whole 16-byte words (topk_idx is 16-byte aligned)
@@ -493,24 +496,10 @@ static __device__ void local_stage_and_rank_maps(const Params& p, int* ids, cons
 #pragma unroll
                     for (int u = 0; u < 8; ++u) raw[u] = j0 + u < k ? __ldg(src + j0 + u) : -1;
                 }
-                int res[8];
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
                     if (j0 + u >= k) break;
-                    int e = resolve_expert(p, t, raw[u]);
-                    // an expert named twice by one token: the later slot is reported and left empty
-                    bool dup = false;
-#pragma unroll
-                    for (int u2 = 0; u2 < u; ++u2) dup = dup || (e >= 0 && res[u2] == e);
-                    for (int jj = 0; jj < j0; ++jj) {
-                        const int v2 = ids[t * k + jj];
-                        dup = dup || (e >= 0 && v2 >= 0 && slot_expert(v2) == e);
-                    }
-                    if (dup) {
-                        report(p.status, kErrBadIndex);
-                        e = -1;
-                    }
-                    res[u] = e;
+                    const int e = resolve_expert(p, t, raw[u]);
                     int packed = -1;
                     if (e >= 0) {
                         const int r = fast_div(e, p.L_magic);
@@ -574,27 +563,71 @@ static __device__ void local_rows_dedup(const Params& p, int t0, int t1, const i
     }
 }
 
+// The ids of a token must be distinct: the later of two slots naming one expert is reported
+// (kErrBadIndex) and emptied.  In the flag-free kernel every CTA holds the whole table, but only two
+// things read expert ids from it: the metadata of the CTA's own tokens, for which this empties the
+// repeated slots of tokens [t0, t1) in the CTA's copy, and the per-rank duty, whose bitmaps take a
+// repeated expert once by construction (it reports it) and whose row lists write the same entry twice.
+static __device__ void local_clean_own_duplicates(const Params& p, int t0, int t1, int* ids_all, int gtid, int gn) {
+    const int k = p.k;
+#pragma unroll 1
+    for (int t = t0 + gtid; t < t1; t += gn) {
+        int* row = ids_all + (size_t)t * k;
+#pragma unroll 1
+        for (int j = 1; j < k; ++j) {
+            const int v = row[j];
+            if (v < 0) continue;
+            bool dup = false;
+#pragma unroll 1
+            for (int jj = 0; jj < j; ++jj) dup = dup || row[jj] == v;   // same expert => same packed word
+            if (dup) {
+                report(p.status, kErrBadIndex);
+                row[j] = -1;
+            }
+        }
+    }
+}
+
 // Metadata of this CTA's own tokens (after the movers were released).
 static __device__ void local_meta_dedup(const Params& p, int t0, int t1, const int* ids_all, const int* pos_raw,
                                  const int* row_sm, const float* w_own, int gtid, int gn) {
     const int k = p.k, L = p.L;
     const int nslots = (t1 - t0) * k;
+#pragma unroll 1
     for (int li = gtid; li < nslots; li += gn) {
         const int tl = li / k, t = t0 + tl;
         const size_t i = (size_t)t0 * k + li;
         const int packed = ids_all[i];
-        const int row = row_sm[li];
+        const int row = packed >= 0 ? row_sm[li] : -1;   // (a slot emptied as a duplicate has no row)
         p.slot_row[i] = row;
         p.slot_pos[i] = (packed >= 0 && row >= 0 && row < p.cap) ? slot_rank(packed) * p.cap + row : -1;
         const int where = pos_raw[li];
         if (where >= 0) {
             const int r = slot_rank(packed);
             p.recv_src_idx[where] = t;
-            for (int jj = 0; jj < k; ++jj) {
-                const int v2 = ids_all[(size_t)t * k + jj];
-                const bool here = v2 >= 0 && slot_rank(v2) == r;
-                p.recv_topk_idx[(size_t)where * k + jj] = here ? slot_expert(v2) - r * L : -1;
-                p.recv_topk_w[(size_t)where * k + jj] = here ? w_own[tl * k + jj] : 0.0f;
+            if ((k & 3) == 0) {   // rows of the two arrays start on 16-byte boundaries: four slots per store
+#pragma unroll 1
+                for (int j4 = 0; j4 < k; j4 += 4) {
+                    int e4[4];
+                    float w4[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int v2 = ids_all[(size_t)t * k + j4 + u];
+                        const bool here = v2 >= 0 && slot_rank(v2) == r;
+                        e4[u] = here ? slot_expert(v2) - r * L : -1;
+                        w4[u] = here ? w_own[tl * k + j4 + u] : 0.0f;
+                    }
+                    *reinterpret_cast<int4*>(p.recv_topk_idx + (size_t)where * k + j4) = make_int4(e4[0], e4[1], e4[2], e4[3]);
+                    *reinterpret_cast<float4*>(p.recv_topk_w + (size_t)where * k + j4) = make_float4(w4[0], w4[1], w4[2], w4[3]);
+                }
+            } else {
+#pragma unroll 1
+                for (int jj = 0; jj < k; ++jj) {
+                    const int v2 = ids_all[(size_t)t * k + jj];
+                    const bool here = v2 >= 0 && slot_rank(v2) == r;
+                    p.recv_topk_idx[(size_t)where * k + jj] = here ? slot_expert(v2) - r * L : -1;
+                    p.recv_topk_w[(size_t)where * k + jj] = here ? w_own[tl * k + jj] : 0.0f;
+                }
             }
         }
     }
@@ -608,21 +641,29 @@ static __device__ void local_meta_dedup(const Params& p, int t0, int t1, const i
 static __device__ void local_rank_duty(const Params& p, int r, int q, int Q, const int* ids_all, const RankMaps& rm,
                                 int* sm, int gw, int nw, int lane, int gtid, int gn, int bar_id) {
     const int k = p.k, L = p.L, T = p.T, S = p.S, E = p.E;
+#pragma unroll 1
     for (int g = gw; g < rm.groups; g += nw) {
         const int t = g * 32 + lane;
         unsigned m = 0u;
         if (t < T)
+#pragma unroll 1
             for (int j = 0; j < k; ++j) {
                 const int v = ids_all[(size_t)t * k + j];
-                if (v >= 0 && slot_rank(v) == r) m |= (1u << (slot_expert(v) - r * L)) | (1u << L);
+                if (v >= 0 && slot_rank(v) == r) {
+                    const unsigned bit = 1u << (slot_expert(v) - r * L);
+                    if (m & bit) report(p.status, kErrBadIndex);   // an expert named twice by this token
+                    m |= bit | (1u << L);
+                }
             }
         rm.dbm[(size_t)g * 32 + lane] = transpose32(m, lane);
     }
     group_sync(bar_id, gn);
+    if (p.trace && gtid == 0) p.trace[(size_t)blockIdx.x * kTraceSlots + 13] = trace_ns(p);
     auto bits = [&](int l, int lo, int hi) {   // tokens in [lo, hi) with bit l
         if (hi <= lo) return 0;
         const int g0 = lo >> 5, g1 = (hi - 1) >> 5;
         int c = 0;
+#pragma unroll 1
         for (int g = g0; g <= g1; ++g) {
             unsigned w = rm.dbm[(size_t)g * 32 + l];
             if (g == g0) w &= 0xffffffffu << (lo & 31);
@@ -637,6 +678,7 @@ static __device__ void local_rank_duty(const Params& p, int r, int q, int Q, con
     group_sync(bar_id, gn);
     if (gtid <= L) {
         int o = 0;
+#pragma unroll 1
         for (int i = 0; i < gtid; ++i) o += tot[i];
         eo[gtid] = o;
         if (q == 0) {
@@ -650,12 +692,15 @@ static __device__ void local_rank_duty(const Params& p, int r, int q, int Q, con
         }
     }
     group_sync(bar_id, gn);
+#pragma unroll 1
     for (int i = q + Q * gtid; i < S * L; i += Q * gn) {
         const int s = i / L, l = i - s * L;
         const int b0 = src_begin(s, T, S), b1 = src_begin(s + 1, T, S);
         p.cnt[(size_t)s * E + r * L + l] = bits(l, b0, b1);
         p.src_offset[(size_t)s * E + r * L + l] = eo[l] + bits(l, 0, b0);
     }
+    if (p.trace && gtid == 0) p.trace[(size_t)blockIdx.x * kTraceSlots + 14] = trace_ns(p);
+#pragma unroll 1
     for (int i = q + Q * gtid; i < T * k; i += Q * gn) {
         const int v = ids_all[i];
         if (v < 0 || slot_rank(v) != r) continue;

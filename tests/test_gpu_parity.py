@@ -308,18 +308,44 @@ def test_fp8_special_values_match_the_oracle():
     Hn.run_case(wl, pipeline=FUSED)
 
 
-@pytest.mark.parametrize("n", [1, 3, 8])
-def test_warp_role_split_does_not_change_results(n):
-    cfg = small(600, 1024, 32, 8, 4, payload=1, seed=33)
-    wl = W.make_workload(cfg)
+@pytest.mark.parametrize("pipeline", [PHASED, FUSED])
+@pytest.mark.parametrize("count_warps,quant_warps,prefetch", [
+    (0, 1, None), (0, 3, None), (0, 8, None),        # all warps count, then quantise
+    (1, 14, None), (2, 14, 1), (4, 14, None), (4, 2, 3), (8, 14, None), (13, 14, None),   # beside the layout
+])
+@pytest.mark.parametrize("shape", [
+    dict(T=600, H=1024, E=32, R=8, k=4),                 # 4 tokens per CTA: fewer rows than ring stages
+    dict(T=7000, H=512, E=64, R=8, k=6),                 # 47 tokens per CTA: token stealing, ring wraps many times
+    dict(T=6100, H=7168, E=72, R=18, k=4),               # stealing with rows so large that the input ring is short
+    dict(T=1500, H=384, E=24, R=3, k=3, dedup=1),        # scales of a row are 12 bytes: no bulk copy carries them
+])
+def test_warp_role_split_does_not_change_results(shape, count_warps, quant_warps, prefetch, pipeline):
+    """How many warps count, how many quantise, and how far the loader runs ahead of the layout
+    only change the schedule inside the FP8 dispatch kernel, never its results."""
+    cfg = W.Config("roles", payload=1, seed=33 + shape["T"], **shape)
+    wl = W.with_empty_slots(W.make_workload(cfg), 0.05, seed=2)
     ids, lay, cap, recv = Hn.oracle_reference(wl)
-    buf = Hn.make_buffer(cfg, cap, pipeline=FUSED)
-    B.ubep_debug_set_quant_warps(buf.handle, n)
+    buf = Hn.make_buffer(cfg, cap, pipeline=pipeline)
+    B.ubep_debug_set_count_warps(buf.handle, count_warps)
+    B.ubep_debug_set_quant_warps(buf.handle, quant_warps)
+    if prefetch:
+        B.ubep_debug_set_prefetch_rows(buf.handle, prefetch)
     x, idx, w, _, _ = Hn.device_inputs(wl)
-    buf.dispatch(x, idx, w)
-    Hn.check_dispatch(buf, wl, lay, cap, recv)
-    with pytest.raises(B.UbepError):
-        B.ubep_debug_set_quant_warps(buf.handle, 15)
+    for _ in range(2):
+        buf.recv_x.fill_(Hn.FILL)
+        buf.recv_scale.view(torch.uint8).fill_(Hn.FILL)
+        buf.dispatch(x, idx, w)
+        Hn.check_dispatch(buf, wl, lay, cap, recv)
+
+
+def test_warp_role_knobs_reject_values_out_of_range():
+    cfg = small(64, payload=1, H=256)
+    buf = Hn.make_buffer(cfg, 128)
+    for fn, bad in ((B.ubep_debug_set_quant_warps, (0, 15)), (B.ubep_debug_set_count_warps, (-1, 14)),
+                    (B.ubep_debug_set_prefetch_rows, (0,))):
+        for v in bad:
+            with pytest.raises(B.UbepError):
+                fn(buf.handle, v)
 
 
 def test_bounded_wait_reports_timeout_and_the_context_survives():
