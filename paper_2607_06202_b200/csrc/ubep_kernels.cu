@@ -217,9 +217,10 @@ __device__ __forceinline__ void mover_warp(Cta& x) {
         int tl = 0;
         // Flag-free kernel: the routing table first, the rows after it.  The table is the one load the
         // whole layout waits for; the rows of 148 CTAs queued in front of it cost about a microsecond.
+        const RankMaps rm{bmaps.bm, bmaps.mask_t, (p.R + 31) / 32, ((p.R + 31) / 32) * 32, (p.T + 31) / 32};
         if (fast_local) {
-            // lend a hand with the routing table
-            const RankMaps rm{bmaps.bm, bmaps.mask_t, (p.R + 31) / 32, ((p.R + 31) / 32) * 32, (p.T + 31) / 32};
+            // lend a hand with the routing table.  (Rows asked for before every warp's share of the table
+            // is in -- even as late as when this warp's own share has arrived -- delay it: measured 0.9 us.)
             local_stage_and_rank_maps(p, ids_sm, rm, 0, kWarps, lane);
             group_sync(2, kThreads);
         } else if (kMode == kModeLocal) {
@@ -379,10 +380,10 @@ __device__ __forceinline__ void mover_warp(Cta& x) {
 
 // ---------------------------------------------------------------------- layout group
 // Warps 1..15: TokenCnt, CalCumSum (by exchange or alone), slot -> row assignment; releases
-// the movers and then writes what nobody inside the kernel waits for.  Returns false if a
-// wait ran out.
+// the movers and then writes what nobody inside the kernel waits for.  Returns 1, 0 if a wait ran
+// out, or 2 for a warp that has done its share of the counting and now leaves to quantise.
 template <int kMode, bool kFp8, bool kSteal>
-__device__ __forceinline__ bool layout_group(Cta& x) {
+__device__ __forceinline__ int layout_group(Cta& x) {
     UBEP_CTA_LOCALS(x, !kFp8);
     bool ok = true;
     const int* ids = ids_sm;  // staged slots of this CTA's tokens
@@ -391,12 +392,12 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
     const int order_r = gtid < p.R ? __ldg(p.order_pos + gtid) : 0;
     const bool stage_w = !(kMode == kModeLocal && p.local_fast);
     const float w_first = (stage_w && gtid < ntok * p.k) ? __ldg(p.topk_w + (size_t)t0 * p.k + gtid) : 0.0f;
-    auto stage_small = [&]() {
+    auto stage_small = [&](int n) {   // by n threads
         if (gtid < p.R) order_sm[gtid] = order_r;
-        for (int r = gtid + gn; r < p.R; r += gn) order_sm[r] = __ldg(p.order_pos + r);
+        for (int r = gtid + n; r < p.R; r += n) order_sm[r] = __ldg(p.order_pos + r);
         if (stage_w) {
             if (gtid < ntok * p.k) w_sm[gtid] = w_first;
-            for (int i = gtid + gn; i < ntok * p.k; i += gn) w_sm[i] = __ldg(p.topk_w + (size_t)t0 * p.k + i);
+            for (int i = gtid + n; i < ntok * p.k; i += n) w_sm[i] = __ldg(p.topk_w + (size_t)t0 * p.k + i);
         }
     };
     if (kMode == kModeLocal && p.local_fast) {
@@ -404,7 +405,7 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
         const RankMaps rm{bmaps.bm, bmaps.mask_t, (p.R + 31) / 32, ((p.R + 31) / 32) * 32, (p.T + 31) / 32};
         int* row_sm = reinterpret_cast<int*>(w_sm);
         local_stage_and_rank_maps(p, ids_sm, rm, warp, kWarps, lane);   // with the mover warp
-        stage_small();
+        stage_small(gn);
         group_sync(2, kThreads);
         if (gtid == 0) trace(p, c, kTrCounted);
         // From here the group splits.  Assigning rows to the CTA's own few tokens keeps a handful of
@@ -463,7 +464,7 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
         int* pre = hist + p.B;
         int* eo = hist + 2 * p.B;
         stage_ids(p, 0, p.T, ids_sm, gtid, gn);
-        stage_small();
+        stage_small(gn);
         group_sync(1, gn);
         if (gtid == 0) {
             mbar_arrive(x.staged_bar);   // the mover may fetch rows now
@@ -492,23 +493,34 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
         if (part == 0)
             for (int s = ch; s < p.S; s += p.nchunks) write_source_from_maps(p, s, bmaps, eo, gtid, gn);   // source ranks this CTA reports
     } else {
-        stage_ids(p, t0, t1, ids_sm, gtid, gn);
-        stage_small();
-        group_sync(1, gn);
+        // FP8 rows with a count group: TokenCnt itself -- staging the ids, the bitmaps, publishing the
+        // chunk's counts -- is pure computation and is done by all 15 warps; then the warps behind the
+        // count group leave to quantise, and the count group alone goes through the steps that mostly
+        // wait for other CTAs (flag exchange, CalCumSum duty) and assigns the rows.
+        const bool split = kFp8 && x.beside;
+        const int an = split ? kThreads - 32 : gn, aw = split ? kWarps - 1 : nw;
+        const int bid = split ? 4 : 1;   // barrier of the count group once the others have left
+        stage_ids(p, t0, t1, ids_sm, gtid, an);
+        stage_small(an);
+        group_sync(1, an);
         if (kFp8 && gtid == 0) mbar_arrive(x.staged_bar);   // the loader may fetch rows now
-        build_bin_maps(p, ids_sm, ntok, bmaps, gw, nw, lane);
-        group_sync(1, gn);
+        build_bin_maps(p, ids_sm, ntok, bmaps, gw, aw, lane);
+        group_sync(1, an);
+        if (kMode == kModeFused) publish_chunk_counts(p, ch, t0, t1, bmaps, gtid, an);
+        if (split) {
+            group_sync(1, an);          // the counts are stored (the flag is released further down)
+            if (gw >= nw) return 2;     // off to quantise
+        }
         int deferred = -1;
         // The mover warp fetched the epoch while the table was staged; one thread makes sure it has
         // arrived, the barrier that follows hands it to the others.
         unsigned ep = 0;
         auto learn_epoch = [&]() {
             if (gtid == 0) (void)mbar_wait(x.epoch_bar, 0, abortp);
-            group_sync(1, gn);
+            group_sync(bid, gn);
             ep = *reinterpret_cast<volatile unsigned*>(x.epoch_late);
         };
         if (kMode == kModeFused) {
-            publish_chunk_counts(p, ch, t0, t1, bmaps, gtid, gn);
             learn_epoch();
             if (gtid == 0) {
                 if (ch != p.withhold) {
@@ -521,16 +533,16 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
             for (int r = ch; r < p.R; r += p.nchunks) {
                 for (int cc = gtid; cc < p.nchunks; cc += gn)
                     if (!wait_flag(p.hist_flag + cc, ep, abortp)) lost = true;
-                if (group_or(1, gn, lost || *abortp)) { lost = true; break; }  // same answer for all
+                if (group_or(bid, gn, lost || *abortp)) { lost = true; break; }  // same answer for all
                 if (gtid == 0) trace(p, c, kTrHistSeen);
-                scan_rank_publish(p, r, hist, gw, nw, lane, 1);
+                scan_rank_publish(p, r, hist, gw, nw, lane, bid);
                 if (gtid == 0) {
                     st_release(p.scan_flag + r, ep);
                     trace(p, c, kTrScanned);
                 }
                 if (r + p.nchunks < p.R) {
                     scan_rank_sources(p, r, hist, gtid, gn);
-                    group_sync(1, gn);
+                    group_sync(bid, gn);
                 } else {
                     deferred = r;   // cnt / src_offset: after our own movers are released
                 }
@@ -539,7 +551,7 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
             if (!lost)
                 for (int r = gtid; r < p.R; r += gn)
                     if (!wait_flag(p.scan_flag + r, ep, abortp)) lost = true;
-            ok = !group_or(1, gn, lost || *abortp);
+            ok = !group_or(bid, gn, lost || *abortp);
             if (gtid == 0) trace(p, c, kTrScanSeen);
             if (!ok && gtid == 0) {
                 report(p.status, kErrTimeout);
@@ -555,16 +567,16 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
             int* base_sm = hist + p.B;   // second half of the scratch (the first may hold scan totals)
             for (int b = gtid; b < p.B; b += gn)
                 base_sm[b] = __ldcg(cb + (size_t)b * p.nchunks) + (b < p.E ? __ldcg(p.expert_offset + b) : 0);
-            group_sync(1, gn);
+            group_sync(bid, gn);
             finalize_chunk(p, t0, t1, ids, w_sm,
                            [&](int e, int tl) { return base_sm[e] + bits_in_range(bmaps, e, 0, tl); },
                            [&](int r, int tl) { return base_sm[p.E + r] + bits_in_range(bmaps, p.E + r, 0, tl); },
                            true, c, order_sm, pos_raw, key, kSteal ? nullptr : arr, gtid, gn);
-            group_sync(1, gn);
+            group_sync(bid, gn);
             if (gtid == 0) trace(p, c, kTrFinalized);
             if (p.ordered) {   // a destination table is set: the copies of a token in its order (else pos_raw is pos)
                 order_destinations(p, pos_raw, key, pos, ntok * p.k, gtid, gn);
-                group_sync(1, gn);
+                group_sync(bid, gn);
             }
         }
         if (gtid == 0) {
@@ -574,7 +586,7 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
         if (ok && kSteal) {
             // this chunk's destinations, for CTAs that run out of work and take over some of its tokens
             for (int i = gtid; i < ntok * p.k; i += gn) p.copy_pos[(size_t)t0 * p.k + i] = pos[i];
-            if (kMode == kModeFused) group_sync(1, gn);
+            if (kMode == kModeFused) group_sync(bid, gn);
             else learn_epoch();   // (with kernel boundaries instead of flags nothing has asked for it yet)
             if (gtid == 0) {
                 st_release(p.pos_flag + ch, ep);
@@ -582,7 +594,7 @@ __device__ __forceinline__ bool layout_group(Cta& x) {
         }
         if (ok && deferred >= 0) scan_rank_sources(p, deferred, hist, gtid, gn);
     }
-    return ok;
+    return ok ? 1 : 0;
 }
 
 // ------------------------------------------------------------ FP8: quantise and store
@@ -790,6 +802,15 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
         mbar_fence_init();
     }
     for (int r = tid; r < p.R; r += kThreads) arr[r] = 0;
+    if (kMode == kModeLocal) {
+        // The routing table is the first thing every CTA of the flag-free kernel needs, and it comes cold
+        // from HBM.  A prefetch into L2 reads no value, so it may run ahead of the wait below: L2 is where
+        // an earlier kernel's stores to the table land too, so the line cannot go stale.
+        const char* tab = reinterpret_cast<const char*>(p.topk_idx);
+        const size_t bytes = (size_t)p.T * p.k * 4;
+        for (size_t off = ((size_t)c * kThreads + tid) * 128; off < bytes; off += (size_t)p.grid * kThreads * 128)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(tab + off));
+    }
     griddep_wait();     // shared-memory set-up done; everything below reads what earlier kernels wrote
     // The epoch is not read here, in front of everything: the flag-free kernel needs it only for the
     // arrival counters at its very end and reads it once the movers are released; in the other
@@ -817,11 +838,11 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
 
     if (x.warp == 0) {
         mover_warp<kMode, kFp8, kSteal>(x);
-    } else if (kFp8 && beside && x.warp >= qwarp0) {
-        if (x.warp - qwarp0 < nq) fp8_quantiser<kSteal>(x, x.warp - qwarp0);   // beside the layout
     } else {
-        const bool ok = layout_group<kMode, kFp8, kSteal>(x);
-        if (kFp8 && ok) {
+        const int lg = layout_group<kMode, kFp8, kSteal>(x);   // 0 = a wait ran out, 1 = done, 2 = left to quantise
+        if (kFp8 && lg == 2) {
+            if (x.warp - qwarp0 < nq) fp8_quantiser<kSteal>(x, x.warp - qwarp0);   // beside the rest of the layout
+        } else if (kFp8 && lg == 1) {
             if (x.warp == 1) fp8_store_issuer<kSteal>(x);
             else if (!beside && x.warp - 2 < nq) fp8_quantiser<kSteal>(x, x.warp - 2);
         }
