@@ -683,6 +683,107 @@ def run_ours(args, cfg, rank: int, world: int, local_rank: int):
     print(json.dumps(line), flush=True)
 
 
+# ------------------------------------------------------------- ranks on different GPUs
+
+def sharded_config(world: int):
+    """Decode-like shape with one rank per GPU: 512 tokens, top-8 of 256 experts on `world` ranks."""
+    from paper_2607_06202_b200 import workload as W
+    return W.Config(f"sharded{world}", T=512, H=7168, E=256, R=world, k=8, dedup=1, seed=1102)
+
+
+def remote_bytes(cfg, slot_row, ids, rank: int) -> int:
+    """Payload bytes rank `rank` stores into other GPUs' regions in one dispatch (one row per (token, rank))."""
+    from paper_2607_06202_b200 import sharded
+    b0, b1 = sharded.token_range(rank, cfg.T, cfg.R)
+    rows = 0
+    for t in range(b0, b1):
+        ranks = {int(e) // cfg.L for e in ids[t] if e >= 0}
+        rows += len(ranks - {rank})
+    _ = slot_row
+    return rows * cfg.H * 2
+
+
+def run_sharded(args, rank: int, world: int, local_rank: int):
+    """The path with the ranks on different GPUs (rank = GPU, rows stored straight into the peers'
+    regions over NVLink): ShardedEP dispatch -> arrival wait -> combine over identity experts, rank 0's
+    region and output compared with the CPU oracle, microseconds per call by CUDA events (max over
+    ranks).  Prints one JSON line with a `sharded` block; any failure becomes its `status`."""
+    import torch
+    import torch.distributed as dist
+    block = {"nranks": world, "status": "not run", "parity": None}
+    try:
+        from paper_2607_06202_b200 import binding as B
+        from paper_2607_06202_b200 import sharded
+        from paper_2607_06202_b200 import workload as W
+        dev = torch.device("cuda", local_rank)
+        cfg = sharded_config(world)
+        wl = W.make_workload(cfg)
+        b0, b1 = sharded.token_range(rank, cfg.T, world)
+        x = torch.from_numpy(wl.x[b0:b1].copy()).view(torch.bfloat16).to(dev)
+        idx = torch.from_numpy(wl.topk_idx[b0:b1].astype(np.int32)).to(dev)
+        w = torch.from_numpy(wl.topk_w[b0:b1].copy()).to(dev)
+        # capacity: every token could visit every rank
+        cap = W.round_up(cfg.T, 128)
+        ep = sharded.ShardedEP(num_experts=cfg.E, hidden=cfg.H, topk=cfg.k, max_tokens=cfg.T, rows_per_rank_cap=cap,
+                               dedup=cfg.dedup, device=dev)
+        parity = None
+
+        def layer():
+            region, n = ep.dispatch(x, idx, w, cfg.T)
+            ep.y[rank].copy_(region)              # identity experts: y = the rows received
+            return ep.combine()
+        out = layer()
+        torch.cuda.synchronize(dev)
+        if rank == 0:
+            import oracle
+            import harness as Hn
+            ids = wl.topk_idx
+            lay = oracle.layout(ids, cfg.E, cfg.R, cfg.S, cfg.dedup, er_cap=cap * min(cfg.k, cfg.L))
+            recv = oracle.dispatch(wl.x, ids, wl.topk_w, lay.slot_row, cfg.E, cfg.R, cap, cfg.payload, cfg.dedup,
+                                   fill=0)
+            n0 = int(lay.num_rows_per_rank[0])
+            got = ep.region[:n0].view(torch.int16).cpu()
+            parity = bool(torch.equal(got, torch.from_numpy(recv.recv_x[0, :n0].view(np.int16))))
+            # identity experts: y of every rank is its region, which the oracle has in full
+            y_bits = recv.recv_x.view(np.uint16).reshape(cfg.R, cap, cfg.H)
+            want, _ = oracle.combine(y_bits, ids, wl.topk_w, lay.slot_row, cfg.E, cfg.R)
+            try:
+                Hn.check_combine(out, want[b0:b1])
+            except AssertionError:
+                parity = False
+            block["remote_payload_bytes_rank0"] = remote_bytes(cfg, lay.slot_row, ids, 0)
+        # timing: dispatch (with the routing all-gather and the arrival wait) and combine (with its fences)
+        n_it = 50
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        td = tc = 0.0
+        for it in range(n_it + 5):
+            ev[0].record()
+            region, n = ep.dispatch(x, idx, w, cfg.T)
+            ev[1].record()
+            ep.combine()
+            ev[2].record()
+            torch.cuda.synchronize(dev)
+            if it >= 5:
+                td += ev[0].elapsed_time(ev[1])
+                tc += ev[1].elapsed_time(ev[2])
+        td_us = max_over_ranks(td / n_it * 1e3, world, dev)
+        tc_us = max_over_ranks(tc / n_it * 1e3, world, dev)
+        status = ep.status()
+        block.update({"status": "ok" if status == 0 else B.ubep_strerror(status), "parity": parity,
+                      "dispatch_us": td_us, "combine_us": tc_us,
+                      "workload": f"T={cfg.T} H={cfg.H} E={cfg.E} R={world} k={cfg.k} bf16 dedup=1, identity experts",
+                      "timed": "dispatch = routing all-gather + ubep_dispatch_sharded + ubep_wait_arrivals; "
+                               "combine = fence + ubep_combine_sharded + fence; CUDA events, max over ranks"})
+        if rank == 0 and block.get("remote_payload_bytes_rank0"):
+            block["nvlink_gbs_rank0_dispatch"] = block["remote_payload_bytes_rank0"] / (td_us * 1e-6) / 1e9
+        _ = dist
+    except Exception as e:          # this block must never take the first line with it
+        block["status"] = f"{type(e).__name__}: {e}"
+    if rank == 0:
+        print(json.dumps({"sharded": block, "n_gpus": world, "metric": "dispatch / combine us with one rank per GPU",
+                          "data": "synthetic"}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -716,12 +817,17 @@ def main():
     args.steps = args.steps if args.steps is not None else 200
     args.warmup = args.warmup if args.warmup is not None else 20
     if world > 1:
+        import datetime
         import torch
         import torch.distributed as dist
         torch.cuda.set_device(local_rank)
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank),
+                                timeout=datetime.timedelta(seconds=120))
     try:
         run_ours(args, cfg, rank, world, local_rank)
+        if world > 1 and not args.profile:
+            sys.stdout.flush()
+            run_sharded(args, rank, world, local_rank)
     finally:
         if world > 1:
             import torch.distributed as dist

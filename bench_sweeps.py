@@ -3,12 +3,18 @@
 
     python bench_sweeps.py spread [--workload skewed prefill] [--rows 4] [--markdown]
     python bench_sweeps.py sync   [--tokens 128] [--iters 200] [--markdown]
+    python bench_sweeps.py roles  [--tokens 512 1024 4096 16384] [--count-warps 0 1 2 4 8] [--markdown]
+    python bench_sweeps.py auto   [--tokens 64 128 256 512 1024 2048] [--markdown]
 
 spread: per-CTA latency spread of dispatch under different destination-ordering tables -- the
 analogue, on one GPU, of the paper's per-worker token-transmission latencies with and without
 expert re-mapping (Sec. 5.4, "Impact of Token Scheduling").
 sync: latency of the readiness protocols (stop-and-wait, Token-Flag Fusion, Data-for-Checksum,
 Sentinel Polling; Sec. 3.4) over synchronisation granularity and rank count.
+roles: FP8 dispatch time over the size of the count group (the paper's core-allocation question:
+Sec. 3.2, the cost model of App. A, the group-size heat maps of App. C.3).
+auto: the flag-free (LOCAL) against the flag-exchanging (FUSED) schedule over token counts and shape
+families, and what AUTO picks.
 """
 from __future__ import annotations
 
@@ -214,7 +220,91 @@ def main_sync(argv):
                       f"{m['layout_us']:.2f} | {m['sent_us']:.2f} | {m['ready_us']:.2f} | {m['wire_ratio']:.3f} |")
 
 
-SWEEPS = {"spread": main_spread, "sync": main_sync}
+# ------------------------------------------------------------------------- roles / auto
+
+def dispatch_us(cfg: W.Config, pipeline: int = 0, count_warps: int = -1, min_timed_s: float = 0.08):
+    """Median time of one ubep_dispatch on rotating buffer sets (cold L2), timed like bench.py does:
+    graphs of dispatches only, blocks between CUDA events.  Returns (us, what AUTO would run it as)."""
+    import bench as BM
+
+    class A:
+        quant_warps = 0
+        prefetch_rows = 0
+        no_graph = False
+    A.pipeline, A.count_warps = pipeline, count_warps
+    b = BM.Bench(cfg, A, 0, 1)
+    steps = 2 * b.nsets
+    blocks = b.time_blocks(b.make_block(b.dispatch, steps), steps, 1, min_timed_s=min_timed_s)
+    us = BM.summarize_blocks(blocks, steps)["median_us"]
+    status = b.sets[0]["buf"].status()
+    b.close()
+    if status != 0:
+        raise RuntimeError(f"device status {status} ({B.ubep_strerror(status)})")
+    return us
+
+
+def predicted_count_share(E: int, k: int, tokens_per_cta: float) -> float:
+    """The paper's cost model (App. A): the share of workers that should count grows with the number
+    of experts and shrinks with top-k times the tokens a worker sends, n_count ~ N_exp / (K_top * B_sz)."""
+    return E / (k * max(tokens_per_cta, 1e-9))
+
+
+def main_roles(argv):
+    ap = argparse.ArgumentParser(prog="bench_sweeps.py roles")
+    ap.add_argument("--tokens", type=int, nargs="*", default=[512, 1024, 4096, 16384])
+    ap.add_argument("--count-warps", type=int, nargs="*", default=[0, 1, 2, 4, 8])
+    ap.add_argument("--shapes", nargs="*", default=["256,8", "128,8", "288,8", "256,4"], help="E,k pairs")
+    ap.add_argument("--markdown", action="store_true")
+    args = ap.parse_args(argv)
+    B.load()
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    head = ["E", "k", "T", "tokens / CTA", "E / (k * tokens per CTA)"] + [f"n_count={n}" for n in args.count_warps] + ["best"]
+    if args.markdown:
+        print("| " + " | ".join(head) + " |")
+        print("|" + "---|" * len(head))
+    for shape in args.shapes:
+        E, k = (int(v) for v in shape.split(","))
+        R = 72 if E == 288 else 32
+        for T in args.tokens:
+            cfg = W.Config(f"roles_E{E}_k{k}_T{T}", T=T, H=7168, E=E, R=R, k=k, payload=1, seed=9000 + T + E + k)
+            # FUSED asked for explicitly: the count group exists in the schedules with an exchange
+            times = [dispatch_us(cfg, B.UBEP_PIPELINE_FUSED, n) for n in args.count_warps]
+            best = args.count_warps[int(np.argmin(times))]
+            row = [E, k, T, f"{T / sms:.1f}", f"{predicted_count_share(E, k, T / sms):.2f}"] + [f"{t:.1f}" for t in times] + [best]
+            print(("| " + " | ".join(str(v) for v in row) + " |") if args.markdown else " ".join(str(v) for v in row), flush=True)
+
+
+def main_auto(argv):
+    ap = argparse.ArgumentParser(prog="bench_sweeps.py auto")
+    ap.add_argument("--tokens", type=int, nargs="*", default=[64, 128, 256, 512, 1024, 2048])
+    ap.add_argument("--markdown", action="store_true")
+    args = ap.parse_args(argv)
+    B.load()
+    families = [("H=7168 E=256 R=32", dict(H=7168, E=256, R=32)), ("H=4096 E=128 R=16", dict(H=4096, E=128, R=16)),
+                ("H=7168 E=288 R=72", dict(H=7168, E=288, R=72))]
+    head = ["family", "rows", "dedup", "T", "FUSED us", "LOCAL us", "AUTO us", "AUTO / better"]
+    if args.markdown:
+        print("| " + " | ".join(head) + " |")
+        print("|" + "---|" * len(head))
+    for label, shp in families:
+        for payload in (0, 1):
+            for dedup in (0, 1):
+                for T in args.tokens:
+                    cfg = W.Config(f"auto_T{T}", T=T, k=8, payload=payload, dedup=dedup, seed=9100 + T, **shp)
+                    fused = dispatch_us(cfg, B.UBEP_PIPELINE_FUSED)
+                    try:
+                        local = dispatch_us(cfg, B.UBEP_PIPELINE_LOCAL)
+                    except B.UbepError:
+                        local = float("nan")      # the table does not fit in shared memory
+                    auto = dispatch_us(cfg, B.UBEP_PIPELINE_AUTO)
+                    better = np.nanmin([fused, local])
+                    row = [label, "fp8" if payload else "bf16", dedup, T, f"{fused:.1f}", f"{local:.1f}", f"{auto:.1f}",
+                           f"{auto / better:.2f}"]
+                    print(("| " + " | ".join(str(v) for v in row) + " |") if args.markdown else " ".join(str(v) for v in row),
+                          flush=True)
+
+
+SWEEPS = {"spread": main_spread, "sync": main_sync, "roles": main_roles, "auto": main_auto}
 
 
 def main():

@@ -54,7 +54,13 @@ enum {
                               /* the bulk-synchronous dispatch (Sec. 2.3, phases 2-5)         */
     UBEP_PIPELINE_FUSED = 2,  /* one persistent kernel: count / prefix-sum warps publish      */
                               /* offsets through release/acquire flags while mover warps      */
-                              /* already stream rows (kernel decomposition, Sec. 3.2)         */
+                              /* already stream rows (kernel decomposition, Sec. 3.2).  Its   */
+                              /* CTAs wait for one another, so all num_ctas of them must be   */
+                              /* resident at once: the kernel is launched cooperatively, the  */
+                              /* launch fails (UBEP_ERR_CUDA) if the grid cannot fit on the   */
+                              /* device, and it starts only when every CTA has an SM -- a     */
+                              /* caller that keeps SMs busy on other streams should create    */
+                              /* the buffer with a smaller num_ctas                           */
     UBEP_PIPELINE_LOCAL = 3   /* one persistent kernel in which every CTA derives its offsets */
                               /* from the whole routing table itself (no flags; small T*k:    */
                               /* asked for explicitly with a table that does not fit in       */
@@ -74,7 +80,8 @@ typedef struct {
                                /* 1: one row per (token, rank), ascending token                */
     int32_t device;            /* CUDA device ordinal                                          */
     int32_t pipeline;          /* UBEP_PIPELINE_*                                              */
-    int32_t num_ctas;          /* persistent CTAs / token chunks; 0 = number of SMs.  The      */
+    int32_t num_ctas;          /* persistent CTAs / token chunks; 0 = number of SMs (never     */
+                               /* more: one CTA per SM, all resident at once).  The            */
                                /* bookkeeping of one chunk lives in shared memory: a dispatch  */
                                /* whose T / num_ctas tokens do not fit there (a few thousand   */
                                /* slots per CTA) returns UBEP_ERR_ARG and launches nothing     */
@@ -273,7 +280,9 @@ int ubep_map_workers(const int32_t *order /*[dev]*/, const int32_t *counts /*[de
  *
  * Limits: bf16 payload only; T * k <= 8192 and the routing table with the bitmaps of all its
  * bins (T x (E + R) bits) must fit in a CTA's shared memory, since every CTA derives the layout
- * from the whole table, as UBEP_PIPELINE_LOCAL does; one CTA per SM at most.  Everything
+ * from the whole table, as UBEP_PIPELINE_LOCAL does; one CTA per SM at most, launched
+ * cooperatively (receivers wait for senders of the same grid, so the grid must be resident at once:
+ * a grid that cannot be is refused with UBEP_ERR_CUDA instead of running into its timeouts).  Everything
  * ubep_dispatch leaves in the arena is left here too, with identical contents; ubep_combine
  * may follow.  The arrival counters of ubep_dispatch (UBEP_VIEW_ARRIVAL) are not touched.
  */
@@ -310,7 +319,8 @@ int ubep_sync_attach(ubep_buffer_t *buf, void *dev_wire /*[dev]*/, size_t bytes,
 /*
  * Dispatch with readiness protocol `protocol` (UBEP_SYNC_*); arguments as ubep_dispatch.
  * One kernel launch (a memset before it when an earlier call left the SP wire dirty, which
- * the library learns when ubep_status reports that call's error).  UBEP_ERR_ARG if no wire
+ * the library learns when ubep_status reports that call's error; until then a word on the
+ * device makes every Sentinel Polling call on that wire report UBEP_ERR_TIMEOUT and move nothing).  UBEP_ERR_ARG if no wire
  * buffer is attached, the payload is not bf16, T * k > 8192 or the table does not fit in shared
  * memory.
  */
@@ -430,9 +440,11 @@ int ubep_debug_trace(ubep_buffer_t *buf, int32_t enable);
  * ubep_debug_set_count_warps: n warps (the store issuer among them) form the count group that
  * computes the layout -- TokenCnt, the flag exchange, CalCumSum, row assignment -- while the
  * remaining 15 - n warps already quantise the rows the loader has fetched into a ring of
- * quantised rows that waits for the layout (1 <= n <= 13; default 4).  n = 0: all 15 warps
- * compute the layout and 14 of them quantise afterwards.  Applies to the PHASED and FUSED
- * schedules; the flag-free LOCAL schedule, whose layout waits for nobody, always runs as n = 0.
+ * quantised rows that waits for the layout (1 <= n <= 13).  TokenCnt itself is done by all 15
+ * warps first; the count group is what goes on through the flag exchange.  n = 0: all 15 warps
+ * compute the layout and 14 of them quantise afterwards.  n = -1 (default): 8, or 0 when slices
+ * are long enough for token stealing.  Applies to the PHASED and FUSED schedules; the flag-free
+ * LOCAL schedule, whose layout waits for nobody, always runs as n = 0.
  * ubep_debug_set_quant_warps: at most n warps quantise (1 <= n <= 14, default 14), the rest idle.
  * ubep_debug_set_prefetch_rows: the loader fetches at most n rows before the layout is done
  * (default: as many as the rings hold).

@@ -3,6 +3,7 @@
 #include <atomic>
 #include <climits>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <string>
@@ -21,11 +22,16 @@ std::atomic<uint64_t> g_launches{0};
 
 constexpr size_t kAlign = 256;
 constexpr int kStealMinTokensPerChunk = 40;  // shorter slices: the hand-out costs more than the tail it removes (measured)
-constexpr int kDefaultCountWarps = 4;            // FP8: warps of the layout group while the others quantise (measured sweep)
+constexpr int kDefaultCountWarps = 8;            // FP8: warps of the count group while the others quantise (measured sweep;
+                                                 // -1 in the buffer = this default, and none with token stealing)
 constexpr int64_t kLocalMaxSlots = 8192;        // small-T limit of the combine launch mode and of the protocol / sharded paths
-constexpr int64_t kLocalFastMaxSlots = 14336;   // AUTO: flag-free kernel with the rank-level fast path up to this many slots
-constexpr int64_t kLocalMaxWeight = 18432;      // AUTO: flag-free kernel over every bin up to this many slots x bin words
-constexpr int64_t kLocalFp8MaxWeight = 9216;    // the same with FP8 rows
+// AUTO's crossovers between the flag-free and the flag-exchanging schedule, in routing-table slots (T * k);
+// measured over three shape families (H / E / R = 7168 / 256 / 32, 4096 / 128 / 16, 7168 / 288 / 72), top-8,
+// 64 .. 2048 tokens: the crossover follows the slots, not the number of bins.
+constexpr int64_t kLocalFastMaxSlots = 14336;     // one row per (token, rank), bf16 rows: the rank-level fast path
+constexpr int64_t kLocalFastFp8MaxSlots = 6144;   // the same with FP8 rows (their quantising warps are the layout warps)
+constexpr int64_t kLocalAllBinsMaxSlots = 3072;   // every bin's bitmaps have to be built, bf16 rows
+constexpr int64_t kLocalAllBinsFp8MaxSlots = 1536;   // ... FP8 rows
 inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 
 struct ArenaLayout {
@@ -109,7 +115,7 @@ ArenaLayout make_layout(const ubep_config_t& c, int nchunks) {
 // Wire buffer of the readiness-protocol dispatch (byte offsets).
 struct WireLayout {
     size_t off[UBEP_SYNC_VIEW_COUNT_];
-    size_t flags_begin, seq_ticket, scan_count, flags_end, total;
+    size_t flags_begin, sp_dirty, seq_ticket, scan_count, flags_end, total;
     int tff_blocks;
 };
 
@@ -125,6 +131,7 @@ WireLayout make_wire_layout(const ubep_config_t& c, int nchunks) {
     w.flags_begin = at;
     w.off[UBEP_SYNC_VIEW_CHECKSUM] = take(2 * R * 8);
     w.off[UBEP_SYNC_VIEW_COUNTERS] = take(4 * R * 4);
+    w.sp_dirty = take(4);   // (inside the range that is cleared when the wire is re-filled)
     w.off[UBEP_SYNC_VIEW_SEQ] = take(4);
     w.seq_ticket = take(4);
     w.scan_count = take(8);
@@ -210,7 +217,7 @@ Params make_params(ubep_buffer* b, int T) {
     p.claimed = at<unsigned>(b, a.claimed);
     p.steal = 0;
     p.quant_warps = b->quant_warps;
-    p.count_warps = b->count_warps;
+    p.count_warps = b->count_warps < 0 ? kDefaultCountWarps : b->count_warps;
     p.prefetch_rows = b->prefetch_rows;
     p.chunk_hist = at<int32_t>(b, a.chunk_hist);
     p.partial = at<int32_t>(b, a.partial);
@@ -279,7 +286,7 @@ int ubep_buffer_create(const ubep_config_t* cfg, void* dev_arena, size_t bytes, 
     b->withhold = -1;
     b->tracing = 0;
     b->quant_warps = ubep::kWarps - 2;
-    b->count_warps = kDefaultCountWarps;
+    b->count_warps = -1;
     b->prefetch_rows = INT32_MAX;
     b->last_stream = nullptr;
     b->phys = nullptr;
@@ -385,14 +392,14 @@ int ubep_dispatch(ubep_buffer_t* buf, const void* x, const int32_t* topk_idx, co
     // than to exchange through flags; larger ones use the decomposed kernel.
     int mode = buf->cfg.pipeline;
     if (mode == UBEP_PIPELINE_AUTO) {
-        // Measured crossovers (H = 7168, 256 experts on 32 ranks, top-8).  With the rank-level fast path
-        // the flag-free kernel wins up to about 1800 tokens; when every CTA has to build the bitmaps of
-        // every bin its cost grows with slots x bin words and it wins only for a few hundred tokens, and
-        // with FP8 rows (whose quantising warps are the layout warps, so nothing moves before the layout
-        // and its outputs are done) for about a hundred.
-        const int64_t slots = (int64_t)T * p.k, weight = slots * ((p.B + 31) / 32);
-        const bool local = p.local_fast ? slots <= kLocalFastMaxSlots
-                                        : weight <= (p.payload ? kLocalFp8MaxWeight : kLocalMaxWeight);
+        // With the rank-level fast path the flag-free kernel wins up to about 1800 tokens of top-8 (bf16 rows);
+        // when every CTA has to build the bitmaps of every bin it wins only for a few hundred tokens, and
+        // with FP8 rows (whose quantising warps are the layout warps there, so nothing moves before the
+        // layout and its outputs are done) for fewer still.
+        const int64_t slots = (int64_t)T * p.k;
+        const int64_t limit = p.local_fast ? (p.payload ? kLocalFastFp8MaxSlots : kLocalFastMaxSlots)
+                                           : (p.payload ? kLocalAllBinsFp8MaxSlots : kLocalAllBinsMaxSlots);
+        const bool local = slots <= limit;
         mode = local ? UBEP_PIPELINE_LOCAL : UBEP_PIPELINE_FUSED;
     }
     ubep::SmemPlan pl{};
@@ -430,6 +437,9 @@ int ubep_dispatch(ubep_buffer_t* buf, const void* x, const int32_t* topk_idx, co
     }
     // slices that are long enough are handed out in blocks so that faster SMs can take over the tail of slower ones
     if (mode != UBEP_PIPELINE_LOCAL) p.steal = T >= kStealMinTokensPerChunk * p.nchunks ? 1 : 0;
+    // With token stealing the count group is not used unless asked for: measured equal at top-8 and slower at
+    // top-4 (16384 tokens: 161 against 174 us) -- every hand-out is a round trip that idle quantising warps do not hide.
+    if (p.steal && buf->count_warps < 0) p.count_warps = 0;
     if (mode != UBEP_PIPELINE_LOCAL && ubep::plan_dispatch(p, mode, buf->max_smem, &pl) != 0) return UBEP_ERR_ARG;
     cudaError_t e = ubep::launch_dispatch(p, mode, pl, st, &launches);
     if (e != cudaSuccess) return cuda_fail(buf, e);
@@ -518,6 +528,7 @@ int ubep_dispatch_sync(ubep_buffer_t* buf, int protocol, const void* x, const in
     sp.sw_rows = sp.announced + 2 * (size_t)p.R;
     sp.seq_ctr = reinterpret_cast<unsigned*>(buf->wire + w.off[UBEP_SYNC_VIEW_SEQ]);
     sp.seq_ticket = reinterpret_cast<unsigned*>(buf->wire + w.seq_ticket);
+    sp.sp_dirty = reinterpret_cast<unsigned*>(buf->wire + w.sp_dirty);
     sp.times = reinterpret_cast<unsigned long long*>(buf->wire + w.off[UBEP_SYNC_VIEW_TIMES]);
     cudaError_t e = cudaSuccess;
     if (buf->sp_dirty) {
@@ -744,7 +755,7 @@ int ubep_debug_set_quant_warps(ubep_buffer_t* buf, int32_t n) {
 }
 
 int ubep_debug_set_count_warps(ubep_buffer_t* buf, int32_t n) {
-    if (!buf || n < 0 || n > ubep::kWarps - 3) return UBEP_ERR_ARG;
+    if (!buf || n < -1 || n > ubep::kWarps - 3) return UBEP_ERR_ARG;
     buf->count_warps = n;
     return UBEP_OK;
 }

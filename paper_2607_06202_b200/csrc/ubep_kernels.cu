@@ -1075,18 +1075,27 @@ int plan_dispatch(const Params& p, int mode, int max_smem, SmemPlan* out) {
 }
 
 // Launch that lets the kernel be placed while its predecessor in the stream drains (the
-// kernels above call griddep_wait() before they read anything).
+// kernels above call griddep_wait() before they read anything).  `together`: a cooperative
+// launch -- the kernel's CTAs wait for flags that other CTAs of the same grid publish, so they
+// must all be resident at once; the runtime then refuses a grid that cannot be (a synchronous
+// error instead of CTAs spinning until their bounded waits run out) and starts the grid only
+// when every CTA has a place.  Such a kernel is not launched ahead of its predecessor's end.
 template <typename... KArgs, typename... Args>
 static cudaError_t launch_overlapped(void (*kern)(KArgs...), int grid, int block, size_t smem, cudaStream_t st,
-                                     Args... args) {
+                                     bool together, Args... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3((unsigned)block);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    if (together) {
+        attr[0].id = cudaLaunchAttributeCooperative;
+        attr[0].val.cooperative = 1;
+    } else {
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+    }
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kern, args...);
@@ -1113,7 +1122,7 @@ static cudaError_t launch_dispatch_s(const Params& p, const SmemPlan& pl, cudaSt
     static std::atomic<int> granted[kAttrDevices];
     cudaError_t e = allow_dynamic_smem(reinterpret_cast<const void*>(kern), pl.total, granted);
     if (e != cudaSuccess) return e;
-    return launch_overlapped(kern, p.grid, kThreads, (size_t)pl.total, st, p, pl);
+    return launch_overlapped(kern, p.grid, kThreads, (size_t)pl.total, st, kMode == kModeFused, p, pl);
 }
 
 template <int kMode, bool kFp8>
@@ -1148,7 +1157,7 @@ cudaError_t launch_dispatch(const Params& p, int mode, const SmemPlan& pl, cudaS
 template <int K>
 static cudaError_t launch_combine_k(bool ahead, int g, cudaStream_t st, const uint16_t* y, const int32_t* slot_pos,
                                     const float* topk_w, int T, int H, int k, uint16_t* out) {
-    if (ahead) return launch_overlapped(combine_kernel<K>, g, 256, 0, st, y, slot_pos, topk_w, T, H, k, out);
+    if (ahead) return launch_overlapped(combine_kernel<K>, g, 256, 0, st, false, y, slot_pos, topk_w, T, H, k, out);
     combine_kernel<K><<<g, 256, 0, st>>>(y, slot_pos, topk_w, T, H, k, out);
     return cudaGetLastError();
 }

@@ -69,6 +69,7 @@ struct Waiter {
     volatile int* abort;
     unsigned long long t_end;
     int32_t* status;
+    unsigned* dirty;   // Sentinel Polling: word that tells the next call that this one gave up (else null)
     __device__ __forceinline__ bool keep_waiting(unsigned& spins) {
         __nanosleep(32);
         if ((++spins & 127u) != 0) return true;
@@ -76,6 +77,7 @@ struct Waiter {
         if (global_ns() > t_end) {
             *abort = 1;
             report(status, kErrTimeout);
+            if (dirty) *dirty = 1u;
             return false;
         }
         return true;
@@ -117,6 +119,13 @@ __global__ void __launch_bounds__(kThreads, 1) sync_dispatch_kernel(const Params
     if (tid == 0) {
         seq_sm = read_seq_and_check_in(sp, p.grid);
         abort_flag = 0;
+        // Sentinel Polling after a call that gave up: blocks of that call may still sit in the wire and
+        // would be taken for this call's.  Nothing is sent or received then; the call reports the
+        // condition again, and the library re-fills the wire once it has learnt of it (ubep_status).
+        if (kProto == kSP && ld_relaxed(sp.sp_dirty) != 0u) {
+            abort_flag = 1;
+            report(p.status, kErrTimeout);
+        }
     }
     if (kProto == kDC)
         for (int r = tid; r < R; r += kThreads) chk_sm[r] = 0ull;
@@ -149,7 +158,8 @@ __global__ void __launch_bounds__(kThreads, 1) sync_dispatch_kernel(const Params
     const int nvec = p.rowB / 16;
     const int nwords = p.rowB / 4;
     const size_t wire_row = (size_t)sp.tff_blocks * 16;
-    for (int tl = 0; tl < ntok; ++tl) {
+    const bool wire_unusable = kProto == kSP && abort_flag != 0;   // (set before the barriers above, uniform in the CTA)
+    for (int tl = 0; tl < ntok && !wire_unusable; ++tl) {
         const int* ps = pos + tl * k;
         if (kProto == kTFF) {
             const uint32_t* xw = reinterpret_cast<const uint32_t*>(p.x + (size_t)(t0 + tl) * p.H);
@@ -212,7 +222,7 @@ __global__ void __launch_bounds__(kThreads, 1) sync_dispatch_kernel(const Params
     if (tid == 0) times[2] = global_ns();
 
     // ---- receiver: region u / Q, slice u % Q of its rows
-    Waiter wt{&abort_flag, global_ns() + kWaitLimitNs, p.status};
+    Waiter wt{&abort_flag, global_ns() + kWaitLimitNs, p.status, kProto == kSP ? sp.sp_dirty : nullptr};
     const int Q = p.grid / R > 1 ? p.grid / R : 1;
     bool duty = false;
     for (int u = c; u < R * Q; u += p.grid) {
@@ -323,8 +333,19 @@ cudaError_t launch_one(const Params& p, const SmemPlan& pl, const SyncParams& sp
     const int smem = pl.total + sync_extra_smem(p);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    kern<<<p.grid, kThreads, smem, st>>>(p, pl, sp);
-    return cudaGetLastError();
+    // Receivers wait for senders that are other CTAs of this grid: a cooperative launch, which the
+    // runtime refuses when the grid cannot be resident at once and starts only when it is.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)p.grid);
+    cfg.blockDim = dim3((unsigned)kThreads);
+    cfg.dynamicSmemBytes = (size_t)smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, p, pl, sp);
 }
 
 }  // namespace

@@ -21,6 +21,7 @@ struct SyncParams {
     unsigned* sw_rows;              // [2][R] rows whose stores have been fenced
     unsigned* seq_ctr;              // calls completed
     unsigned* seq_ticket;           // CTAs of the running call that have read seq_ctr
+    unsigned* sp_dirty;             // != 0: a Sentinel Polling call gave up and may have left arrived blocks in the wire
     unsigned long long* times;      // [grid][kSyncTimeSlots]
 };
 

@@ -64,7 +64,12 @@ class ShardedEP:
 
     def __init__(self, *, num_experts: int, hidden: int, topk: int, max_tokens: int, rows_per_rank_cap: int,
                  dedup: int = 0, payload: int = 0, group=None, device: Optional[torch.device] = None,
-                 alloc: Callable = symmetric_alloc):
+                 alloc: Callable = symmetric_alloc, backend=B):
+        """`alloc(nbytes, device, group)` returns memory every rank can address and its address on every
+        rank; `backend` is the binding module.  Both can be replaced by stand-ins, which is how the
+        order of the steps is tested on CPU ranks."""
+        B = backend  # noqa: N806  (the names below are the binding's)
+        self.B = backend
         self.group = group
         self.rank, self.world = dist.get_rank(group), dist.get_world_size(group)
         self.device = device if device is not None else torch.device("cuda", torch.cuda.current_device())
@@ -104,8 +109,8 @@ class ShardedEP:
         """Routes this rank's tokens; returns when (on the stream) this rank's region is complete."""
         self.T = T
         self.idx, self.w = gather_routing(idx_local, w_local, T, self.group)
-        B.ubep_dispatch_sharded(self.buf.handle, x_local.contiguous(), self.idx, self.w, T)
-        B.ubep_wait_arrivals(self.buf.handle)
+        self.B.ubep_dispatch_sharded(self.buf.handle, x_local.contiguous(), self.idx, self.w, T)
+        self.B.ubep_wait_arrivals(self.buf.handle)
         return self.region, self.buf.num_rows_per_rank[self.rank]
 
     def combine(self, out_local: Optional[torch.Tensor] = None) -> torch.Tensor:
@@ -114,7 +119,7 @@ class ShardedEP:
         if out_local is None:
             out_local = torch.empty((b1 - b0, self.H), dtype=torch.bfloat16, device=self.device)
         self.fence()     # every rank's y is complete
-        B.ubep_combine_sharded(self.buf.handle, self.y_ptrs, self.w, self.T, out_local)
+        self.B.ubep_combine_sharded(self.buf.handle, self.y_ptrs, self.w, self.T, out_local)
         self.fence()     # nobody overwrites a region or a y that a peer still reads
         return out_local
 

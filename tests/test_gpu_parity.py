@@ -341,7 +341,7 @@ def test_warp_role_split_does_not_change_results(shape, count_warps, quant_warps
 def test_warp_role_knobs_reject_values_out_of_range():
     cfg = small(64, payload=1, H=256)
     buf = Hn.make_buffer(cfg, 128)
-    for fn, bad in ((B.ubep_debug_set_quant_warps, (0, 15)), (B.ubep_debug_set_count_warps, (-1, 14)),
+    for fn, bad in ((B.ubep_debug_set_quant_warps, (0, 15)), (B.ubep_debug_set_count_warps, (-2, 14)),
                     (B.ubep_debug_set_prefetch_rows, (0,))):
         for v in bad:
             with pytest.raises(B.UbepError):

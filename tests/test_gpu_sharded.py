@@ -183,3 +183,38 @@ def test_driver_with_one_rank(tmp_path):
     out_path = str(tmp_path / "r0.txt")
     mp.spawn(_driver_worker, args=(1, 29751, out_path), nprocs=1, join=True)
     assert open(out_path).read() == "ok"
+
+
+def _bench_block_worker(rank, world, port, out_path):
+    import contextlib
+    import io
+    import json
+    import os
+    import sys
+    import torch.distributed as dist
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    sys.path.insert(0, root)
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    torch.cuda.set_device(0)
+    dist.init_process_group("nccl", rank=rank, world_size=world)
+    import bench
+    buf = io.StringIO()
+    with contextlib.redirect_stdout(buf):
+        bench.run_sharded(None, rank, world, 0)
+    line = json.loads(buf.getvalue().strip().splitlines()[-1])
+    with open(out_path, "w") as f:
+        json.dump(line, f)
+    dist.destroy_process_group()
+
+
+def test_the_benchmarks_block_for_ranks_on_different_gpus_with_one_rank(tmp_path):
+    """What bench.py prints as its second line under torchrun, run here with a group of one: the
+    decode-like shape through ShardedEP, rank 0's region and output against the oracle."""
+    import json
+    import torch.multiprocessing as mp
+    out_path = str(tmp_path / "line.json")
+    mp.spawn(_bench_block_worker, args=(1, 29753, out_path), nprocs=1, join=True)
+    blk = json.load(open(out_path))["sharded"]
+    assert blk["status"] == "ok", blk
+    assert blk["parity"] is True and blk["nranks"] == 1
+    assert blk["dispatch_us"] > 0 and blk["combine_us"] > 0

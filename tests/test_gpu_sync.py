@@ -163,6 +163,17 @@ def test_sentinel_in_the_data_runs_into_the_bounded_wait_and_the_next_call_recov
     buf.dispatch_sync("sp", x, idx, w)
     Hn.check_dispatch(buf, wl, lay, cap, recv, arrival=False)
     wire_checks(buf, "sp", cfg, lay, recv, buf.sync_views["times"].shape[0])
+    # A caller that does not ask for the status after the call that gave up: the next Sentinel Polling
+    # call must not take that call's leftover blocks for its own -- it reports the condition again
+    # and moves nothing; once the status has been read the wire is re-filled and all is well.
+    buf.dispatch_sync("sp", Hn.to_dev(xb, torch.bfloat16), idx, w)      # gives up
+    buf.recv_x.fill_(Hn.FILL)
+    buf.dispatch_sync("sp", x, idx, w)                                   # no status read in between
+    torch.cuda.synchronize()
+    assert bool((buf.recv_x == Hn.FILL).all()), "a call on a dirty wire must not deliver anything"
+    assert buf.status() == B.UBEP_ERR_TIMEOUT
+    buf.dispatch_sync("sp", x, idx, w)
+    Hn.check_dispatch(buf, wl, lay, cap, recv, arrival=False)
     # the other protocols carry the same bytes without trouble
     for proto in ("tff", "dc", "sw"):
         buf.dispatch_sync(proto, Hn.to_dev(xb, torch.bfloat16), idx, w)
