@@ -264,6 +264,8 @@ class Bench:
         # rotating sets: by the time a set comes round again, several L2s' worth of other data went by
         self.touched = self.disp_b + self.comb_b
         self.nsets = int(min(16, max(4, np.ceil(4 * L2_BYTES / self.touched) + 1)))
+        if getattr(args, "sets", 0):
+            self.nsets = int(args.sets)      # (profiling runs: fewer sets, less memory held under ncu)
         self.sets = [self.make_set() for _ in range(self.nsets)]
         self.stream = torch.cuda.Stream(device=dev)
         self._graphs = []
@@ -799,6 +801,7 @@ def main():
     ap.add_argument("--count-warps", type=int, default=-1,
                     help="FP8 dispatch: warps of the count group, the others quantise beside it (-1 = library default)")
     ap.add_argument("--prefetch-rows", type=int, default=0, help="FP8 dispatch: rows fetched before the layout is done")
+    ap.add_argument("--sets", type=int, default=0, help="buffer sets to rotate through (0 = enough to exceed L2 fourfold)")
     ap.add_argument("--profile", action="store_true",
                     help="plain launches of the timed steps only (for ncu): no graph, no e2e, no CPU leg")
     args = ap.parse_args()

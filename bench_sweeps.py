@@ -5,6 +5,7 @@
     python bench_sweeps.py sync   [--tokens 128] [--iters 200] [--markdown]
     python bench_sweeps.py roles  [--tokens 512 1024 4096 16384] [--count-warps 0 1 2 4 8] [--markdown]
     python bench_sweeps.py auto   [--tokens 64 128 256 512 1024 2048] [--markdown]
+    python bench_sweeps.py budget [--workload decode] [--markdown]
 
 spread: per-CTA latency spread of dispatch under different destination-ordering tables -- the
 analogue, on one GPU, of the paper's per-worker token-transmission latencies with and without
@@ -15,6 +16,9 @@ roles: FP8 dispatch time over the size of the count group (the paper's core-allo
 Sec. 3.2, the cost model of App. A, the group-size heat maps of App. C.3).
 auto: the flag-free (LOCAL) against the flag-exchanging (FUSED) schedule over token counts and shape
 families, and what AUTO picks.
+budget: where the microseconds of one layer go: the dispatch kernel's phases from the library's trace,
+taken inside the steady replay of dispatch + combine graphs, beside what a kernel boundary costs by
+itself (a chain of empty kernels).
 """
 from __future__ import annotations
 
@@ -304,7 +308,79 @@ def main_auto(argv):
                           flush=True)
 
 
-SWEEPS = {"spread": main_spread, "sync": main_sync, "roles": main_roles, "auto": main_auto}
+# ----------------------------------------------------------------------------------- budget
+
+PHASES = [(0, "CTA starts (predecessor complete)"), (1, "routing table staged, bitmaps built"), (5, "rows assigned"),
+          (6, "movers released"), (7, "first row in shared memory, first copies issued"), (8, "last copy issued"),
+          (9, "copies complete"), (3, "expert-level outputs written (duty group)"), (10, "CTA ends")]
+
+
+def main_budget(argv):
+    import bench as BM
+    ap = argparse.ArgumentParser(prog="bench_sweeps.py budget")
+    ap.add_argument("--workload", default="decode")
+    ap.add_argument("--markdown", action="store_true")
+    args = ap.parse_args(argv)
+    B.load()
+
+    class A:
+        pipeline = 0
+        quant_warps = 0
+        count_warps = -1
+        prefetch_rows = 0
+        no_graph = False
+    cfg = W.CONFIGS[args.workload]
+    b = BM.Bench(cfg, A, 0, 1)
+    steps = 4 * b.nsets
+    # (1) the layer and its kernels, as bench.py times them
+    layer = BM.summarize_blocks(b.time_blocks(b.make_block(b.step, steps), steps, 2, min_timed_s=0.1), steps)
+    disp = BM.summarize_blocks(b.time_blocks(b.make_block(b.dispatch, steps), steps, 1, min_timed_s=0.05), steps)
+    comb = BM.summarize_blocks(b.time_blocks(b.make_block(b.combine, steps), steps, 1, min_timed_s=0.05), steps)
+    # (2) what a kernel boundary costs: chains of empty kernels, ordinary and programmatic launches
+    h = b.sets[0]["buf"].handle
+    empty = {}
+    for label, ahead in (("ordinary launch", False), ("programmatic stream serialization", True)):
+        def one(_s, ahead=ahead):
+            B.ubep_debug_empty_launch(h, ahead, b.stream)
+        blocks = b.time_blocks(b.make_block(one, 200), 200, 1, min_timed_s=0.05)
+        empty[label] = BM.summarize_blocks(blocks, 200)
+    # (3) the dispatch kernel's phases inside the steady replay of dispatch + combine
+    for s in b.sets:
+        B.ubep_debug_trace(s["buf"].handle, True)
+    blk = b.make_block(b.step, steps)
+    for _ in range(3):
+        blk()
+    torch.cuda.synchronize()
+    acc = []
+    for _ in range(6):
+        blk()
+        torch.cuda.synchronize()
+        acc += [s["buf"].trace.cpu().numpy().astype(np.int64).copy() for s in b.sets]
+    rows = []
+    for slot, label in PHASES:
+        per = []
+        for tr in acc:
+            t0 = tr[:, 0].min()
+            ok = (tr[:, slot] >= t0) & (tr[:, slot] < t0 + 10 ** 7)
+            col = (tr[ok, slot] - t0) / 1e3
+            if len(col):
+                per.append((col.min(), np.median(col), col.max()))
+        if per:
+            rows.append((label,) + tuple(np.median(np.array(per), 0)))
+    b.close()
+    p = print
+    p(f"workload {args.workload}: layer {layer['median_us']:.2f} us (min {layer['min_us']:.2f}); dispatch alone "
+      f"{disp['median_us']:.2f}, combine alone {comb['median_us']:.2f} (each: per kernel in a chain of its own kind)")
+    for label, e in empty.items():
+        p(f"empty kernel, {label}: {e['median_us']:.2f} us per launch in a chain (min {e['min_us']:.2f})")
+    if args.markdown:
+        p("\n| phase of the dispatch kernel (us after the first CTA's start) | earliest CTA | median CTA | last CTA |")
+        p("|---|---|---|---|")
+    for label, lo, med, hi in rows:
+        p((f"| {label} | {lo:.2f} | {med:.2f} | {hi:.2f} |") if args.markdown else f"{label:60s} {lo:7.2f} {med:7.2f} {hi:7.2f}")
+
+
+SWEEPS = {"spread": main_spread, "sync": main_sync, "roles": main_roles, "auto": main_auto, "budget": main_budget}
 
 
 def main():

@@ -365,8 +365,11 @@ int ubep_sync_scan_sentinel(ubep_buffer_t *buf, const void *x /*[dev]*/, int32_t
  * The caller orders the steps across ranks where data is reused: no rank may start dispatch
  * n + 1 before every rank has finished reading what dispatch n delivered, and no rank may
  * start combine before the y of every peer is complete (a barrier on the streams, e.g. an
- * NCCL one).  Limit of this path: T * k <= 8192 and the table with the bitmaps of all its
- * bins must fit in a CTA's shared memory (else UBEP_ERR_ARG).  Both payloads (FP8 rows are
+ * NCCL one).  A table of up to 8192 slots is recounted by every CTA (one launch); a larger one --
+ * or one whose bitmaps do not fit in a CTA's shared memory -- goes through two launches that count and
+ * prefix-sum the whole table, in chunks that do not straddle ranks, and a third that moves the
+ * rank's rows with (persistent CTAs / R) CTAs; R may not exceed the number of persistent CTAs then
+ * (else UBEP_ERR_ARG).  No count is exchanged either way.  Both payloads (FP8 rows are
  * quantised by the sender; scales land in the receiver's scale array).  Kernels of different
  * ranks never wait for one another except in ubep_wait_arrivals, which therefore must not be
  * emulated by launches queued on one GPU ahead of the senders it waits for.
@@ -453,6 +456,14 @@ int ubep_debug_trace(ubep_buffer_t *buf, int32_t enable);
 int ubep_debug_set_quant_warps(ubep_buffer_t *buf, int32_t n);
 int ubep_debug_set_count_warps(ubep_buffer_t *buf, int32_t n);
 int ubep_debug_set_prefetch_rows(ubep_buffer_t *buf, int32_t n);
+
+/*
+ * Measurement aid: launches a kernel that does nothing (one small CTA per SM) on `cuda_stream`,
+ * the ordinary way or, with ahead != 0, with programmatic stream serialization like the dispatch
+ * and the small-batch combine kernels.  Timed in a chain it gives the floor that every kernel
+ * boundary of a layer costs on this device.
+ */
+int ubep_debug_empty_launch(ubep_buffer_t *buf, int32_t ahead, void *cuda_stream);
 
 /* Text of the last CUDA runtime error seen by this buffer's calls ("" if none). */
 const char *ubep_last_cuda_error(const ubep_buffer_t *buf);

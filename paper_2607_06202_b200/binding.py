@@ -43,7 +43,7 @@ _VIEW_DTYPES = [torch.uint8, torch.float32, torch.int32, torch.float32, torch.in
 EXPORTS = ["ubep_buffer_bytes", "ubep_buffer_create", "ubep_buffer_destroy", "ubep_set_replicas",
            "ubep_set_dest_order", "ubep_get_dispatch_layout", "ubep_get_dispatch_layout_static", "ubep_dispatch", "ubep_combine", "ubep_view",
            "ubep_status", "ubep_epoch", "ubep_launch_count", "ubep_debug_withhold_flag", "ubep_debug_trace",
-           "ubep_debug_set_quant_warps", "ubep_debug_set_count_warps", "ubep_debug_set_prefetch_rows",
+           "ubep_debug_set_quant_warps", "ubep_debug_set_count_warps", "ubep_debug_set_prefetch_rows", "ubep_debug_empty_launch",
            "ubep_last_cuda_error", "ubep_strerror", "ubep_map_workers",
            "ubep_sync_wire_bytes", "ubep_sync_attach", "ubep_dispatch_sync", "ubep_sync_view",
            "ubep_sync_scan_sentinel",
@@ -91,6 +91,7 @@ def load() -> ctypes.CDLL:
     lib.ubep_debug_set_quant_warps.restype, lib.ubep_debug_set_quant_warps.argtypes = ctypes.c_int, [vp, i32]
     lib.ubep_debug_set_count_warps.restype, lib.ubep_debug_set_count_warps.argtypes = ctypes.c_int, [vp, i32]
     lib.ubep_debug_set_prefetch_rows.restype, lib.ubep_debug_set_prefetch_rows.argtypes = ctypes.c_int, [vp, i32]
+    lib.ubep_debug_empty_launch.restype, lib.ubep_debug_empty_launch.argtypes = ctypes.c_int, [vp, i32, vp]
     lib.ubep_last_cuda_error.restype, lib.ubep_last_cuda_error.argtypes = ctypes.c_char_p, [vp]
     lib.ubep_strerror.restype, lib.ubep_strerror.argtypes = ctypes.c_char_p, [ctypes.c_int]
     lib.ubep_map_workers.restype = ctypes.c_int
@@ -247,6 +248,10 @@ def ubep_debug_set_count_warps(buf, n: int) -> None:
 
 def ubep_debug_set_prefetch_rows(buf, n: int) -> None:
     _check(load().ubep_debug_set_prefetch_rows(buf, n), "ubep_debug_set_prefetch_rows", buf)
+
+
+def ubep_debug_empty_launch(buf, ahead: bool, stream=None) -> None:
+    _check(load().ubep_debug_empty_launch(buf, int(bool(ahead)), _stream(stream)), "ubep_debug_empty_launch", buf)
 
 
 def ubep_debug_withhold_flag(buf, chunk: int) -> None:

@@ -609,7 +609,7 @@ int ubep_set_peers(ubep_buffer_t* buf, int32_t my_rank, void* const* peer_arenas
 int ubep_dispatch_sharded(ubep_buffer_t* buf, const void* x_local, const int32_t* topk_idx, const float* topk_w,
                           int32_t T, void* cuda_stream) {
     if (!buf || buf->my_rank < 0) return UBEP_ERR_ARG;
-    if (T < 0 || T > buf->cfg.max_tokens || (int64_t)T * buf->cfg.topk > kLocalMaxSlots) return UBEP_ERR_ARG;
+    if (T < 0 || T > buf->cfg.max_tokens) return UBEP_ERR_ARG;
     if (T > 0 && (!topk_idx || !topk_w)) return UBEP_ERR_ARG;
     if (!aligned16(x_local) || !aligned16(topk_idx) || !aligned16(topk_w)) return UBEP_ERR_ARG;
     DeviceGuard guard(buf->cfg.device);
@@ -633,11 +633,28 @@ int ubep_dispatch_sharded(ubep_buffer_t* buf, const void* x_local, const int32_t
     p.parts = 1;
     p.grid = p.nchunks;
     ubep::SmemPlan pl{};
-    if (ubep::plan_dispatch(p, UBEP_PIPELINE_LOCAL, buf->max_smem - ubep::sharded_extra_smem(p), &pl) != 0)
-        return UBEP_ERR_ARG;
-    cudaError_t e = ubep::launch_sharded_dispatch(p, pl, st);
+    const bool whole_table = (int64_t)T * buf->cfg.topk <= kLocalMaxSlots &&
+                             ubep::plan_dispatch(p, UBEP_PIPELINE_LOCAL, buf->max_smem - ubep::sharded_extra_smem(p), &pl) == 0;
+    cudaError_t e;
+    if (whole_table) {
+        e = ubep::launch_sharded_dispatch(p, pl, true, st);
+        g_launches += 1;
+    } else {
+        // A table too large to recount in every CTA: TokenCnt and CalCumSum as launches of their own over the
+        // whole (all-gathered) table -- every rank still derives every count alone, nothing is exchanged --
+        // cut into R * m chunks so that no chunk straddles two ranks; m CTAs then move this rank's rows.
+        const int m = buf->lay.nchunks / R;
+        if (m < 1) return UBEP_ERR_ARG;   // more ranks than persistent CTAs
+        p.nchunks = R * m;
+        p.grid = m;
+        p.trace = nullptr;
+        if (ubep::plan_dispatch(p, UBEP_PIPELINE_PHASED, buf->max_smem - ubep::sharded_extra_smem(p), &pl) != 0)
+            return UBEP_ERR_ARG;
+        e = ubep::launch_count_scan(p, pl, st);
+        if (e == cudaSuccess) e = ubep::launch_sharded_dispatch(p, pl, false, st);
+        g_launches += 3;
+    }
     if (e != cudaSuccess) return cuda_fail(buf, e);
-    g_launches += 1;
     return UBEP_OK;
 }
 
@@ -763,6 +780,16 @@ int ubep_debug_set_count_warps(ubep_buffer_t* buf, int32_t n) {
 int ubep_debug_set_prefetch_rows(ubep_buffer_t* buf, int32_t n) {
     if (!buf || n < 1) return UBEP_ERR_ARG;
     buf->prefetch_rows = n;
+    return UBEP_OK;
+}
+
+int ubep_debug_empty_launch(ubep_buffer_t* buf, int32_t ahead, void* cuda_stream) {
+    if (!buf) return UBEP_ERR_ARG;
+    DeviceGuard guard(buf->cfg.device);
+    if (guard.err != cudaSuccess) return cuda_fail(buf, guard.err);
+    cudaError_t e = ubep::launch_empty(buf->num_sms, ahead != 0, static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return cuda_fail(buf, e);
+    g_launches += 1;
     return UBEP_OK;
 }
 

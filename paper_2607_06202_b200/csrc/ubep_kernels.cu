@@ -1131,18 +1131,25 @@ static cudaError_t launch_dispatch_t(const Params& p, const SmemPlan& pl, cudaSt
     return launch_dispatch_s<kMode, kFp8, false>(p, pl, st);
 }
 
+// TokenCnt and CalCumSum as two launches over the whole routing table (chunk histograms, then per rank
+// the prefix over chunks, expert offsets, totals and the per-source tables).
+cudaError_t launch_count_scan(const Params& p, const SmemPlan& pl, cudaStream_t st) {
+    cudaError_t e;
+    const int count_smem = pl.off_pos - pl.off_ids;   // ids + both bitmap arrays
+    static std::atomic<int> granted[kAttrDevices];
+    if ((e = allow_dynamic_smem(reinterpret_cast<const void*>(count_kernel), count_smem, granted)) != cudaSuccess)
+        return e;
+    count_kernel<<<p.nchunks, 256, count_smem, st>>>(p, pl);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    scan_kernel<<<p.R, 256, sizeof(int) * (p.L + 1), st>>>(p);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_dispatch(const Params& p, int mode, const SmemPlan& pl, cudaStream_t st, int* launches) {
     cudaError_t e;
     *launches = 1;
     if (mode == kModePhased) {
-        const int count_smem = pl.off_pos - pl.off_ids;   // ids + both bitmap arrays
-        static std::atomic<int> granted[kAttrDevices];
-        if ((e = allow_dynamic_smem(reinterpret_cast<const void*>(count_kernel), count_smem, granted)) != cudaSuccess)
-            return e;
-        count_kernel<<<p.nchunks, 256, count_smem, st>>>(p, pl);
-        if ((e = cudaGetLastError()) != cudaSuccess) return e;
-        scan_kernel<<<p.R, 256, sizeof(int) * (p.L + 1), st>>>(p);
-        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        if ((e = launch_count_scan(p, pl, st)) != cudaSuccess) return e;
         *launches = 3;
         return p.payload ? launch_dispatch_t<kModePhased, true>(p, pl, st)
                          : launch_dispatch_t<kModePhased, false>(p, pl, st);
@@ -1181,6 +1188,18 @@ cudaError_t launch_combine(const uint16_t* y, const int32_t* slot_pos, const flo
         case 8: return launch_combine_k<8>(ahead, g, st, y, slot_pos, topk_w, T, H, k, out);
         default: return launch_combine_k<0>(ahead, g, st, y, slot_pos, topk_w, T, H, k, out);
     }
+}
+
+// A kernel that does nothing, one CTA per SM: what a launch costs by itself.
+__global__ void __launch_bounds__(32) empty_kernel(int) {
+    griddep_launch();
+    griddep_wait();
+}
+
+cudaError_t launch_empty(int num_sms, bool ahead, cudaStream_t st) {
+    if (ahead) return launch_overlapped(empty_kernel, num_sms, 32, 0, st, false, 0);
+    empty_kernel<<<num_sms, 32, 0, st>>>(0);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_layout(const Params& p, int32_t* num_tokens_per_rank, int32_t* num_tokens_per_expert,

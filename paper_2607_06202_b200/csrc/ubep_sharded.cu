@@ -5,9 +5,11 @@
 // producing rank's buffer.  Plain loads and stores only: no TMA, no multicast, no collective.
 // FP8 rows are quantised by the sender, payload and scales go to the receiver's arrays.  No kernel here waits for another rank except wait_arrivals_kernel.
 //
-// Every rank derives the whole layout from the all-gathered routing table, alone, with the
-// same device functions and in the same order as the flag-free instance of the main dispatch
-// kernel, so all ranks agree on every row without exchanging a count.
+// Every rank derives the whole layout from the all-gathered routing table, alone, so all ranks
+// agree on every row without exchanging a count: for a small table inside the sender kernel, with
+// the same device functions and in the same order as the flag-free instance of the main dispatch
+// kernel; for a large one with the count and prefix-sum launches of the three-launch pipeline,
+// over chunks that do not straddle ranks.
 #include "ubep_layout.cuh"
 #include "ubep_quant.cuh"
 #include "ubep_sharded.h"
@@ -25,6 +27,10 @@ __device__ __forceinline__ unsigned ld_acquire_sys(const unsigned* ptr) {
     return v;
 }
 
+// kTable: the layout is derived here from the whole routing table in shared memory (small tables).
+// Otherwise it comes from count_kernel / scan_kernel, run before over the whole table with chunks that
+// do not straddle ranks: CTA c then owns chunk my_rank * grid + c of them and only stages its own tokens.
+template <bool kTable>
 __global__ void __launch_bounds__(kThreads, 1) sharded_dispatch_kernel(const Params p, const SmemPlan pl) {
     extern __shared__ __align__(128) uint8_t smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, c = blockIdx.x;
@@ -42,7 +48,9 @@ __global__ void __launch_bounds__(kThreads, 1) sharded_dispatch_kernel(const Par
                         pl.map_wb, pl.map_bp, pl.map_groups};
     // this CTA's share of the rank's own tokens [tok0, tok1)
     const int nloc = p.tok1 - p.tok0;
-    const int t0 = p.tok0 + (int)chunk_begin(c, nloc, p.nchunks), t1 = p.tok0 + (int)chunk_begin(c + 1, nloc, p.nchunks);
+    const int gch = p.my_rank * p.grid + c;   // (large tables) its chunk among the nchunks = R * grid chunks of all tokens
+    const int t0 = kTable ? p.tok0 + (int)chunk_begin(c, nloc, p.nchunks) : (int)chunk_begin(gch, p.T, p.nchunks);
+    const int t1 = kTable ? p.tok0 + (int)chunk_begin(c + 1, nloc, p.nchunks) : (int)chunk_begin(gch + 1, p.T, p.nchunks);
     const int ntok = t1 - t0;
 
     for (int r = tid; r < R; r += kThreads) {
@@ -50,29 +58,51 @@ __global__ void __launch_bounds__(kThreads, 1) sharded_dispatch_kernel(const Par
         sent[r] = 0;
         order_sm[r] = __ldg(p.order_pos + r);
     }
-    // ---- layout over the table of all T tokens (identical on every rank)
-    int* tot = hist;
-    int* pre = hist + p.B;
-    int* eo = hist + 2 * p.B;
-    stage_ids(p, 0, p.T, ids_sm, tid, kThreads);
-    for (int i = tid; i < ntok * k; i += kThreads) w_sm[i] = __ldg(p.topk_w + (size_t)t0 * k + i);
-    __syncthreads();
-    local_counts_all_bins(p, ids_sm, bmaps, t0, tot, pre, eo, tid, kThreads, warp, kWarps, lane, 0);
-    for (int r = tid; r < R; r += kThreads) nrows[r] = rows_of_rank(p, tot, r);
-    __syncthreads();
-    // rows of this CTA's slots; the metadata of every row goes to the arena of the rank that receives it
-    finalize_chunk<true>(p, t0, t1, ids_sm + (size_t)t0 * k, w_sm,
-                         [&](int e, int tl) { return eo[e] + pre[e] + bits_in_range(bmaps, e, t0, t0 + tl); },
-                         [&](int r, int tl) { return pre[p.E + r] + bits_in_range(bmaps, p.E + r, t0, t0 + tl); },
-                         true, c, order_sm, pos, key, sent, tid, kThreads, delta);
-    __syncthreads();
-    // counts and offsets: every rank keeps the whole set in its own arena
-    if (c == 0) {
-        write_totals(p, tot, eo, tid, kThreads);
-        // what the local receiver has to wait for (read by wait_arrivals_kernel, later in this stream)
-        if (tid == 0) atomicAdd(p.shard_arrival + 1, (unsigned)(nrows[p.my_rank] < p.cap ? nrows[p.my_rank] : p.cap));
+    if (kTable) {
+        // ---- layout over the table of all T tokens (identical on every rank)
+        int* tot = hist;
+        int* pre = hist + p.B;
+        int* eo = hist + 2 * p.B;
+        stage_ids(p, 0, p.T, ids_sm, tid, kThreads);
+        for (int i = tid; i < ntok * k; i += kThreads) w_sm[i] = __ldg(p.topk_w + (size_t)t0 * k + i);
+        __syncthreads();
+        local_counts_all_bins(p, ids_sm, bmaps, t0, tot, pre, eo, tid, kThreads, warp, kWarps, lane, 0);
+        for (int r = tid; r < R; r += kThreads) nrows[r] = rows_of_rank(p, tot, r);
+        __syncthreads();
+        // rows of this CTA's slots; the metadata of every row goes to the arena of the rank that receives it
+        finalize_chunk<true>(p, t0, t1, ids_sm + (size_t)t0 * k, w_sm,
+                             [&](int e, int tl) { return eo[e] + pre[e] + bits_in_range(bmaps, e, t0, t0 + tl); },
+                             [&](int r, int tl) { return pre[p.E + r] + bits_in_range(bmaps, p.E + r, t0, t0 + tl); },
+                             true, c, order_sm, pos, key, sent, tid, kThreads, delta);
+        __syncthreads();
+        // counts and offsets: every rank keeps the whole set in its own arena
+        if (c == 0) {
+            write_totals(p, tot, eo, tid, kThreads);
+            // what the local receiver has to wait for (read by wait_arrivals_kernel, later in this stream)
+            if (tid == 0) atomicAdd(p.shard_arrival + 1, (unsigned)(nrows[p.my_rank] < p.cap ? nrows[p.my_rank] : p.cap));
+        }
+        for (int s = c; s < p.S; s += p.grid) write_source_from_maps(p, s, bmaps, eo, tid, kThreads);
+    } else {
+        // ---- layout from the launches before: bitmaps of this CTA's own tokens, and per bin the rows of
+        // all earlier chunks (+ the expert's offset in its region) that the prefix-sum launch left
+        stage_ids(p, t0, t1, ids_sm, tid, kThreads);
+        for (int i = tid; i < ntok * k; i += kThreads) w_sm[i] = __ldg(p.topk_w + (size_t)t0 * k + i);
+        __syncthreads();
+        build_bin_maps(p, ids_sm, ntok, bmaps, warp, kWarps, lane);
+        int* base_sm = hist;
+        for (int b = tid; b < p.B; b += kThreads)
+            base_sm[b] = __ldcg(p.chunk_base + (size_t)b * p.nchunks + gch) + (b < p.E ? __ldcg(p.expert_offset + b) : 0);
+        __syncthreads();
+        finalize_chunk<true>(p, t0, t1, ids_sm, w_sm,
+                             [&](int e, int tl) { return base_sm[e] + bits_in_range(bmaps, e, 0, tl); },
+                             [&](int r, int tl) { return base_sm[p.E + r] + bits_in_range(bmaps, p.E + r, 0, tl); },
+                             true, c, order_sm, pos, key, sent, tid, kThreads, delta);
+        __syncthreads();
+        if (c == 0 && tid == 0) {
+            const int n_mine = __ldcg(p.num_rows_per_rank + p.my_rank);
+            atomicAdd(p.shard_arrival + 1, (unsigned)(n_mine < p.cap ? n_mine : p.cap));
+        }
     }
-    for (int s = c; s < p.S; s += p.grid) write_source_from_maps(p, s, bmaps, eo, tid, kThreads);
 
     // ---- sender: one token at a time, all threads on its row, one store per copy and vector
     const int nvec = p.H / 8;   // 16-byte vectors of the bf16 input row
@@ -165,11 +195,12 @@ __global__ void __launch_bounds__(256) sharded_combine_kernel(const uint16_t* co
 
 int sharded_extra_smem(const Params& p) { return p.R * 12 + 128; }
 
-cudaError_t launch_sharded_dispatch(const Params& p, const SmemPlan& pl, cudaStream_t st) {
+cudaError_t launch_sharded_dispatch(const Params& p, const SmemPlan& pl, bool whole_table, cudaStream_t st) {
     const int smem = pl.total + sharded_extra_smem(p);
-    cudaError_t e = cudaFuncSetAttribute(sharded_dispatch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    auto kern = whole_table ? sharded_dispatch_kernel<true> : sharded_dispatch_kernel<false>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    sharded_dispatch_kernel<<<p.grid, kThreads, smem, st>>>(p, pl);
+    kern<<<p.grid, kThreads, smem, st>>>(p, pl);
     return cudaGetLastError();
 }
 

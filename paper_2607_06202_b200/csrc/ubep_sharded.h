@@ -10,7 +10,9 @@ namespace ubep {
 // Dynamic shared memory the sharded dispatch kernel needs beyond the dispatch plan's total.
 int sharded_extra_smem(const Params& p);
 
-cudaError_t launch_sharded_dispatch(const Params& p, const SmemPlan& pl, cudaStream_t st);
+// whole_table: every CTA derives the layout from the whole routing table in shared memory; otherwise the
+// count / prefix-sum launches (launch_count_scan) have run before with p.nchunks = R * p.grid chunks.
+cudaError_t launch_sharded_dispatch(const Params& p, const SmemPlan& pl, bool whole_table, cudaStream_t st);
 
 // One CTA: waits until arrival[0] (rows announced) equals arrival[1] (rows expected).
 cudaError_t launch_wait_arrivals(const unsigned* arrival, int32_t* status, cudaStream_t st);

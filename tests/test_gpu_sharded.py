@@ -25,6 +25,12 @@ CASES = {
     "replicas": W.Config("replicas", T=96, H=512, E=36, R=4, k=4, seed=5105, E_logical=32),
     "fp8": W.Config("fp8", T=96, H=384, E=16, R=4, k=4, payload=1, seed=5106),
     "fp8_dedup": W.Config("fp8_dedup", T=70, H=1024, E=32, R=8, k=4, payload=1, dedup=1, seed=5107),
+    # routing tables too large to recount in every CTA (T * k > 8192): counts and prefix sums by launches of
+    # their own over the whole table, chunks aligned with the ranks' token ranges
+    "large": W.Config("large", T=1203, H=512, E=64, R=8, k=8, seed=5108),
+    "large_dedup": W.Config("large_dedup", T=2500, H=256, E=48, R=6, k=4, dedup=1, seed=5109),
+    "large_fp8_replicas": W.Config("large_fp8", T=1500, H=384, E=36, R=4, k=6, payload=1, seed=5110, E_logical=32),
+    "prefill_sized": W.Config("prefill_sized", T=4096, H=1024, E=256, R=8, k=8, seed=5111),
 }
 
 
