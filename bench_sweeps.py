@@ -151,14 +151,14 @@ def measure(cfg: W.Config, iters: int, warmup: int = 20):
     x = torch.from_numpy(wl.x).view(torch.bfloat16).to(dev)
     w = torch.from_numpy(wl.topk_w.astype(np.float32)).to(dev)
     probe = B.Buffer(num_ranks=cfg.R, num_experts=cfg.E, hidden=cfg.H, topk=cfg.k, max_tokens=cfg.T,
-                     rows_per_rank_cap=1, dedup=cfg.dedup)
+                     rows_per_rank_cap=1, dedup=cfg.dedup, payload=cfg.payload)
     npr, npe, _ = probe.get_dispatch_layout(idx)
     rows_per_rank = npr if cfg.dedup else npe.view(cfg.R, cfg.L).sum(1)
     cap = W.round_up(max(1, int(rows_per_rank.max().item())), 16)
     n_rows = int(rows_per_rank.sum().item())
     probe.close()
     buf = B.Buffer(num_ranks=cfg.R, num_experts=cfg.E, hidden=cfg.H, topk=cfg.k, max_tokens=cfg.T,
-                   rows_per_rank_cap=cap, dedup=cfg.dedup)
+                   rows_per_rank_cap=cap, dedup=cfg.dedup, payload=cfg.payload)
     views = buf.attach_sync()
     out = {}
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -186,7 +186,7 @@ def measure(cfg: W.Config, iters: int, warmup: int = 20):
             rec["layout_us"] = (int(t[:, 1].max()) - t_first) / 1e3
             rec["sent_us"] = (int(t[:, 2].max()) - t_first) / 1e3
             rec["ready_us"] = (int(t[:, 3].max()) - t_first) / 1e3
-            rec["wire_ratio"] = wire_ratio(proto, 2 * cfg.H)
+            rec["wire_ratio"] = wire_ratio(proto, cfg.H + 4 * (cfg.H // 128) if cfg.payload else 2 * cfg.H)
         out[proto] = rec
     buf.close()
     return out, n_rows
@@ -199,15 +199,18 @@ def main_sync(argv):
     ap.add_argument("--iters", type=int, default=200)
     ap.add_argument("--hidden", type=int, nargs="*", default=[256, 1024, 4096, 7168])
     ap.add_argument("--ranks", type=int, nargs="*", default=[8, 32, 128])
+    ap.add_argument("--payload", type=int, default=0, choices=[0, 1], help="1 = FP8 rows (payload + scales on the wire)")
     ap.add_argument("--markdown", action="store_true")
     args = ap.parse_args(argv)
     B.load()
     rows = []
     for R in args.ranks:
         for H in args.hidden:
-            cfg = W.Config(f"sync_T{args.tokens}_H{H}_R{R}", T=args.tokens, H=H, E=256, R=R, k=8, seed=7000 + R + H)
+            cfg = W.Config(f"sync_T{args.tokens}_H{H}_R{R}", T=args.tokens, H=H, E=256, R=R, k=8, payload=args.payload,
+                           seed=7000 + R + H)
             res, n_rows = measure(cfg, args.iters)
-            rows.append({"tokens": args.tokens, "row_bytes": 2 * H, "ranks": R, "rows": n_rows, **res})
+            row_bytes = H + 4 * (H // 128) if args.payload else 2 * H
+            rows.append({"tokens": args.tokens, "row_bytes": row_bytes, "ranks": R, "rows": n_rows, **res})
     if not args.markdown:
         for r in rows:
             print(json.dumps(r))

@@ -278,7 +278,12 @@ int ubep_map_workers(const int32_t *order /*[dev]*/, const int32_t *counts /*[de
  * promises for vector accesses.  All waits are bounded (about 1.5 s); a wait that runs out
  * records UBEP_ERR_TIMEOUT and the kernel returns.
  *
- * Limits: bf16 payload only; T * k <= 8192 and the routing table with the bitmaps of all its
+ * FP8 rows (UBEP_PAYLOAD_FP8_E4M3) travel quantised: the sender quantises a row once, and a wire row is
+ * the H payload bytes followed by the 4 * H / 128 bytes of its scales (the W8A8 rows of the paper's
+ * Table 3); Token-Flag blocks and Sentinel blocks are cut from that, the checksum markers from the
+ * payload.  What arrives goes to the region's payload and scale arrays.
+ *
+ * Limits: T * k <= 8192 and the routing table with the bitmaps of all its
  * bins (T x (E + R) bits) must fit in a CTA's shared memory, since every CTA derives the layout
  * from the whole table, as UBEP_PIPELINE_LOCAL does; one CTA per SM at most, launched
  * cooperatively (receivers wait for senders of the same grid, so the grid must be resident at once:
@@ -295,8 +300,9 @@ enum { UBEP_SYNC_SW = 0, UBEP_SYNC_TFF = 1, UBEP_SYNC_DC = 2, UBEP_SYNC_SP = 3 }
 
 /* Arrays of the wire buffer (ubep_sync_view). */
 enum {
-    UBEP_SYNC_VIEW_TFF_WIRE = 0, /* u8  [R, cap, 16 * ceil(2H / 12)]  DataBlocks of every row     */
-    UBEP_SYNC_VIEW_SP_WIRE = 1,  /* u8  [R, cap, 2H]  all sentinel between calls                  */
+    UBEP_SYNC_VIEW_TFF_WIRE = 0, /* u8  [R, cap, 16 * ceil(W / 12)]  DataBlocks of every row; W = 2H, */
+                                 /*     or H + 4 * H / 128 for FP8 rows                           */
+    UBEP_SYNC_VIEW_SP_WIRE = 1,  /* u8  [R, cap, W rounded up to 16]  all sentinel between calls  */
     UBEP_SYNC_VIEW_CHECKSUM = 2, /* u64 [2, R]  DC: marker sums announced (half = call number & 1)*/
     UBEP_SYNC_VIEW_COUNTERS = 3, /* u32 [4, R]  DC announcements [2, R], then SW row counts [2, R]*/
     UBEP_SYNC_VIEW_TIMES = 4,    /* u64 [CTAs, 8]  device nanosecond timer of the last call, per CTA:
@@ -306,7 +312,7 @@ enum {
     UBEP_SYNC_VIEW_COUNT_
 };
 
-/* Bytes of the wire buffer for this configuration (0 if it is invalid or not bf16). */
+/* Bytes of the wire buffer for this configuration (0 if it is invalid). */
 size_t ubep_sync_wire_bytes(const ubep_config_t *cfg /*[host]*/);
 
 /*
@@ -321,8 +327,7 @@ int ubep_sync_attach(ubep_buffer_t *buf, void *dev_wire /*[dev]*/, size_t bytes,
  * One kernel launch (a memset before it when an earlier call left the SP wire dirty, which
  * the library learns when ubep_status reports that call's error; until then a word on the
  * device makes every Sentinel Polling call on that wire report UBEP_ERR_TIMEOUT and move nothing).  UBEP_ERR_ARG if no wire
- * buffer is attached, the payload is not bf16, T * k > 8192 or the table does not fit in shared
- * memory.
+ * buffer is attached, T * k > 8192 or the table does not fit in shared memory.
  */
 int ubep_dispatch_sync(ubep_buffer_t *buf, int protocol, const void *x /*[dev]*/,
                        const int32_t *topk_idx /*[dev]*/, const float *topk_w /*[dev]*/, int32_t T,

@@ -116,18 +116,21 @@ ArenaLayout make_layout(const ubep_config_t& c, int nchunks) {
 struct WireLayout {
     size_t off[UBEP_SYNC_VIEW_COUNT_];
     size_t flags_begin, sp_dirty, seq_ticket, scan_count, flags_end, total;
-    int tff_blocks;
+    int tff_blocks, sp_row;
 };
 
 WireLayout make_wire_layout(const ubep_config_t& c, int nchunks) {
     WireLayout w{};
-    const size_t R = c.num_ranks, cap = c.rows_per_rank_cap, rowB = 2 * (size_t)c.hidden;
+    // bytes of one row on the wire: the bf16 row, or the e4m3 payload followed by its fp32 scales
+    const size_t R = c.num_ranks, cap = c.rows_per_rank_cap;
+    const size_t rowB = c.payload ? (size_t)c.hidden + 4 * (size_t)(c.hidden / 128) : 2 * (size_t)c.hidden;
     const int payload = UBEP_SYNC_BLOCK_BYTES - UBEP_SYNC_FLAG_BYTES;
     w.tff_blocks = (int)((rowB + payload - 1) / payload);
+    w.sp_row = (int)((rowB + UBEP_SYNC_BLOCK_BYTES - 1) / UBEP_SYNC_BLOCK_BYTES * UBEP_SYNC_BLOCK_BYTES);
     size_t at = 0;
     auto take = [&](size_t bytes) { size_t o = at; at = align_up(at + bytes); return o; };
     w.off[UBEP_SYNC_VIEW_TFF_WIRE] = take(R * cap * (size_t)w.tff_blocks * UBEP_SYNC_BLOCK_BYTES);
-    w.off[UBEP_SYNC_VIEW_SP_WIRE] = take(R * cap * rowB);
+    w.off[UBEP_SYNC_VIEW_SP_WIRE] = take(R * cap * (size_t)w.sp_row);
     w.flags_begin = at;
     w.off[UBEP_SYNC_VIEW_CHECKSUM] = take(2 * R * 8);
     w.off[UBEP_SYNC_VIEW_COUNTERS] = take(4 * R * 4);
@@ -465,12 +468,12 @@ int ubep_combine(ubep_buffer_t* buf, const void* y, const float* topk_w, int32_t
 }
 
 size_t ubep_sync_wire_bytes(const ubep_config_t* cfg) {
-    if (!cfg || !valid_config(*cfg) || cfg->payload != UBEP_PAYLOAD_BF16) return 0;
+    if (!cfg || !valid_config(*cfg)) return 0;
     return make_wire_layout(*cfg, cfg->num_ctas).total;
 }
 
 int ubep_sync_attach(ubep_buffer_t* buf, void* dev_wire, size_t bytes, void* cuda_stream) {
-    if (!buf || !dev_wire || buf->cfg.payload != UBEP_PAYLOAD_BF16) return UBEP_ERR_ARG;
+    if (!buf || !dev_wire) return UBEP_ERR_ARG;
     if ((reinterpret_cast<uintptr_t>(dev_wire) & (kAlign - 1)) != 0) return UBEP_ERR_ARENA;
     if (bytes < make_wire_layout(buf->cfg, buf->cfg.num_ctas).total) return UBEP_ERR_ARENA;
     DeviceGuard guard(buf->cfg.device);
@@ -555,7 +558,7 @@ int ubep_sync_view(ubep_buffer_t* buf, int which, void** dev_ptr, int64_t shape[
         case UBEP_SYNC_VIEW_TFF_WIRE:
             s[0] = c.num_ranks; s[1] = c.rows_per_rank_cap; s[2] = (int64_t)buf->wlay.tff_blocks * UBEP_SYNC_BLOCK_BYTES;
             break;
-        case UBEP_SYNC_VIEW_SP_WIRE: s[0] = c.num_ranks; s[1] = c.rows_per_rank_cap; s[2] = 2 * (int64_t)c.hidden; break;
+        case UBEP_SYNC_VIEW_SP_WIRE: s[0] = c.num_ranks; s[1] = c.rows_per_rank_cap; s[2] = buf->wlay.sp_row; break;
         case UBEP_SYNC_VIEW_CHECKSUM: s[0] = 2; s[1] = c.num_ranks; break;
         case UBEP_SYNC_VIEW_COUNTERS: s[0] = 4; s[1] = c.num_ranks; break;
         case UBEP_SYNC_VIEW_TIMES: s[0] = buf->lay.nchunks; s[1] = ubep::kSyncTimeSlots; break;

@@ -12,6 +12,7 @@
 //
 // A DataBlock is the 16 bytes one thread stores with a single 128-bit access.
 #include "ubep_layout.cuh"
+#include "ubep_quant.cuh"
 #include "ubep_sync.h"
 
 namespace ubep {
@@ -91,7 +92,11 @@ __device__ __forceinline__ bool wait_count(const unsigned* ctr, unsigned want, W
     return true;
 }
 
-template <int kProto>
+// kFp8: rows travel quantised (e4m3 payload, then the fp32 scales of the row's 128-channel groups, as one
+// wire row of H + 4 * H / 128 bytes); the sender quantises a row once into shared memory and sends from
+// there; what arrives goes to the payload and the scale array of the receive region.  The checksum
+// markers of Data-for-Checksum are taken from the payload bytes.
+template <int kProto, bool kFp8>
 __global__ void __launch_bounds__(kThreads, 1) sync_dispatch_kernel(const Params p, const SmemPlan pl,
                                                                    const SyncParams sp) {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -111,6 +116,7 @@ __global__ void __launch_bounds__(kThreads, 1) sync_dispatch_kernel(const Params
     int* nrows = reinterpret_cast<int*>(smem + pl.off_arr);     // rows every region receives
     int* order_sm = reinterpret_cast<int*>(smem + pl.off_order);
     unsigned long long* chk_sm = reinterpret_cast<unsigned long long*>(smem + pl.total);   // DC: [R]
+    uint8_t* qrow = smem + pl.total + (((size_t)p.R * 8 + 15) & ~(size_t)15);              // FP8: the quantised row
     const BinMaps bmaps{reinterpret_cast<unsigned*>(smem + pl.off_mask), reinterpret_cast<unsigned*>(smem + pl.off_bm),
                         pl.map_wb, pl.map_bp, pl.map_groups};
     const int t0 = (int)chunk_begin(c, p.T, p.nchunks), t1 = (int)chunk_begin(c + 1, p.T, p.nchunks);
@@ -155,39 +161,71 @@ __global__ void __launch_bounds__(kThreads, 1) sync_dispatch_kernel(const Params
     for (int s = c; s < p.S; s += p.grid) write_source_from_maps(p, s, bmaps, eo, tid, kThreads);
 
     // ---- sender: the rows of tokens [t0, t1), one token at a time, all threads on a row
-    const int nvec = p.rowB / 16;
-    const int nwords = p.rowB / 4;
+    const int wbytes = kFp8 ? p.H + 4 * p.G : p.rowB;   // bytes of one row on the wire
+    const int nvec = (wbytes + 15) / 16;                // its 16-byte blocks (FP8: the last may be cut short)
+    const int pvec = p.rowB / 16;                       // blocks of the payload (all of them for bf16 rows)
+    const int nwords = wbytes / 4;
+    const int pwords = p.rowB / 4;
     const size_t wire_row = (size_t)sp.tff_blocks * 16;
+    const size_t sp_row = (size_t)nvec * 16;
     const bool wire_unusable = kProto == kSP && abort_flag != 0;   // (set before the barriers above, uniform in the CTA)
+    // word w of the wire row of global row `where` lands in the payload or, beyond it, in the scales
+    auto put_word = [&](size_t where, int w, uint32_t val) {
+        if (!kFp8 || w < pwords) reinterpret_cast<uint32_t*>(p.recv_x + where * p.rowB)[w] = val;
+        else reinterpret_cast<uint32_t*>(p.recv_scale + where * p.G)[w - pwords] = val;
+    };
     for (int tl = 0; tl < ntok && !wire_unusable; ++tl) {
         const int* ps = pos + tl * k;
+        const uint4* xrow = reinterpret_cast<const uint4*>(p.x + (size_t)(t0 + tl) * p.H);
+        if (kFp8) {
+            // quantise the row once (every copy carries the same bytes)
+            const int xvec = p.H / 8;
+            for (int v0 = 0; v0 < xvec; v0 += kThreads) {   // same trip count for every thread (the quantiser shuffles)
+                const int v = v0 + tid;
+                const bool in = v < xvec;
+                const uint4 d = in ? __ldg(xrow + v) : make_uint4(0, 0, 0, 0);
+                uint2 q;
+                float scale;
+                quantize8(d, in, q, scale);
+                if (in) {
+                    *reinterpret_cast<uint2*>(qrow + (size_t)v * 8) = q;
+                    if ((v & 15) == 0) reinterpret_cast<float*>(qrow + p.H)[v >> 4] = scale;
+                }
+            }
+            for (int w = nwords + tid; w < nvec * 4; w += kThreads) reinterpret_cast<uint32_t*>(qrow)[w] = 0u;   // padding
+            __syncthreads();
+        }
         if (kProto == kTFF) {
-            const uint32_t* xw = reinterpret_cast<const uint32_t*>(p.x + (size_t)(t0 + tl) * p.H);
+            const uint32_t* xw = kFp8 ? reinterpret_cast<const uint32_t*>(qrow) : reinterpret_cast<const uint32_t*>(xrow);
             for (int g = tid; g < sp.tff_blocks; g += kThreads) {
                 const int w0 = 3 * g;
                 uint4 blk;
                 blk.x = seq;   // the flag leads the block
-                blk.y = w0 < nwords ? __ldg(xw + w0) : 0u;
-                blk.z = w0 + 1 < nwords ? __ldg(xw + w0 + 1) : 0u;
-                blk.w = w0 + 2 < nwords ? __ldg(xw + w0 + 2) : 0u;
+                blk.y = w0 < nwords ? (kFp8 ? xw[w0] : __ldg(xw + w0)) : 0u;
+                blk.z = w0 + 1 < nwords ? (kFp8 ? xw[w0 + 1] : __ldg(xw + w0 + 1)) : 0u;
+                blk.w = w0 + 2 < nwords ? (kFp8 ? xw[w0 + 2] : __ldg(xw + w0 + 2)) : 0u;
                 for (int j = 0; j < k; ++j) {
                     const int where = ps[j];
                     if (where >= 0) st_relaxed_v4(sp.tff_wire + (size_t)where * wire_row + (size_t)g * 16, blk);
                 }
             }
         } else {
-            const uint4* src = reinterpret_cast<const uint4*>(p.x + (size_t)(t0 + tl) * p.H);
-            uint8_t* dst = kProto == kSP ? sp.sp_wire : p.recv_x;
             unsigned long long mine = 0ull;
             for (int v = tid; v < nvec; v += kThreads) {
-                const uint4 d = __ldg(src + v);
-                if (kProto == kDC && (v % kDcBlockVecs) < kDcMarkerVecs) mine += marker_words(d);
+                const uint4 d = kFp8 ? reinterpret_cast<const uint4*>(qrow)[v] : __ldg(xrow + v);
+                if (kProto == kDC && v < pvec && (v % kDcBlockVecs) < kDcMarkerVecs) mine += marker_words(d);
                 for (int j = 0; j < k; ++j) {
                     const int where = ps[j];
                     if (where < 0) continue;
-                    uint8_t* at = dst + (size_t)where * p.rowB + (size_t)v * 16;
-                    if (kProto == kSP) st_relaxed_v4(at, d);
-                    else *reinterpret_cast<uint4*>(at) = d;
+                    if (kProto == kSP) {
+                        st_relaxed_v4(sp.sp_wire + (size_t)where * sp_row + (size_t)v * 16, d);
+                    } else if (!kFp8 || v < pvec) {
+                        *reinterpret_cast<uint4*>(p.recv_x + (size_t)where * p.rowB + (size_t)v * 16) = d;
+                    } else {
+                        const uint32_t dw[4] = {d.x, d.y, d.z, d.w};
+                        for (int i = 0; i < 4; ++i)
+                            if (4 * v + i < nwords) put_word((size_t)where, 4 * v + i, dw[i]);
+                    }
                 }
             }
             if (kProto == kDC) {
@@ -209,6 +247,7 @@ __global__ void __launch_bounds__(kThreads, 1) sync_dispatch_kernel(const Params
                 if (tid < k && ps[tid] >= 0) red_release_add(sp.sw_rows + par * R + ps[tid] / p.cap, 1u);
             }
         }
+        if (kFp8) __syncthreads();   // the quantised row is reused for the next token
     }
     if (kProto == kDC) {
         // one fence per sender and batch, then the checksum packet of every region
@@ -236,9 +275,9 @@ __global__ void __launch_bounds__(kThreads, 1) sync_dispatch_kernel(const Params
             // is polled on its own).
             constexpr int kBatch = 4;
             const int per_row = kProto == kTFF ? sp.tff_blocks : nvec;
-            const size_t row_stride = kProto == kTFF ? wire_row : (size_t)p.rowB;
+            const size_t row_stride = kProto == kTFF ? wire_row : sp_row;
             uint8_t* const wire = (kProto == kTFF ? sp.tff_wire : sp.sp_wire) + ((size_t)r * p.cap + lo) * row_stride;
-            uint8_t* const region = p.recv_x + ((size_t)r * p.cap + lo) * p.rowB;
+            const size_t row0 = (size_t)r * p.cap + lo;   // global row of the slice's first row
             const int items = (hi - lo) * per_row;
             const uint4 sentinel = make_uint4(0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu);
             bool ok = true;
@@ -262,14 +301,20 @@ __global__ void __launch_bounds__(kThreads, 1) sync_dispatch_kernel(const Params
                         blk[b] = ld_relaxed_v4(src);
                     }
                     if (!ok) break;
+                    const size_t grow = row0 + row[b];
                     if (kProto == kTFF) {
-                        uint32_t* out = reinterpret_cast<uint32_t*>(region + (size_t)row[b] * p.rowB);
                         const int w0 = 3 * g[b];
-                        if (w0 < nwords) out[w0] = blk[b].y;
-                        if (w0 + 1 < nwords) out[w0 + 1] = blk[b].z;
-                        if (w0 + 2 < nwords) out[w0 + 2] = blk[b].w;
+                        if (w0 < nwords) put_word(grow, w0, blk[b].y);
+                        if (w0 + 1 < nwords) put_word(grow, w0 + 1, blk[b].z);
+                        if (w0 + 2 < nwords) put_word(grow, w0 + 2, blk[b].w);
                     } else {
-                        *reinterpret_cast<uint4*>(region + (size_t)row[b] * p.rowB + (size_t)g[b] * 16) = blk[b];
+                        if (!kFp8 || g[b] < pvec) {
+                            *reinterpret_cast<uint4*>(p.recv_x + grow * p.rowB + (size_t)g[b] * 16) = blk[b];
+                        } else {
+                            const uint32_t dw[4] = {blk[b].x, blk[b].y, blk[b].z, blk[b].w};
+                            for (int i = 0; i < 4; ++i)
+                                if (4 * g[b] + i < nwords) put_word(grow, 4 * g[b] + i, dw[i]);
+                        }
                         st_relaxed_v4(src, sentinel);   // consumed: ready for the next call
                     }
                 }
@@ -282,13 +327,13 @@ __global__ void __launch_bounds__(kThreads, 1) sync_dispatch_kernel(const Params
                 if (tid == 0) (void)wait_count(sp.announced + par * R + r, (unsigned)p.grid, wt);
                 __syncthreads();
                 if (!abort_flag) {
-                    const int nblk = (nvec + kDcBlockVecs - 1) / kDcBlockVecs;
+                    const int nblk = (pvec + kDcBlockVecs - 1) / kDcBlockVecs;
                     const int per_row = nblk * kDcMarkerVecs;
                     unsigned long long mine = 0ull;
                     for (int i = tid; i < n_r * per_row; i += kThreads) {
                         const int row = i / per_row, rem = i - row * per_row;
                         const int v = (rem / kDcMarkerVecs) * kDcBlockVecs + rem % kDcMarkerVecs;
-                        if (v < nvec)
+                        if (v < pvec)
                             mine += marker_words(__ldcg(
                                 reinterpret_cast<const uint4*>(p.recv_x + ((size_t)r * p.cap + row) * p.rowB) + v));
                     }
@@ -329,7 +374,7 @@ __global__ void __launch_bounds__(256) sentinel_scan_kernel(const uint4* __restr
 
 template <int kProto>
 cudaError_t launch_one(const Params& p, const SmemPlan& pl, const SyncParams& sp, cudaStream_t st) {
-    auto kern = sync_dispatch_kernel<kProto>;
+    auto kern = p.payload ? sync_dispatch_kernel<kProto, true> : sync_dispatch_kernel<kProto, false>;
     const int smem = pl.total + sync_extra_smem(p);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
@@ -350,7 +395,10 @@ cudaError_t launch_one(const Params& p, const SmemPlan& pl, const SyncParams& sp
 
 }  // namespace
 
-int sync_extra_smem(const Params& p) { return p.R * 8 + 128; }
+int sync_extra_smem(const Params& p) {
+    const int qrow = p.payload ? ((p.H + 4 * p.G + 15) / 16) * 16 : 0;   // FP8: the quantised row of the token being sent
+    return p.R * 8 + 128 + qrow + 16;
+}
 
 cudaError_t launch_sync_dispatch(const Params& p, const SmemPlan& pl, const SyncParams& sp, cudaStream_t st) {
     switch (sp.protocol) {

@@ -95,7 +95,10 @@ def test_wire_bytes_of_the_readiness_protocols(lib):
     tff_row = 16 * -(-14336 // 12)
     n = B.ubep_sync_wire_bytes(_cfg(**kw))
     assert rows * (tff_row + 14336) < n < rows * (tff_row + 14336) * 1.01
-    assert B.ubep_sync_wire_bytes(_cfg(payload=1)) == 0            # bf16 rows only
+    # FP8 rows: payload plus scales, 7168 + 224 bytes
+    n8 = B.ubep_sync_wire_bytes(_cfg(payload=1, **kw))
+    w8 = 7168 + 224
+    assert rows * (16 * -(-w8 // 12) + w8) < n8 < rows * (16 * -(-w8 // 12) + w8) * 1.01
     assert B.ubep_sync_wire_bytes(_cfg(num_experts=18)) == 0
     assert (B.UBEP_SYNC_BLOCK_BYTES - B.UBEP_SYNC_FLAG_BYTES) / B.UBEP_SYNC_BLOCK_BYTES == 0.75
     header = open(os.path.join(ROOT, "include", "ubep.h")).read()

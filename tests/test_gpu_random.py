@@ -41,7 +41,7 @@ def test_random_cases(seed):
     for _ in range(8):
         cfg, wl, pipeline, ctas, order = draw(rng)
         Hn.run_case(wl, pipeline=pipeline, num_ctas=ctas, dest_order=order)
-        if cfg.payload or cfg.T * cfg.k > 8192:
+        if cfg.T * cfg.k > 8192:
             continue
         ids, lay, cap, recv = Hn.oracle_reference(wl)
         x, idx, w, _, _ = Hn.device_inputs(wl)

@@ -26,7 +26,22 @@ CASES = {
     "padded_dedup": W.Config("padded_dedup", T=61, H=2056, E=24, R=6, k=4, dedup=1, seed=4102),
     "one_rank": W.Config("one_rank", T=19, H=64, E=4, R=1, k=2, seed=4103),
     "replicas": W.Config("replicas", T=96, H=512, E=36, R=4, k=4, seed=4104, E_logical=32),
+    # FP8 rows: a wire row is the e4m3 payload followed by its fp32 scales.  396 bytes: 33 Token-Flag
+    # blocks, the 25th Sentinel block cut short after 12 bytes
+    "fp8_ragged": W.Config("fp8_ragged", T=96, H=384, E=16, R=4, k=4, payload=1, seed=4105),
+    "fp8_dedup": W.Config("fp8_dedup", T=70, H=1024, E=32, R=8, k=4, payload=1, dedup=1, seed=4106),
+    # the W8A8 row of the paper's Table 3: hidden 7168, 256 experts, top-8
+    "fp8_w8a8": W.Config("fp8_w8a8", T=64, H=7168, E=256, R=32, k=8, payload=1, seed=4107),
 }
+
+
+def wire_rows(cfg, recv, r, n):
+    """The first n rows of region r as they travel: bf16 rows as they are, FP8 rows as payload bytes
+    followed by the bytes of their scales."""
+    rows = recv.recv_x[r, :n].reshape(n, -1)
+    if cfg.payload:
+        rows = np.concatenate([rows, recv.recv_scale[r, :n].reshape(n, -1).view(np.uint8)], axis=1)
+    return np.ascontiguousarray(rows)
 
 
 def wire_checks(buf, proto, cfg, lay, recv, grid):
@@ -40,12 +55,13 @@ def wire_checks(buf, proto, cfg, lay, recv, grid):
     if proto == "tff":
         wire = v["tff_wire"].cpu().numpy()
         for r in range(cfg.R):
+            sent = wire_rows(cfg, recv, r, int(n_rows[r]))
             for row in range(int(n_rows[r])):
-                want = oracle.tff_pack(recv.recv_x[r, row], B.UBEP_SYNC_BLOCK_BYTES, B.UBEP_SYNC_FLAG_BYTES, seq)
+                want = oracle.tff_pack(sent[row], B.UBEP_SYNC_BLOCK_BYTES, B.UBEP_SYNC_FLAG_BYTES, seq)
                 assert np.array_equal(wire[r, row], want.reshape(-1)), f"DataBlocks of region {r} row {row}"
-                back, missing = oracle.tff_unpack(wire[r, row], 2 * cfg.H, B.UBEP_SYNC_BLOCK_BYTES,
+                back, missing = oracle.tff_unpack(wire[r, row], sent.shape[1], B.UBEP_SYNC_BLOCK_BYTES,
                                                   B.UBEP_SYNC_FLAG_BYTES, seq)
-                assert missing == 0 and np.array_equal(back, recv.recv_x[r, row])
+                assert missing == 0 and np.array_equal(back, sent[row])
     elif proto == "dc":
         sums = v["checksum"].cpu().numpy().view(np.uint64)[half]
         for r in range(cfg.R):
@@ -56,7 +72,9 @@ def wire_checks(buf, proto, cfg, lay, recv, grid):
     elif proto == "sp":
         wire = v["sp_wire"]
         assert bool((wire == 0xFF).all()), "consumed blocks must show the sentinel again"
-        assert oracle.sp_pending(wire[0, :2].cpu().numpy(), 16, 16, B.UBEP_SYNC_SENTINEL) == 2 * (2 * cfg.H // 16)
+        row_w = cfg.H + 4 * (cfg.H // 128) if cfg.payload else 2 * cfg.H
+        assert wire.shape[2] == -(-row_w // 16) * 16
+        assert oracle.sp_pending(wire[0, :2].cpu().numpy(), 16, 16, B.UBEP_SYNC_SENTINEL) == 2 * (wire.shape[2] // 16)
     else:
         assert np.array_equal(v["counters"].cpu().numpy()[2 + half], n_rows), "one count per fenced row"
 
@@ -84,8 +102,14 @@ def test_protocols_match_oracle(case, proto):
     if phys2 is not None:
         buf.set_replicas(phys2, ncopies2)      # the other seed drew another replica table
     buf.recv_x.fill_(Hn.FILL)
+    if cfg.payload:
+        buf.recv_scale.view(torch.uint8).fill_(Hn.FILL)
     buf.dispatch_sync(proto, x2, idx2, w2)
     Hn.check_dispatch(buf, wl2, lay2, cap, recv2, check_tails=False, arrival=False)
+    if cfg.payload:       # (with tails unchecked the harness leaves the scales out: compare the rows that exist)
+        for r in range(cfg.R):
+            n = int(lay2.num_rows_per_rank[r])
+            Hn._eq(f"recv_scale[{r}]", buf.recv_scale[r, :n].view(torch.int32), recv2.recv_scale[r, :n].view(np.int32))
     wire_checks(buf, proto, cfg, lay2, recv2, grid)
     # combine runs on what the protocol dispatch left
     y_bits = W.make_expert_outputs(cfg, cap)
@@ -208,7 +232,7 @@ def test_argument_errors():
     assert e.value.code == B.UBEP_ERR_ARG
     fp8 = dataclasses.replace(W.CONFIGS["tiny"], payload=1, H=256)
     fbuf = Hn.make_buffer(fp8, cap)
-    assert B.ubep_sync_wire_bytes(fbuf.cfg) == 0
+    assert 0 < B.ubep_sync_wire_bytes(fbuf.cfg) < B.ubep_sync_wire_bytes(buf.cfg)   # FP8 rows are shorter on the wire
     # T == 0 leaves zero counts like the main dispatch
     buf.dispatch_sync("dc", x[:0], idx[:0], w[:0])
     assert int(buf.num_rows_per_rank.sum()) == 0 and buf.status() == 0
