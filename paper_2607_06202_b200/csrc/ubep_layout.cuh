@@ -14,16 +14,28 @@ namespace ubep {
 
 // Physical expert of slot (t, j): logical id -> phys[l][t mod ncopies[l]] when a replica
 // table is set.  -1 for an empty slot; ids out of range are reported and treated as empty.
-__device__ __forceinline__ int resolve_expert(const Params& p, int t, int raw) {
+// v / L for 0 <= v < 65536, with magic = ceil(2^32 / L)
+__device__ __forceinline__ int fast_div(int v, unsigned magic) { return (int)__umulhi((unsigned)v, magic); }
+
+// `bad` is set instead of reporting on the spot: a call to the out-of-line report() inside an unrolled loop,
+// taken or not, was measured to cost about 125 cycles per slot (the staging of a 512-token table: 1865
+// cycles per warp with the calls, 840 without).  The caller reports once, after its loop.
+__device__ __forceinline__ int resolve_expert(const Params& p, int t, int raw, bool& bad) {
     if (raw == -1) return -1;
     int e = raw;
     if (p.phys != nullptr) {
-        if (raw < 0 || raw >= p.E_log) { report(p.status, kErrBadIndex); return -1; }
+        if (raw < 0 || raw >= p.E_log) { bad = true; return -1; }
         int nc = __ldg(p.ncopies + raw);
-        if (nc < 1 || nc > p.C) { report(p.status, kErrBadIndex); return -1; }
+        if (nc < 1 || nc > p.C) { bad = true; return -1; }
         e = __ldg(p.phys + (size_t)raw * p.C + (t % nc));
     }
-    if (e < 0 || e >= p.E) { report(p.status, kErrBadIndex); return -1; }
+    if (e < 0 || e >= p.E) { bad = true; return -1; }
+    return e;
+}
+__device__ __forceinline__ int resolve_expert(const Params& p, int t, int raw) {
+    bool bad = false;
+    const int e = resolve_expert(p, t, raw, bad);
+    if (bad) report(p.status, kErrBadIndex);
     return e;
 }
 
@@ -51,13 +63,37 @@ __device__ __forceinline__ int rotated_key(const int* order_sm, int r, int worke
     return kv < 0 ? kv + R : kv;
 }
 
+// One slot of the routing table, resolved and packed (expert | rank << 16), -1 for an empty slot or a bad
+// id (`bad` is set then).  `slot` is its index in the whole table; the token it belongs to is worked out
+// only where a replica has to be picked, and nothing branches per slot without a replica table: a lone
+// warp staging four slots per thread spent 1300 cycles on the divisions and branches of the earlier form.
+__device__ __forceinline__ int pack_slot(const Params& p, size_t slot, int raw, bool& bad) {
+    int e = raw;
+    if (p.phys != nullptr) {
+        const bool in = (unsigned)e < (unsigned)p.E_log;
+        bad |= !in && e != -1;
+        const int nc = in ? __ldg(p.ncopies + e) : 1;
+        const bool okc = in && nc >= 1 && nc <= p.C;
+        bad |= in && !okc;
+        const int t = (int)((unsigned)slot / (unsigned)p.k);   // (the table has fewer than 2^31 slots)
+        e = okc ? __ldg(p.phys + (size_t)e * p.C + (t % nc)) : -1;
+        bad |= okc && e < 0;
+    }
+    const bool valid = (unsigned)e < (unsigned)p.E;
+    bad |= !valid && e != -1;
+    const int r = p.L == 1 ? e : fast_div(e, p.L_magic);
+    return valid ? (e | (r << 16)) : -1;
+}
+
 // Resolved expert ids (with their ranks) of tokens [t0, t1) into shared memory.  The raw ids
-// are gathered eight at a time before any of them is resolved, so that the loads overlap.
+// are gathered several at a time before any of them is resolved, so that the loads overlap.
 __device__ __forceinline__ void stage_ids(const Params& p, int t0, int t1, int* ids, int tid, int nthreads) {
     const int k = p.k, n = (t1 - t0) * k;
-    const int32_t* src = p.topk_idx + (size_t)t0 * k;
-    if ((((size_t)t0 * k) & 3) == 0 && (n & 3) == 0) {
-        // 16-byte loads, four of them in flight per thread
+    const size_t slot0 = (size_t)t0 * k;
+    const int32_t* src = p.topk_idx + slot0;
+    bool bad = false;
+    if ((slot0 & 3) == 0 && (n & 3) == 0) {
+        // 16-byte loads and stores, four of them in flight per thread
         const int4* src4 = reinterpret_cast<const int4*>(src);
         const int n4 = n >> 2;
         for (int i0 = tid; i0 < n4; i0 += 4 * nthreads) {
@@ -71,33 +107,29 @@ __device__ __forceinline__ void stage_ids(const Params& p, int t0, int t1, int* 
             for (int u = 0; u < 4; ++u) {
                 const int i = i0 + u * nthreads;
                 if (i < n4) {
-                    const int r4[4] = {raw[u].x, raw[u].y, raw[u].z, raw[u].w};
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const int e = resolve_expert(p, t0 + (4 * i + q) / k, r4[q]);
-                        ids[4 * i + q] = e < 0 ? -1 : (e | ((e / p.L) << 16));
-                    }
+                    const size_t s4 = slot0 + 4 * (size_t)i;
+                    *reinterpret_cast<int4*>(ids + 4 * i) =
+                        make_int4(pack_slot(p, s4, raw[u].x, bad), pack_slot(p, s4 + 1, raw[u].y, bad),
+                                  pack_slot(p, s4 + 2, raw[u].z, bad), pack_slot(p, s4 + 3, raw[u].w, bad));
                 }
             }
         }
-        return;
-    }
-    for (int i0 = tid; i0 < n; i0 += 8 * nthreads) {
-        int raw[8];
+    } else {
+        for (int i0 = tid; i0 < n; i0 += 8 * nthreads) {
+            int raw[8];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const int i = i0 + u * nthreads;
-            raw[u] = i < n ? __ldg(src + i) : -1;
-        }
+            for (int u = 0; u < 8; ++u) {
+                const int i = i0 + u * nthreads;
+                raw[u] = i < n ? __ldg(src + i) : -1;
+            }
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const int i = i0 + u * nthreads;
-            if (i < n) {
-                const int e = resolve_expert(p, t0 + i / k, raw[u]);
-                ids[i] = e < 0 ? -1 : (e | ((e / p.L) << 16));
+            for (int u = 0; u < 8; ++u) {
+                const int i = i0 + u * nthreads;
+                if (i < n) ids[i] = pack_slot(p, slot0 + i, raw[u], bad);
             }
         }
     }
+    if (bad) report(p.status, kErrBadIndex);
 }
 
 // ------------------------------------------------------------------- TokenCnt
@@ -469,7 +501,6 @@ struct RankMaps {
 };
 constexpr int kRankWords = 4;
 
-__device__ __forceinline__ int fast_div(int v, unsigned magic) { return (int)__umulhi((unsigned)v, magic); }
 
 // Stage all T*k slots (packed id | rank << 16) and build the rank bitmaps; lane = token.
 // (An expert named twice by a token does not change any rank-level row, so this step, which every
@@ -478,6 +509,7 @@ __device__ __forceinline__ int fast_div(int v, unsigned magic) { return (int)__u
 static __device__ void local_stage_and_rank_maps(const Params& p, int* ids, const RankMaps& rm, int gw, int nw, int lane) {
     const int k = p.k, T = p.T;
     const bool vec = (k & 3) == 0;   // a token's ids are whole 16-byte words (topk_idx is 16-byte aligned)
+    bool bad = false;
     for (int g = gw; g < rm.groups; g += nw) {
         const int t = g * 32 + lane;
         unsigned m[kRankWords];
@@ -496,14 +528,15 @@ static __device__ void local_stage_and_rank_maps(const Params& p, int* ids, cons
 #pragma unroll
                     for (int u = 0; u < 8; ++u) raw[u] = j0 + u < k ? __ldg(src + j0 + u) : -1;
                 }
+                int pk[8];
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
-                    if (j0 + u >= k) break;
-                    const int e = resolve_expert(p, t, raw[u]);
-                    int packed = -1;
+                    pk[u] = -1;
+                    if (j0 + u >= k) continue;
+                    const int e = resolve_expert(p, t, raw[u], bad);
                     if (e >= 0) {
                         const int r = fast_div(e, p.L_magic);
-                        packed = e | (r << 16);
+                        pk[u] = e | (r << 16);
                         if (rm.wr == 1) {
                             m[0] |= 1u << r;
                         } else {
@@ -511,13 +544,86 @@ static __device__ void local_stage_and_rank_maps(const Params& p, int* ids, cons
                             for (int w = 0; w < kRankWords; ++w) m[w] |= (w == (r >> 5)) ? 1u << (r & 31) : 0u;
                         }
                     }
-                    ids[t * k + j0 + u] = packed;
+                }
+                // (one 16-byte store per four slots: scalar stores of a lane's slots, 32 bytes apart from
+                // the next lane's, would meet in four banks)
+                if (vec) {
+                    *reinterpret_cast<int4*>(ids + (size_t)t * k + j0) = make_int4(pk[0], pk[1], pk[2], pk[3]);
+                    if (j0 + 4 < k) *reinterpret_cast<int4*>(ids + (size_t)t * k + j0 + 4) = make_int4(pk[4], pk[5], pk[6], pk[7]);
+                } else {
+#pragma unroll
+                    for (int u = 0; u < 8; ++u)
+                        if (j0 + u < k) ids[t * k + j0 + u] = pk[u];
                 }
             }
         }
 #pragma unroll
         for (int w = 0; w < kRankWords; ++w)
             if (w < rm.wr) rm.rbm[(size_t)g * rm.rp + w * 32 + lane] = transpose32(m[w], lane);
+    }
+    if (bad) report(p.status, kErrBadIndex);
+}
+
+// The rank bitmaps alone, of tokens [0, t_end) rounded up to whole groups: what the rows of a CTA whose
+// tokens end at t_end depend on.  Every CTA runs this redundantly before its first copy, and the step is
+// bound by instruction issue (16 warps, one group of 32 tokens each): measured per warp and group, warm,
+// 2380 cycles for the pass above, 900 for this one, 730 with the slot count fixed at eight.  So nothing
+// is stored per slot, nothing is reported (the pass that stages the ids reports), a bad id just sets no bit.
+template <bool kPlain, int kK>   // kPlain: no replica table and at most 32 ranks; kK: slots per token if fixed
+__device__ __forceinline__ void rank_maps_pass(const Params& p, const RankMaps& rm, int t_end, int gw, int nw, int lane) {
+    const int k = kK ? kK : p.k, T = p.T;
+    const bool vec = (k & 3) == 0;
+    constexpr int kW = kPlain ? 1 : kRankWords;
+    const int groups = (min(t_end, T) + 31) >> 5;
+    for (int g = gw; g < groups; g += nw) {
+        const int t = g * 32 + lane;
+        unsigned m[kW];
+#pragma unroll
+        for (int w = 0; w < kW; ++w) m[w] = 0u;
+        if (t < T) {
+            const int32_t* src = p.topk_idx + (size_t)t * k;
+            for (int j0 = 0; j0 < k; j0 += 8) {
+                int raw[8];
+                if (vec) {
+                    const int4 a = __ldg(reinterpret_cast<const int4*>(src + j0));
+                    const int4 b = j0 + 4 < k ? __ldg(reinterpret_cast<const int4*>(src + j0 + 4)) : make_int4(-1, -1, -1, -1);
+                    raw[0] = a.x; raw[1] = a.y; raw[2] = a.z; raw[3] = a.w;
+                    raw[4] = b.x; raw[5] = b.y; raw[6] = b.z; raw[7] = b.w;
+                } else {
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) raw[u] = j0 + u < k ? __ldg(src + j0 + u) : -1;
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    int e = raw[u];
+                    if (!kPlain && p.phys != nullptr) {
+                        const bool in = (unsigned)e < (unsigned)p.E_log;
+                        const int nc = in ? __ldg(p.ncopies + e) : 1;
+                        const bool okc = in && nc >= 1 && nc <= p.C;
+                        e = okc ? __ldg(p.phys + (size_t)e * p.C + (t % nc)) : -1;
+                    }
+                    const bool valid = (unsigned)e < (unsigned)p.E;
+                    const int r = fast_div(e, p.L_magic);
+                    if (kPlain) {
+                        m[0] |= valid ? 1u << r : 0u;
+                    } else {
+#pragma unroll
+                        for (int w = 0; w < kW; ++w) m[w] |= (valid && w == (r >> 5)) ? 1u << (r & 31) : 0u;
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int w = 0; w < kW; ++w)
+            if (w < rm.wr) rm.rbm[(size_t)g * rm.rp + w * 32 + lane] = transpose32(m[w], lane);
+    }
+}
+static __device__ void local_rank_maps(const Params& p, const RankMaps& rm, int t_end, int gw, int nw, int lane) {
+    if (p.phys == nullptr && rm.wr == 1) {
+        if (p.k == 8) rank_maps_pass<true, 8>(p, rm, t_end, gw, nw, lane);
+        else rank_maps_pass<true, 0>(p, rm, t_end, gw, nw, lane);
+    } else {
+        rank_maps_pass<false, 0>(p, rm, t_end, gw, nw, lane);
     }
 }
 
