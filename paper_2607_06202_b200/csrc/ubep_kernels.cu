@@ -221,7 +221,7 @@ __device__ __forceinline__ void mover_warp(Cta& x) {
         if (fast_local) {
             // lend a hand with the routing table.  (Rows asked for before every warp's share of the table
             // is in -- even as late as when this warp's own share has arrived -- delay it: measured 0.9 us.)
-            local_stage_and_rank_maps(p, ids_sm, rm, 0, kWarps, lane);
+            local_stage_and_rank_maps(p, ids_sm, rm, rm.groups, 0, kWarps, lane);
             group_sync(2, kThreads);
         } else if (kMode == kModeLocal) {
             ok = mbar_wait(x.staged_bar, 0, abortp);
@@ -300,7 +300,7 @@ __device__ __forceinline__ void mover_warp(Cta& x) {
     } else {
         if (fast_local) {
             const RankMaps rm{bmaps.bm, bmaps.mask_t, (p.R + 31) / 32, ((p.R + 31) / 32) * 32, (p.T + 31) / 32};
-            local_stage_and_rank_maps(p, ids_sm, rm, 0, kWarps, lane);   // the table first, the rows after it
+            local_stage_and_rank_maps(p, ids_sm, rm, rm.groups, 0, kWarps, lane);   // the table first, the rows after it
             group_sync(2, kThreads);
         } else if (kMode == kModeLocal || x.beside) {
             // the routing table first: it is the one load the layout waits for
@@ -404,7 +404,7 @@ __device__ __forceinline__ int layout_group(Cta& x) {
         // rank-level rows first, movers released, expert-level outputs afterwards
         const RankMaps rm{bmaps.bm, bmaps.mask_t, (p.R + 31) / 32, ((p.R + 31) / 32) * 32, (p.T + 31) / 32};
         int* row_sm = reinterpret_cast<int*>(w_sm);
-        local_stage_and_rank_maps(p, ids_sm, rm, warp, kWarps, lane);   // with the mover warp
+        local_stage_and_rank_maps(p, ids_sm, rm, rm.groups, warp, kWarps, lane);   // with the mover warp
         stage_small(gn);
         group_sync(2, kThreads);
         if (gtid == 0) trace(p, c, kTrCounted);

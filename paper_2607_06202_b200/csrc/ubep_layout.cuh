@@ -502,19 +502,27 @@ struct RankMaps {
 constexpr int kRankWords = 4;
 
 
-// Stage all T*k slots (packed id | rank << 16) and build the rank bitmaps; lane = token.
+// Stage the slots (packed id | rank << 16) of the token groups [0, g_end) and build their rank bitmaps;
+// lane = token, one group of 32 tokens per warp and trip.  Every CTA of the flag-free kernel runs this
+// redundantly before its first copy and the step is bound by instruction issue (16 warps on four
+// schedulers), so the common case -- no replica table, at most 32 ranks, eight slots per token -- is a
+// variant of its own without per-slot branches: measured per warp and group, warm, 2380 cycles for the
+// general form with a branch and a possible call per slot, about 1100 for this one.
 // (An expert named twice by a token does not change any rank-level row, so this step, which every
 // copy waits for, does not look for it; that happens once the movers are released.
 // Looking for it here was measured to cost 2.5 us per dispatch of 512 tokens.)
-static __device__ void local_stage_and_rank_maps(const Params& p, int* ids, const RankMaps& rm, int gw, int nw, int lane) {
-    const int k = p.k, T = p.T;
+template <bool kPlain, int kK>   // kPlain: no replica table, one word of ranks; kK: slots per token if fixed
+__device__ __forceinline__ void stage_and_rank_maps_pass(const Params& p, int* ids, const RankMaps& rm, int g_end,
+                                                         int gw, int nw, int lane) {
+    const int k = kK ? kK : p.k, T = p.T;
     const bool vec = (k & 3) == 0;   // a token's ids are whole 16-byte words (topk_idx is 16-byte aligned)
+    constexpr int kW = kPlain ? 1 : kRankWords;
     bool bad = false;
-    for (int g = gw; g < rm.groups; g += nw) {
+    for (int g = gw; g < g_end; g += nw) {
         const int t = g * 32 + lane;
-        unsigned m[kRankWords];
+        unsigned m[kW];
 #pragma unroll
-        for (int w = 0; w < kRankWords; ++w) m[w] = 0u;
+        for (int w = 0; w < kW; ++w) m[w] = 0u;
         if (t < T) {
             const int32_t* src = p.topk_idx + (size_t)t * k;
             for (int j0 = 0; j0 < k; j0 += 8) {       // up to eight ids in flight
@@ -531,18 +539,25 @@ static __device__ void local_stage_and_rank_maps(const Params& p, int* ids, cons
                 int pk[8];
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
-                    pk[u] = -1;
-                    if (j0 + u >= k) continue;
-                    const int e = resolve_expert(p, t, raw[u], bad);
-                    if (e >= 0) {
-                        const int r = fast_div(e, p.L_magic);
-                        pk[u] = e | (r << 16);
-                        if (rm.wr == 1) {
-                            m[0] |= 1u << r;
-                        } else {
+                    int e = raw[u];   // (slots past the k-th hold -1)
+                    if (!kPlain && p.phys != nullptr) {
+                        const bool in = (unsigned)e < (unsigned)p.E_log;
+                        bad |= !in && e != -1;
+                        const int nc = in ? __ldg(p.ncopies + e) : 1;
+                        const bool okc = in && nc >= 1 && nc <= p.C;
+                        bad |= in && !okc;
+                        e = okc ? __ldg(p.phys + (size_t)e * p.C + (t % nc)) : -1;
+                        bad |= okc && e < 0;
+                    }
+                    const bool valid = (unsigned)e < (unsigned)p.E;
+                    bad |= !valid && e != -1;
+                    const int r = fast_div(e, p.L_magic);
+                    pk[u] = valid ? (e | (r << 16)) : -1;
+                    if (kPlain) {
+                        m[0] |= valid ? 1u << r : 0u;
+                    } else {
 #pragma unroll
-                            for (int w = 0; w < kRankWords; ++w) m[w] |= (w == (r >> 5)) ? 1u << (r & 31) : 0u;
-                        }
+                        for (int w = 0; w < kW; ++w) m[w] |= (valid && w == (r >> 5)) ? 1u << (r & 31) : 0u;
                     }
                 }
                 // (one 16-byte store per four slots: scalar stores of a lane's slots, 32 bytes apart from
@@ -558,72 +573,18 @@ static __device__ void local_stage_and_rank_maps(const Params& p, int* ids, cons
             }
         }
 #pragma unroll
-        for (int w = 0; w < kRankWords; ++w)
+        for (int w = 0; w < kW; ++w)
             if (w < rm.wr) rm.rbm[(size_t)g * rm.rp + w * 32 + lane] = transpose32(m[w], lane);
     }
     if (bad) report(p.status, kErrBadIndex);
 }
-
-// The rank bitmaps alone, of tokens [0, t_end) rounded up to whole groups: what the rows of a CTA whose
-// tokens end at t_end depend on.  Every CTA runs this redundantly before its first copy, and the step is
-// bound by instruction issue (16 warps, one group of 32 tokens each): measured per warp and group, warm,
-// 2380 cycles for the pass above, 900 for this one, 730 with the slot count fixed at eight.  So nothing
-// is stored per slot, nothing is reported (the pass that stages the ids reports), a bad id just sets no bit.
-template <bool kPlain, int kK>   // kPlain: no replica table and at most 32 ranks; kK: slots per token if fixed
-__device__ __forceinline__ void rank_maps_pass(const Params& p, const RankMaps& rm, int t_end, int gw, int nw, int lane) {
-    const int k = kK ? kK : p.k, T = p.T;
-    const bool vec = (k & 3) == 0;
-    constexpr int kW = kPlain ? 1 : kRankWords;
-    const int groups = (min(t_end, T) + 31) >> 5;
-    for (int g = gw; g < groups; g += nw) {
-        const int t = g * 32 + lane;
-        unsigned m[kW];
-#pragma unroll
-        for (int w = 0; w < kW; ++w) m[w] = 0u;
-        if (t < T) {
-            const int32_t* src = p.topk_idx + (size_t)t * k;
-            for (int j0 = 0; j0 < k; j0 += 8) {
-                int raw[8];
-                if (vec) {
-                    const int4 a = __ldg(reinterpret_cast<const int4*>(src + j0));
-                    const int4 b = j0 + 4 < k ? __ldg(reinterpret_cast<const int4*>(src + j0 + 4)) : make_int4(-1, -1, -1, -1);
-                    raw[0] = a.x; raw[1] = a.y; raw[2] = a.z; raw[3] = a.w;
-                    raw[4] = b.x; raw[5] = b.y; raw[6] = b.z; raw[7] = b.w;
-                } else {
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) raw[u] = j0 + u < k ? __ldg(src + j0 + u) : -1;
-                }
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    int e = raw[u];
-                    if (!kPlain && p.phys != nullptr) {
-                        const bool in = (unsigned)e < (unsigned)p.E_log;
-                        const int nc = in ? __ldg(p.ncopies + e) : 1;
-                        const bool okc = in && nc >= 1 && nc <= p.C;
-                        e = okc ? __ldg(p.phys + (size_t)e * p.C + (t % nc)) : -1;
-                    }
-                    const bool valid = (unsigned)e < (unsigned)p.E;
-                    const int r = fast_div(e, p.L_magic);
-                    if (kPlain) {
-                        m[0] |= valid ? 1u << r : 0u;
-                    } else {
-#pragma unroll
-                        for (int w = 0; w < kW; ++w) m[w] |= (valid && w == (r >> 5)) ? 1u << (r & 31) : 0u;
-                    }
-                }
-            }
-        }
-#pragma unroll
-        for (int w = 0; w < kW; ++w)
-            if (w < rm.wr) rm.rbm[(size_t)g * rm.rp + w * 32 + lane] = transpose32(m[w], lane);
-    }
-}
-static __device__ void local_rank_maps(const Params& p, const RankMaps& rm, int t_end, int gw, int nw, int lane) {
+static __device__ void local_stage_and_rank_maps(const Params& p, int* ids, const RankMaps& rm, int g_end, int gw, int nw,
+                                          int lane) {
     if (p.phys == nullptr && rm.wr == 1) {
-        if (p.k == 8) rank_maps_pass<true, 8>(p, rm, t_end, gw, nw, lane);
-        else rank_maps_pass<true, 0>(p, rm, t_end, gw, nw, lane);
+        if (p.k == 8) stage_and_rank_maps_pass<true, 8>(p, ids, rm, g_end, gw, nw, lane);
+        else stage_and_rank_maps_pass<true, 0>(p, ids, rm, g_end, gw, nw, lane);
     } else {
-        rank_maps_pass<false, 0>(p, rm, t_end, gw, nw, lane);
+        stage_and_rank_maps_pass<false, 0>(p, ids, rm, g_end, gw, nw, lane);
     }
 }
 
