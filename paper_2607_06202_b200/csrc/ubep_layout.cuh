@@ -597,37 +597,60 @@ __device__ __forceinline__ int rank_rows_before(const RankMaps& rm, int r, int t
     return c;
 }
 
-// Destinations of this CTA's tokens [t0, t1): pos_raw (slot order), dst_rank, row_sm, arr.
+// Destinations of this CTA's tokens [t0, t1): pos_raw (slot order), dst_key (only with a destination
+// table), row_sm, arr.  Every copy of the CTA waits for this step and a handful of threads run it, so it
+// is written for latency: no branch per slot, the token's other slots compared in registers, the bit
+// counts of the groups below the token unrolled (independent loads), one report after the loop.
 // (Ordering the destinations with warp shuffles right here instead of in a separate pass
 // was measured slower on the decode shape and is not done.)
+template <int kK>   // slots per token if fixed
+__device__ __forceinline__ void rows_dedup_pass(const Params& p, int t0, int t1, const int* ids_all, const RankMaps& rm,
+                                                int worker, const int* order_sm, int* pos_raw, int* dst_key, int* row_sm,
+                                                int* arr, int gtid, int gn) {
+    const int k = kK ? kK : p.k;
+    const int nslots = (t1 - t0) * k;
+    const int rot = worker % p.R;
+    bool full = false;
+    for (int li = gtid; li < nslots; li += gn) {
+        const int tl = li / k, j = li - tl * k, t = t0 + tl;
+        const int* tok = ids_all + (size_t)t * k;
+        const int packed = tok[j];
+        const bool have = packed >= 0;
+        const int r = have ? slot_rank(packed) : 0;
+        bool first = have;   // no earlier slot of the token names the same rank (-1 >> 16 is no rank)
+        if (kK == 8) {
+            const int4 a = *reinterpret_cast<const int4*>(tok), b = *reinterpret_cast<const int4*>(tok + 4);
+            const int v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int jj = 0; jj < 7; ++jj) first = first && !(jj < j && slot_rank(v[jj]) == r);
+        } else {
+            for (int jj = 0; jj < j; ++jj) first = first && slot_rank(tok[jj]) != r;
+        }
+        // tokens below t that visit rank r
+        const int g1 = t >> 5;
+        const unsigned* col = rm.rbm + r;
+        int row = __popc(col[(size_t)g1 * rm.rp] & ((1u << (t & 31)) - 1u));
+#pragma unroll 8
+        for (int g = 0; g < g1; ++g) row += __popc(col[(size_t)g * rm.rp]);
+        const bool fits = row < p.cap;
+        full = full || (have && !fits);
+        const bool send = first && fits;
+        if (send) atomicAdd(&arr[r], 1);
+        pos_raw[li] = send ? r * p.cap + row : -1;
+        if (p.ordered) {
+            int kv = order_sm[r] - rot;
+            kv = kv < 0 ? kv + p.R : kv;
+            dst_key[li] = send ? kv : p.R;
+        }
+        row_sm[li] = have ? row : -1;
+    }
+    if (full) report(p.status, kErrCapacity);
+}
 static __device__ void local_rows_dedup(const Params& p, int t0, int t1, const int* ids_all, const RankMaps& rm,
                                  int worker, const int* order_sm, int* pos_raw, int* dst_key, int* row_sm, int* arr,
                                  int gtid, int gn) {
-    const int k = p.k;
-    const int nslots = (t1 - t0) * k;
-    for (int li = gtid; li < nslots; li += gn) {
-        const int tl = li / k, j = li - tl * k, t = t0 + tl;
-        const int packed = ids_all[(size_t)t * k + j];
-        int where = -1, row = -1, r = 0;
-        if (packed >= 0) {
-            r = slot_rank(packed);
-            bool first = true;
-            for (int jj = 0; jj < j; ++jj) {
-                const int v2 = ids_all[(size_t)t * k + jj];
-                if (v2 >= 0 && slot_rank(v2) == r) { first = false; break; }
-            }
-            row = rank_rows_before(rm, r, t);
-            if (row >= p.cap) {
-                report(p.status, kErrCapacity);
-            } else if (first) {
-                where = r * p.cap + row;
-                atomicAdd(&arr[r], 1);
-            }
-        }
-        pos_raw[li] = where;
-        dst_key[li] = where >= 0 ? rotated_key(order_sm, r, worker, p.R) : p.R;
-        row_sm[li] = row;
-    }
+    if (p.k == 8) rows_dedup_pass<8>(p, t0, t1, ids_all, rm, worker, order_sm, pos_raw, dst_key, row_sm, arr, gtid, gn);
+    else rows_dedup_pass<0>(p, t0, t1, ids_all, rm, worker, order_sm, pos_raw, dst_key, row_sm, arr, gtid, gn);
 }
 
 // The ids of a token must be distinct: the later of two slots naming one expert is reported
