@@ -421,6 +421,9 @@ int ubep_dispatch(ubep_buffer_t* buf, const void* x, const int32_t* topk_idx, co
             const int chunks = n / parts;
             if (chunks < 1 || (p.H * 2 / parts) % 16 != 0 || (p.H * 2) % parts != 0) break;
             if (p.payload && ((p.H / parts) % 128 != 0 || p.H % parts != 0)) break;
+            // FP8 rows: a piece's scales must still be a bulk copy (a multiple of 16 bytes); with plain stores for
+            // the scales and payload pieces under 2 KB a dispatch of 384 tokens took 33 us against 21 us for 512
+            if (p.payload && parts > 1 && ((p.G / parts) * 4) % 16 != 0) break;
             const double cost = (double)((T + chunks - 1) / chunks) / parts * kPiecePenalty[i];
             if (parts == 1 || cost < best_cost * 0.999) {
                 best = parts;

@@ -388,6 +388,19 @@ __device__ __forceinline__ void mover_warp(Cta& x) {
             }
         }
     }
+    if (kFp8 && fast_local && ok) {
+        // metadata of the CTA's own tokens (see the row group): one warp, no barrier but its own
+        ok = mbar_wait(&ready_bar, 0, abortp);
+        ok = __all_sync(0xffffffffu, ok);
+        if (ok) {
+            float* w_own = reinterpret_cast<float*>(key);   // the ordering keys are no longer needed
+            if (part == 0)
+                for (int i = lane; i < ntok * p.k; i += 32) w_own[i] = __ldg(p.topk_w + (size_t)t0 * p.k + i);
+            local_clean_own_duplicates(p, t0, t1, ids_sm, lane, 32);
+            __syncwarp();
+            if (part == 0) local_meta_dedup(p, t0, t1, ids_sm, pos_raw, reinterpret_cast<int*>(w_sm), w_own, lane, 32);
+        }
+    }
     if (!ok && lane == 0) {
         report(p.status, kErrTimeout);  // a wait gave up: record it and let everybody leave
         abort_flag = 1;
@@ -453,6 +466,14 @@ __device__ __forceinline__ int layout_group(Cta& x) {
                 *x.epoch_late = ep_mine;
                 ticket = atomicAdd(p.done_ticket, 1u);
             }
+            if (kFp8) {
+                // FP8 rows: every copy waits for a quantised row, so this group goes straight on to quantise
+                // (its first warp to issue the copies; the warps of the duty group take no part, a CTA of
+                // this kernel has few rows).  The metadata of the own tokens is written by the loader warp,
+                // which is idle once the CTA's few rows are asked for.
+                if (gtid == 0) epoch_finish_check_in(p, ticket, ep_mine);
+                return 1;
+            }
             if (part == 0) {
                 float* w_own = reinterpret_cast<float*>(key);   // the ordering keys are no longer needed
                 for (int i = gtid; i < ntok * p.k; i += rn) w_own[i] = __ldg(p.topk_w + (size_t)t0 * p.k + i);
@@ -465,16 +486,20 @@ __device__ __forceinline__ int layout_group(Cta& x) {
                 epoch_finish_check_in(p, ticket, ep_mine);
                 if (p.trace) p.trace[(size_t)c * kTraceSlots + 12] = trace_ns(p);
             }
+        } else if (kFp8 && warp - x.qwarp0 < x.nq) {
+            return 1;   // FP8 rows: the first warps behind the row group quantise as well
         } else {
             // expert-level outputs of rank r: shared by Q CTAs so that no CTA trails the others
-            const int dn = gn - kRowThreads, dw = nw - kRowWarps;
+            const int dgw0 = kFp8 ? max(kRowWarps, x.qwarp0 + x.nq - 1) : kRowWarps;   // first warp of the duty group
+            const int dn = gn - dgw0 * 32, dw = nw - dgw0;
             const int Q = p.grid / p.R > 1 ? p.grid / p.R : 1;
             // ... once the movers are released: started earlier, these warps take issue slots and
             // shared-memory bandwidth from the few threads every copy of this CTA is waiting for
             const bool go = mbar_wait_idle(&ready_bar, 0, abortp);
             for (int u = c; go && u < p.R * Q; u += p.grid)
-                local_rank_duty(p, u / Q, u % Q, Q, ids_sm, rm, hist, gw - kRowWarps, dw, lane, gtid - kRowThreads, dn, 3);
-            if (gtid == kRowThreads) trace(p, c, kTrScanned);   // deferred outputs written
+                local_rank_duty(p, u / Q, u % Q, Q, ids_sm, rm, hist, gw - dgw0, dw, lane, gtid - dgw0 * 32, dn, 3);
+            if (gtid == dgw0 * 32) trace(p, c, kTrScanned);   // deferred outputs written
+            if (kFp8) return go ? 3 : 0;   // (these warps do not quantise: the row group's warps do)
         }
     } else if (kMode == kModeLocal) {
         // every CTA: bitmaps over the whole routing table -> totals, the rows before its
@@ -800,7 +825,10 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
     const bool beside = kFp8 && kMode != kModeLocal && p.count_warps > 0;
     const int nw = beside ? p.count_warps : kWarps - 1;      // layout group: warps 1 .. nw
     const int qwarp0 = beside ? nw + 1 : 2;                    // FP8: warps qwarp0 .. qwarp0 + nq - 1 quantise
-    const int nq = kFp8 ? min(p.quant_warps, kWarps - qwarp0) : kWarps - 2;
+    // (flag-free kernel with rank-level rows: a CTA has few rows, and the warps that do not quantise write
+    // the expert-level outputs meanwhile)
+    const int nq = kFp8 ? min(kMode == kModeLocal && p.local_fast ? min(p.quant_warps, kFastQuantWarps) : p.quant_warps, kWarps - qwarp0)
+                        : kWarps - 2;
     int* arr = reinterpret_cast<int*>(smem + pl.off_arr);
     griddep_launch();   // the next kernel in the stream may be placed as soon as SMs have room
 
