@@ -283,7 +283,7 @@ def main_roles(argv):
 
 def main_auto(argv):
     ap = argparse.ArgumentParser(prog="bench_sweeps.py auto")
-    ap.add_argument("--tokens", type=int, nargs="*", default=[64, 128, 256, 512, 1024, 2048])
+    ap.add_argument("--tokens", type=int, nargs="*", default=[64, 128, 256, 512, 768, 1024, 1536, 2048])
     ap.add_argument("--markdown", action="store_true")
     args = ap.parse_args(argv)
     B.load()
