@@ -62,6 +62,7 @@ struct Cta {
     unsigned* epoch_late;
     size_t in_off, out_off;
     bool fast_local;
+    bool early0;  // flag-free kernel: the copies of the CTA's first row are issued by the warp that assigns the rows
     int issued;   // rows whose load the mover has started (thread 0's copy is used when leaving early)
 };
 
@@ -264,12 +265,13 @@ __device__ __forceinline__ void mover_warp(Cta& x) {
         }
         if (!kSteal) {
             // the CTA's own rows, in order: row n sits in stage n % stages
-            for (int n = 0; ok && n < ntok; ++n) {
+            const int n0 = x.early0 ? 1 : 0;   // (the first row's copies may have been issued by the row group)
+            for (int n = n0; ok && n < ntok; ++n) {
                 const int s = n % stages;
                 ok = mbar_wait(&full_bar[s], (n / stages) & 1, abortp);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                if (n == 0 && lane == 0) trace(p, c, kTrFirstRow);
+                if (n == n0 && lane == 0) trace(p, c, kTrFirstRow);
                 const uint8_t* src = smem + (size_t)s * pl.stage_bytes;
                 for (int j = lane; j < p.k; j += 32) {
                     const int where = pos[n * p.k + j];
@@ -449,6 +451,22 @@ __device__ __forceinline__ int layout_group(Cta& x) {
         if (gw < kRowWarps) {
             const int rn = kRowThreads;
             local_rows_dedup(p, t0, t1, ids_sm, rm, c, order_sm, pos_raw, key, row_sm, arr, gtid, rn);
+            if (x.early0 && gw == 0) {
+                // The copies of the CTA's first row leave from here: lane j has just worked out where slot j of
+                // the first token goes (its own write to pos_raw), and the row was asked for before the routing
+                // table was (and prefetched into L2 before that), so it sits in the ring's first stage or is
+                // about to.  The mover warp, which needs another 0.5 us to notice the release and get going,
+                // starts with the second row.  (Measured per layer, 512 tokens: 25.2 us against 25.6; neither
+                // this nor the prefetch of the rows changes anything without the other.)
+                const int where = lane < p.k ? pos_raw[lane] : -1;
+                const bool got = mbar_wait(&full_bar[0], 0, abortp);
+                if (got && where >= 0) bulk_store(p.recv_x + (size_t)where * p.rowB + out_off, smem, out_bytes);
+                bulk_commit();
+                if (!got && lane == 0) {
+                    report(p.status, kErrTimeout);
+                    *abortp = 1;
+                }
+            }
             group_sync(1, rn);
             if (gtid == 0) trace(p, c, kTrFinalized);
             if (p.ordered) {   // a destination table is set: the copies of a token in its order (else pos_raw is pos)
@@ -857,6 +875,15 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
         const size_t bytes = (size_t)p.T * p.k * 4;
         for (size_t off = ((size_t)c * kThreads + tid) * 128; off < bytes; off += (size_t)p.grid * kThreads * 128)
             asm volatile("prefetch.global.L2 [%0];" ::"l"(tab + off));
+        // The same for the CTA's own pieces of its rows: inside a layer they come from HBM while it is still
+        // writing back what the kernels before left in L2, and the first of them is what the first copy waits for.
+        const unsigned piece = (unsigned)(p.H * 2 / p.parts);
+        const int lines = (int)((piece + 127u) / 128u);
+        const char* xs = reinterpret_cast<const char*>(p.x) + (size_t)t0 * p.H * 2 + (size_t)part * piece;
+        for (int i = tid; i < (t1 - t0) * lines; i += kThreads) {
+            const int tl = i / lines, l = i - tl * lines;
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(xs + (size_t)tl * p.H * 2 + (size_t)l * 128));
+        }
     }
     griddep_wait();     // shared-memory set-up done; everything below reads what earlier kernels wrote
     // The epoch is not read here, in front of everything: the flag-free kernel needs it only for the
@@ -881,12 +908,17 @@ __global__ void __launch_bounds__(kThreads, 1) dispatch_kernel(const Params p, c
                   pl.map_wb, pl.map_bp, pl.map_groups},
           reinterpret_cast<int*>(smem + pl.off_hist), arr, reinterpret_cast<int*>(smem + pl.off_order),
           epoch, in_bytes, out_bytes, &epoch_sm, (size_t)part * in_bytes, (size_t)part * out_bytes,
-          kMode == kModeLocal && p.local_fast != 0, 0};
+          kMode == kModeLocal && p.local_fast != 0,
+          // (its stage is never loaded a second time, no order of destinations is asked for, a lane per copy)
+          kMode == kModeLocal && p.local_fast != 0 && !kFp8 && !kSteal && !p.ordered && p.k <= 32 && t1 > t0 &&
+              t1 - t0 <= stages,
+          0};
 
     if (x.warp == 0) {
         mover_warp<kMode, kFp8, kSteal>(x);
     } else {
         const int lg = layout_group<kMode, kFp8, kSteal>(x);   // 0 = a wait ran out, 1 = done, 2 = left to quantise
+        if (!kFp8 && x.early0 && x.warp == 1) bulk_wait_all<0>();   // the first row's copies (issued by this warp)
         if (kFp8 && lg == 2) {
             if (x.warp - qwarp0 < nq) fp8_quantiser<kSteal>(x, x.warp - qwarp0);   // beside the rest of the layout
         } else if (kFp8 && lg == 1) {
