@@ -314,7 +314,7 @@ def main_auto(argv):
 # ----------------------------------------------------------------------------------- budget
 
 PHASES = [(0, "CTA starts (predecessor complete)"), (1, "routing table staged, bitmaps built"), (5, "rows assigned"),
-          (6, "movers released"), (7, "first row in shared memory, first copies issued"), (8, "last copy issued"),
+          (6, "movers released"), (7, "mover warp's first row in shared memory, its copies issued"), (8, "last copy issued"),
           (9, "copies complete"), (3, "expert-level outputs written (duty group)"), (10, "CTA ends")]
 
 
