@@ -105,6 +105,32 @@ def test_many_tokens_per_chunk(payload, dedup):
     Hn.run_case(W.make_workload(cfg), pipeline=FUSED, threads=oracle.host_cores())
 
 
+@pytest.mark.parametrize("payload", [0, 1])
+def test_flag_free_kernel_with_one_row_per_rank_at_its_edges(payload):
+    """The rank-level fast path of the flag-free kernel: the first row's copies issued by the warp that
+    assigns the rows (only without a destination table and while the ring never reloads its first stage),
+    routing tables up to AUTO's crossover, FP8 pieces whose scales are or are not a bulk copy."""
+    rng = np.random.default_rng(5)
+    cfg = small(300, 256, 32, 8, 4, payload, 1, seed=41)
+    wl = W.with_empty_slots(W.make_workload(cfg), 0.1, seed=9)
+    for order in (None, list(rng.permutation(8))):
+        Hn.run_case(wl, pipeline=LOCAL, dest_order=order)
+    # about 15 tokens per CTA: the ring is as long as it gets and holds every row of the CTA
+    Hn.run_case(W.make_workload(small(1100, 128, 64, 16, 8, payload, 1, seed=42)), pipeline=LOCAL)
+    # 2048 tokens x top-8: AUTO's largest flag-free table (bf16), more rows per CTA than ring stages
+    Hn.run_case(W.make_workload(small(2048, 128, 64, 16, 8, payload, 1, seed=43)), pipeline=AUTO,
+                threads=oracle.host_cores())
+    # a CTA whose first token has no destination at all
+    wl = W.make_workload(small(148 * 3, 256, 32, 8, 4, payload, 1, seed=44))
+    wl.topk_idx[::3] = -1
+    Hn.run_case(wl, pipeline=LOCAL)
+    if payload:
+        # 7168 channels: 56 scales per row; four column parts would leave 14 scales (56 bytes) per piece
+        for T in (256, 384):
+            cfg = W.Config("fp8rows", T=T, H=7168, E=256, R=32, k=8, payload=1, dedup=1, seed=45 + T)
+            Hn.run_case(W.make_workload(cfg), pipeline=LOCAL, threads=oracle.host_cores())
+
+
 def test_destination_order_table_does_not_change_results():
     cfg = small(300, 256, 32, 8, 4, seed=4)
     wl = W.make_workload(cfg)
