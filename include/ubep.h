@@ -283,9 +283,10 @@ int ubep_map_workers(const int32_t *order /*[dev]*/, const int32_t *counts /*[de
  * Table 3); Token-Flag blocks and Sentinel blocks are cut from that, the checksum markers from the
  * payload.  What arrives goes to the region's payload and scale arrays.
  *
- * Limits: T * k <= 8192 and the routing table with the bitmaps of all its
- * bins (T x (E + R) bits) must fit in a CTA's shared memory, since every CTA derives the layout
- * from the whole table, as UBEP_PIPELINE_LOCAL does; one CTA per SM at most, launched
+ * Routing tables of any size: up to 8192 slots (T * k), and while the table with the bitmaps of all its
+ * bins (T x (E + R) bits) fits in a CTA's shared memory, every CTA derives the layout from the whole
+ * table, as UBEP_PIPELINE_LOCAL does (one launch); for a larger table the counting and prefix-sum
+ * kernels of UBEP_PIPELINE_PHASED run in front of the protocol kernel (three launches).  One CTA per SM at most, launched
  * cooperatively (receivers wait for senders of the same grid, so the grid must be resident at once:
  * a grid that cannot be is refused with UBEP_ERR_CUDA instead of running into its timeouts).  Everything
  * ubep_dispatch leaves in the arena is left here too, with identical contents; ubep_combine
@@ -324,10 +325,10 @@ int ubep_sync_attach(ubep_buffer_t *buf, void *dev_wire /*[dev]*/, size_t bytes,
 
 /*
  * Dispatch with readiness protocol `protocol` (UBEP_SYNC_*); arguments as ubep_dispatch.
- * One kernel launch (a memset before it when an earlier call left the SP wire dirty, which
+ * One kernel launch, three for large routing tables (a memset before it when an earlier call left the SP wire dirty, which
  * the library learns when ubep_status reports that call's error; until then a word on the
  * device makes every Sentinel Polling call on that wire report UBEP_ERR_TIMEOUT and move nothing).  UBEP_ERR_ARG if no wire
- * buffer is attached, T * k > 8192 or the table does not fit in shared memory.
+ * buffer is attached or T exceeds the buffer's max_tokens.
  */
 int ubep_dispatch_sync(ubep_buffer_t *buf, int protocol, const void *x /*[dev]*/,
                        const int32_t *topk_idx /*[dev]*/, const float *topk_w /*[dev]*/, int32_t T,

@@ -502,7 +502,7 @@ int ubep_sync_attach(ubep_buffer_t* buf, void* dev_wire, size_t bytes, void* cud
 int ubep_dispatch_sync(ubep_buffer_t* buf, int protocol, const void* x, const int32_t* topk_idx, const float* topk_w,
                        int32_t T, void* cuda_stream) {
     if (!buf || !buf->wire || protocol < UBEP_SYNC_SW || protocol > UBEP_SYNC_SP) return UBEP_ERR_ARG;
-    if (T < 0 || T > buf->cfg.max_tokens || (int64_t)T * buf->cfg.topk > kLocalMaxSlots) return UBEP_ERR_ARG;
+    if (T < 0 || T > buf->cfg.max_tokens) return UBEP_ERR_ARG;
     if (T > 0 && (!x || !topk_idx || !topk_w)) return UBEP_ERR_ARG;
     if (!aligned16(x) || !aligned16(topk_idx) || !aligned16(topk_w)) return UBEP_ERR_ARG;
     DeviceGuard guard(buf->cfg.device);
@@ -523,7 +523,12 @@ int ubep_dispatch_sync(ubep_buffer_t* buf, int protocol, const void* x, const in
     p.grid = p.nchunks;
     ubep::SmemPlan pl{};
     const int extra = ubep::sync_extra_smem(p);
-    if (ubep::plan_dispatch(p, UBEP_PIPELINE_LOCAL, buf->max_smem - extra, &pl) != 0) return UBEP_ERR_ARG;
+    // Small tables are recounted by every CTA; for larger ones TokenCnt and CalCumSum run as launches of their
+    // own in front of the kernel, over the same chunks (as the phased schedule of ubep_dispatch does).
+    const bool whole_table = (int64_t)T * buf->cfg.topk <= kLocalMaxSlots &&
+                             ubep::plan_dispatch(p, UBEP_PIPELINE_LOCAL, buf->max_smem - extra, &pl) == 0;
+    if (!whole_table && ubep::plan_dispatch(p, UBEP_PIPELINE_PHASED, buf->max_smem - extra, &pl) != 0)
+        return UBEP_ERR_ARG;
     const WireLayout& w = buf->wlay;
     ubep::SyncParams sp{};
     sp.protocol = protocol;
@@ -548,7 +553,12 @@ int ubep_dispatch_sync(ubep_buffer_t* buf, int protocol, const void* x, const in
         if (e != cudaSuccess) return cuda_fail(buf, e);
         buf->sp_dirty = false;
     }
-    e = ubep::launch_sync_dispatch(p, pl, sp, st);
+    if (!whole_table) {
+        e = ubep::launch_count_scan(p, pl, st);
+        if (e != cudaSuccess) return cuda_fail(buf, e);
+        g_launches += 2;
+    }
+    e = ubep::launch_sync_dispatch(p, pl, sp, whole_table, st);
     if (e != cudaSuccess) return cuda_fail(buf, e);
     g_launches += 1;
     return UBEP_OK;

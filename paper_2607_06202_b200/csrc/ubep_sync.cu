@@ -96,7 +96,10 @@ __device__ __forceinline__ bool wait_count(const unsigned* ctr, unsigned want, W
 // wire row of H + 4 * H / 128 bytes); the sender quantises a row once into shared memory and sends from
 // there; what arrives goes to the payload and the scale array of the receive region.  The checksum
 // markers of Data-for-Checksum are taken from the payload bytes.
-template <int kProto, bool kFp8>
+// kTable: the layout is derived here from the whole routing table in shared memory (small tables).
+// Otherwise it comes from count_kernel / scan_kernel, launched before over the same chunks: the CTA stages
+// only its own tokens and reads the rows of earlier chunks, the expert offsets and the region sizes.
+template <int kProto, bool kFp8, bool kTable>
 __global__ void __launch_bounds__(kThreads, 1) sync_dispatch_kernel(const Params p, const SmemPlan pl,
                                                                    const SyncParams sp) {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -141,24 +144,40 @@ __global__ void __launch_bounds__(kThreads, 1) sync_dispatch_kernel(const Params
     int* tot = hist;
     int* pre = hist + p.B;
     int* eo = hist + 2 * p.B;
-    stage_ids(p, 0, p.T, ids_sm, tid, kThreads);
+    if (kTable) stage_ids(p, 0, p.T, ids_sm, tid, kThreads);
+    else stage_ids(p, t0, t1, ids_sm, tid, kThreads);
     for (int r = tid; r < R; r += kThreads) order_sm[r] = __ldg(p.order_pos + r);
     for (int i = tid; i < ntok * k; i += kThreads) w_sm[i] = __ldg(p.topk_w + (size_t)t0 * k + i);
     __syncthreads();
     const unsigned seq = seq_sm;
     const int par = (int)(seq & 1u);
-    local_counts_all_bins(p, ids_sm, bmaps, t0, tot, pre, eo, tid, kThreads, warp, kWarps, lane, 0);
-    for (int r = tid; r < R; r += kThreads) nrows[r] = rows_of_rank(p, tot, r);
-    __syncthreads();
-    finalize_chunk(p, t0, t1, ids_sm + (size_t)t0 * k, w_sm,
-                   [&](int e, int tl) { return eo[e] + pre[e] + bits_in_range(bmaps, e, t0, t0 + tl); },
-                   [&](int r, int tl) { return pre[p.E + r] + bits_in_range(bmaps, p.E + r, t0, t0 + tl); },
-                   true, c, order_sm, pos, key, nullptr, tid, kThreads);
+    if (kTable) {
+        local_counts_all_bins(p, ids_sm, bmaps, t0, tot, pre, eo, tid, kThreads, warp, kWarps, lane, 0);
+        for (int r = tid; r < R; r += kThreads) nrows[r] = rows_of_rank(p, tot, r);
+        __syncthreads();
+        finalize_chunk(p, t0, t1, ids_sm + (size_t)t0 * k, w_sm,
+                       [&](int e, int tl) { return eo[e] + pre[e] + bits_in_range(bmaps, e, t0, t0 + tl); },
+                       [&](int r, int tl) { return pre[p.E + r] + bits_in_range(bmaps, p.E + r, t0, t0 + tl); },
+                       true, c, order_sm, pos, key, nullptr, tid, kThreads);
+    } else {
+        build_bin_maps(p, ids_sm, ntok, bmaps, warp, kWarps, lane);
+        int* base_sm = hist;   // per bin: rows of all earlier chunks (+ the expert's offset in its region)
+        for (int b = tid; b < p.B; b += kThreads)
+            base_sm[b] = __ldcg(p.chunk_base + (size_t)b * p.nchunks + c) + (b < p.E ? __ldcg(p.expert_offset + b) : 0);
+        for (int r = tid; r < R; r += kThreads) nrows[r] = __ldcg(p.num_rows_per_rank + r);
+        __syncthreads();
+        finalize_chunk(p, t0, t1, ids_sm, w_sm,
+                       [&](int e, int tl) { return base_sm[e] + bits_in_range(bmaps, e, 0, tl); },
+                       [&](int r, int tl) { return base_sm[p.E + r] + bits_in_range(bmaps, p.E + r, 0, tl); },
+                       true, c, order_sm, pos, key, nullptr, tid, kThreads);
+    }
     __syncthreads();
     if (tid == 0) times[1] = global_ns();
-    // counts and offsets nobody inside this kernel waits for
-    if (c == 0) write_totals(p, tot, eo, tid, kThreads);
-    for (int s = c; s < p.S; s += p.grid) write_source_from_maps(p, s, bmaps, eo, tid, kThreads);
+    if (kTable) {
+        // counts and offsets nobody inside this kernel waits for (the launches before wrote them otherwise)
+        if (c == 0) write_totals(p, tot, eo, tid, kThreads);
+        for (int s = c; s < p.S; s += p.grid) write_source_from_maps(p, s, bmaps, eo, tid, kThreads);
+    }
 
     // ---- sender: the rows of tokens [t0, t1), one token at a time, all threads on a row
     const int wbytes = kFp8 ? p.H + 4 * p.G : p.rowB;   // bytes of one row on the wire
@@ -373,8 +392,9 @@ __global__ void __launch_bounds__(256) sentinel_scan_kernel(const uint4* __restr
 }
 
 template <int kProto>
-cudaError_t launch_one(const Params& p, const SmemPlan& pl, const SyncParams& sp, cudaStream_t st) {
-    auto kern = p.payload ? sync_dispatch_kernel<kProto, true> : sync_dispatch_kernel<kProto, false>;
+cudaError_t launch_one(const Params& p, const SmemPlan& pl, const SyncParams& sp, bool whole_table, cudaStream_t st) {
+    auto kern = whole_table ? (p.payload ? sync_dispatch_kernel<kProto, true, true> : sync_dispatch_kernel<kProto, false, true>)
+                            : (p.payload ? sync_dispatch_kernel<kProto, true, false> : sync_dispatch_kernel<kProto, false, false>);
     const int smem = pl.total + sync_extra_smem(p);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
@@ -400,12 +420,13 @@ int sync_extra_smem(const Params& p) {
     return p.R * 8 + 128 + qrow + 16;
 }
 
-cudaError_t launch_sync_dispatch(const Params& p, const SmemPlan& pl, const SyncParams& sp, cudaStream_t st) {
+cudaError_t launch_sync_dispatch(const Params& p, const SmemPlan& pl, const SyncParams& sp, bool whole_table,
+                                 cudaStream_t st) {
     switch (sp.protocol) {
-        case kSW: return launch_one<kSW>(p, pl, sp, st);
-        case kTFF: return launch_one<kTFF>(p, pl, sp, st);
-        case kDC: return launch_one<kDC>(p, pl, sp, st);
-        case kSP: return launch_one<kSP>(p, pl, sp, st);
+        case kSW: return launch_one<kSW>(p, pl, sp, whole_table, st);
+        case kTFF: return launch_one<kTFF>(p, pl, sp, whole_table, st);
+        case kDC: return launch_one<kDC>(p, pl, sp, whole_table, st);
+        case kSP: return launch_one<kSP>(p, pl, sp, whole_table, st);
         default: return cudaErrorInvalidValue;
     }
 }

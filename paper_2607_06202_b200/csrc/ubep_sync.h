@@ -28,7 +28,10 @@ struct SyncParams {
 // Dynamic shared memory the kernel needs beyond the dispatch plan's total.
 int sync_extra_smem(const Params& p);
 
-cudaError_t launch_sync_dispatch(const Params& p, const SmemPlan& pl, const SyncParams& sp, cudaStream_t st);
+// whole_table: every CTA derives the layout from the whole routing table in shared memory; otherwise the
+// count / prefix-sum launches (launch_count_scan) have run before over the same p.nchunks chunks.
+cudaError_t launch_sync_dispatch(const Params& p, const SmemPlan& pl, const SyncParams& sp, bool whole_table,
+                                 cudaStream_t st);
 
 // Counts the 16-byte vectors of x that consist of 0xFFFF elements only.
 cudaError_t launch_sentinel_scan(const void* x, long long n_vec, unsigned long long* count, int num_sms,

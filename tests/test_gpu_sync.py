@@ -32,6 +32,11 @@ CASES = {
     "fp8_dedup": W.Config("fp8_dedup", T=70, H=1024, E=32, R=8, k=4, payload=1, dedup=1, seed=4106),
     # the W8A8 row of the paper's Table 3: hidden 7168, 256 experts, top-8
     "fp8_w8a8": W.Config("fp8_w8a8", T=64, H=7168, E=256, R=32, k=8, payload=1, seed=4107),
+    # routing tables no CTA can recount alone (more than 8192 slots): counting and prefix sums are launches
+    # of their own in front of the protocol kernel
+    "large": W.Config("large", T=1500, H=256, E=32, R=8, k=8, seed=4108),
+    "large_fp8_dedup": W.Config("large_fp8_dedup", T=2100, H=256, E=64, R=16, k=8, payload=1, dedup=1, seed=4109),
+    "large_replicas": W.Config("large_replicas", T=3000, H=128, E=36, R=4, k=4, seed=4110, E_logical=32),
 }
 
 
@@ -223,12 +228,12 @@ def test_argument_errors():
     buf.attach_sync()
     with pytest.raises(B.UbepError):
         buf.dispatch_sync(7, x, idx, w)
-    big_T = 8192 // cfg.k + 1                       # beyond what every CTA can recount alone
+    big_T = 5001                                    # more tokens than the buffer was made for
     xb = torch.zeros((big_T, cfg.H), dtype=torch.bfloat16, device="cuda")
     ib = torch.zeros((big_T, cfg.k), dtype=torch.int32, device="cuda")
     wb = torch.zeros((big_T, cfg.k), dtype=torch.float32, device="cuda")
     with pytest.raises(B.UbepError) as e:
-        buf.dispatch_sync("sw", xb, ib, wb)
+        B.ubep_dispatch_sync(buf.handle, B.UBEP_SYNC_SW, xb, ib, wb, big_T)
     assert e.value.code == B.UBEP_ERR_ARG
     fp8 = dataclasses.replace(W.CONFIGS["tiny"], payload=1, H=256)
     fbuf = Hn.make_buffer(fp8, cap)
