@@ -1,6 +1,6 @@
 """Seeded random sweep over shapes, payloads, schedules, chunk counts, destination tables and empty
 slots: every case through the C ABI against the oracle (dispatch bit for bit, combine within the
-tolerance); small cases also through the readiness protocols and the sharded path."""
+tolerance), also through the readiness protocols and the sharded path."""
 import numpy as np
 import pytest
 import torch
@@ -41,8 +41,6 @@ def test_random_cases(seed):
     for _ in range(8):
         cfg, wl, pipeline, ctas, order = draw(rng)
         Hn.run_case(wl, pipeline=pipeline, num_ctas=ctas, dest_order=order)
-        if cfg.T * cfg.k > 8192:
-            continue
         ids, lay, cap, recv = Hn.oracle_reference(wl)
         x, idx, w, _, _ = Hn.device_inputs(wl)
         buf = Hn.make_buffer(cfg, cap, num_ctas=ctas)
